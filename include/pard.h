@@ -1,0 +1,208 @@
+/*
+ * pard.h -- C ABI of the PARD drop planner for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, for a snapshot of every stage queue of a DAG
+ * inference pipeline, the per-request keep/drop decision of PARD's State
+ * Planner and Request Broker (paper Sec. 4.2, Eq. 1-3), in the decision order
+ * of the low-budget-first priority queue (Sec. 4.3), then compacts the kept
+ * requests and counts goodput (Sec. 5.1, Metrics).
+ *
+ * Vocabulary: "stage" is the paper's module M_k; a "ctx" (context) is one
+ * independent planning problem (one pipeline instance at one decision epoch);
+ * a "segment" is the queue of one (ctx, stage).  segment id = ctx *
+ * stage_stride + stage.  All times are int64 microseconds on one clock.
+ *
+ * Pointers whose name starts with d_ are DEVICE pointers; every other pointer
+ * is a HOST pointer.  No function throws, aborts or prints; each returns
+ * PARD_OK (0) or a negative pard_status.  Entry points may be called from
+ * several host threads as long as they use distinct streams, workspaces and
+ * output buffers; a pipeline handle is immutable after loading.
+ */
+#ifndef PARD_H_
+#define PARD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- limits ------------------------------------------------------------ */
+#define PARD_MAX_STAGES      64        /* stages per pipeline                       */
+#define PARD_MAX_BATCH       4096      /* largest profiled batch size per stage     */
+#define PARD_MAX_PATH_SLOTS  65536     /* sum over stages of downstream paths       */
+#define PARD_MAX_PATH_LEN_SUM (1 << 20)/* sum of the lengths of all those paths     */
+#define PARD_MAX_REQUESTS    (1ull << 30) /* requests per pard_plan call            */
+#define PARD_MAX_SEGMENTS    (1u << 24)   /* n_ctx * stage_stride                   */
+#define PARD_TIME_LIMIT_US   (1ll << 60)  /* every time input lies in [0, 2^60)     */
+#define PARD_LAT_LIMIT_US    (1ll << 40)  /* every profile entry lies in [1, 2^40)  */
+
+/* ---- status codes ------------------------------------------------------ */
+typedef enum pard_status {
+  PARD_OK          =  0,
+  PARD_EINVAL      = -1,  /* null pointer, bad count, malformed CSR, bad flag        */
+  PARD_ECYCLE      = -2,  /* the stage graph has a cycle                             */
+  PARD_ERANGE      = -3,  /* a host-visible value is outside the limits above        */
+  PARD_ENOMEM      = -4,  /* host or device allocation failed (load time only)       */
+  PARD_EWORKSPACE  = -5,  /* caller's workspace is smaller than required             */
+  PARD_ETIMEOUT    = -6,  /* a bounded device-side wait ran out; outputs unspecified */
+  PARD_ECUDA       = -7,  /* a CUDA runtime call failed                              */
+  PARD_EDATA       = -8   /* device found ctx, stage or batch size out of range, or
+                             a deadline outside [0, 2^60); outputs unspecified       */
+} pard_status;
+
+const char* pard_strerror(int status);
+
+/* ---- pipeline description (Sec. 5.1, Implementation) -------------------
+ * The paper describes a pipeline as a list of modules (name, id, pres, subs).
+ * Here the ids are 0..n_stages-1 and only `subs` is given, as a CSR adjacency;
+ * `pres` is implied.  A stage without successors is a sink. */
+typedef struct pard_dag {
+  int32_t        n_stages;     /* 1..PARD_MAX_STAGES                                */
+  const int32_t* sub_offsets;  /* [n_stages+1], non-decreasing, sub_offsets[0] = 0  */
+  const int32_t* sub_ids;      /* [sub_offsets[n_stages]] successor ids; no self
+                                  loops, no duplicate edge                          */
+} pard_dag_t;
+
+/* Offline profile d_k(b): execution duration of stage k at batch size b
+ * (Sec. 4.2, State Planner, second bullet; Sec. 5.1, Implementation). */
+typedef struct pard_profile {
+  const int32_t* bmax;         /* [n_stages] largest profiled batch, 1..PARD_MAX_BATCH */
+  const int64_t* lat_offsets;  /* [n_stages+1]; lat_offsets[s+1]-lat_offsets[s] == bmax[s] */
+  const int64_t* lat_us;       /* lat_us[lat_offsets[s] + b - 1] = d_s(b), in [1, 2^40) */
+} pard_profile_t;
+
+typedef struct pard_pipeline pard_pipeline_t;   /* opaque, owned by the library */
+
+#define PARD_LOAD_HOST_ONLY 1u  /* build the host tables only (no CUDA call); such a
+                                   handle answers pard_pipeline_* queries but is
+                                   rejected by pard_plan with PARD_EINVAL           */
+
+/* Validates the graph (PARD_EINVAL / PARD_ECYCLE / PARD_ERANGE), enumerates for
+ * every stage k its downstream paths -- every stage sequence that starts at a
+ * successor of k and ends at a sink (Sec. 4.2: the estimate is taken along
+ * each subsequent DAG path) -- ordered lexicographically by stage-id sequence,
+ * and, unless PARD_LOAD_HOST_ONLY is set, copies the tables to the current
+ * CUDA device (one device allocation, released by pard_free_pipeline).
+ * Inputs are copied; the caller may free them on return. */
+int pard_load_pipeline(const pard_dag_t* dag, const pard_profile_t* profile,
+                       uint32_t flags, pard_pipeline_t** out);
+int pard_free_pipeline(pard_pipeline_t* pipeline);
+
+/* Path-slot layout.  Slot index of (stage k, its j-th downstream path) is
+ * slot_base(k) + j with slot_base(k) = number of downstream paths of all
+ * stages < k.  queue_state.w_us rows are indexed by slot.  */
+int pard_pipeline_n_stages(const pard_pipeline_t* p, int32_t* n_stages);
+int pard_pipeline_n_slots(const pard_pipeline_t* p, int32_t* n_slots);
+/* Returns HOST pointers into the handle (valid until pard_free_pipeline):
+ * path j of the stage is path_stage_ids[path_offsets[j] .. path_offsets[j+1]). */
+int pard_pipeline_paths(const pard_pipeline_t* p, int32_t stage,
+                        int32_t* n_paths, int32_t* slot_base,
+                        const int32_t** path_offsets, const int32_t** path_stage_ids);
+
+/* ---- requests and runtime state ----------------------------------------
+ * One queued request.  deadline_us = t_s + SLO: the send time of Eq. 3 plus
+ * the request's latency objective, so that "estimated latency exceeds the
+ * SLO" becomes "estimated completion time exceeds deadline_us". */
+typedef struct pard_request {
+  int64_t  deadline_us;   /* in [0, 2^60)                                            */
+  uint32_t ctx;           /* < n_ctx                                                 */
+  uint16_t stage;         /* stage whose queue holds the request, < n_stages         */
+  uint16_t flags;         /* reserved, ignored                                       */
+} pard_request_t;         /* 16 bytes, 16-byte aligned arrays                        */
+
+/* Runtime state the State Planner monitors and synchronises (Sec. 4.1, steps
+ * 1-3; Sec. 4.2).  All arrays are DEVICE memory, row-major per ctx. */
+typedef struct pard_queue_state {
+  int32_t        stage_stride;     /* row length of the [n_ctx][stage] arrays; >= every
+                                      used pipeline's n_stages, <= PARD_MAX_STAGES   */
+  int32_t        slot_stride;      /* row length of d_w_us; >= every used pipeline's
+                                      n_slots (ignored when d_w_us is NULL)          */
+  const int32_t* d_pipeline_of_ctx;/* [n_ctx] index into `pipelines`; NULL => 0      */
+  const int64_t* d_now_us;         /* [n_ctx] decision instant t_b of the snapshot   */
+  const int32_t* d_batch;          /* [n_ctx][stage_stride] current batch size B_k in
+                                      1..bmax[k]                                     */
+  const int64_t* d_free_at_us;     /* [n_ctx][stage_stride] expected end of the batch
+                                      now executing (t_e of the batch being formed)  */
+  const int64_t* d_q_us;           /* [n_ctx][stage_stride] recent average queueing
+                                      delay q_k                                      */
+  const int64_t* d_w_us;           /* [n_ctx][slot_stride] batch-wait estimate w per
+                                      (stage, downstream path) slot; NULL => 0       */
+  const int32_t* d_workers;        /* [n_ctx][stage_stride] identical workers m_k >= 1
+                                      draining the queue; NULL => 1                  */
+} pard_queue_state_t;
+
+/* Outputs of pard_plan, all DEVICE memory owned by the caller.  Per-request
+ * outputs are in service order: segments ascending, inside a segment by
+ * (deadline, original index) ascending.  A NULL member is not produced. */
+typedef struct pard_plan_out {
+  uint8_t*  d_keep;        /* [n]  1 = kept, 0 = dropped                             */
+  int64_t*  d_est_us;      /* [n]  estimated completion time t_s + L of Eq. 3        */
+  uint32_t* d_perm;        /* [n]  original index of the request at each position    */
+  uint32_t* d_kept_idx;    /* [n]  capacity; first *d_n_kept entries = original
+                                   indices of kept requests, in service order        */
+  uint64_t* d_n_kept;      /* [1]                                                    */
+  uint32_t* d_seg_offsets; /* [n_ctx*stage_stride + 1] first position of each segment */
+  uint32_t* d_seg_kept;    /* [n_ctx*stage_stride] kept requests per segment         */
+} pard_plan_out_t;
+
+#define PARD_MODE_ADMITTED 0u   /* a dropped request takes no batch slot (default)   */
+#define PARD_MODE_RAW      1u   /* every queued request ahead takes a batch slot     */
+
+/* Device scratch pard_plan needs for n requests in n_ctx contexts. */
+int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
+                              uint64_t* bytes);
+
+/* The planner (Sec. 4.2 Eq. 1-3, Sec. 4.3 low-budget-first order).
+ * For every segment, in ascending (deadline, index) order, with
+ *   d    = d_k(B_k)                         profile at the current batch size
+ *   cap  = B_k * m_k                        requests started per batch round
+ *   base = max(now, free_at_k)              start of the next batch to form
+ *   Lsub = 0 for a sink, else max over downstream paths P of
+ *          sum_{i in P} (q_i + d_i(B_i)) + w[slot(k,P)]
+ * a request at position c (kept requests ahead of it, or all requests ahead
+ * in PARD_MODE_RAW) gets est = base + floor(c/cap)*d + d + Lsub and is kept
+ * iff est <= deadline.
+ *
+ * `pipelines` is a host array of n_pipelines handles loaded on the current
+ * device.  d_requests is read only.  d_workspace must be 256-byte aligned and
+ * hold pard_plan_workspace_bytes() bytes; nothing in it survives the call.
+ * All work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default
+ * stream); the call then waits for the stream and reads back one status word,
+ * so a PARD_EDATA / PARD_ETIMEOUT found on the device is returned here.  The
+ * library allocates no device memory in this call.
+ * Host-detectable errors are returned before anything is launched. */
+int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+              const pard_request_t* d_requests, uint64_t n,
+              const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,
+              const pard_plan_out_t* out,
+              void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+
+/* Same computation with HOST inputs and outputs: `requests`, the arrays of
+ * `state` and the members of `out` are host pointers (pinned memory makes the
+ * copies asynchronous).  Inputs are copied to the device, planned, and the
+ * non-NULL outputs copied back, all on `cuda_stream`; the call returns after
+ * the stream has drained.  d_workspace must hold
+ * pard_plan_host_workspace_bytes() bytes. */
+int pard_plan_host_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
+                                   int32_t slot_stride, uint64_t* bytes);
+int pard_plan_host(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+                   const pard_request_t* requests, uint64_t n,
+                   const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,
+                   const pard_plan_out_t* out,
+                   void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+
+/* Goodput counters (Sec. 5.1, Metrics): per ctx, the number of queued
+ * requests and the number predicted to finish within their SLO (kept);
+ * dropped = total - kept, drop rate = dropped / total.  Reads d_keep and
+ * d_seg_offsets as produced by pard_plan; writes d_out_total[n_ctx] and
+ * d_out_kept[n_ctx] (overwritten, not accumulated).  Enqueued on cuda_stream;
+ * does not synchronise. */
+int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets,
+                 uint64_t n, uint32_t n_ctx, int32_t stage_stride,
+                 int64_t* d_out_total, int64_t* d_out_kept, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* PARD_H_ */

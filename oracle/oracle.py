@@ -1,0 +1,141 @@
+"""ctypes loader for the CPU oracle (test infrastructure only).
+
+Nothing in the product path imports this module; it is used by the tests, the
+smoke check and the benchmark's CPU-baseline leg.  Inputs are duck-typed: any
+object with the attributes used below (numpy arrays) is accepted, so that this
+module imports nothing but numpy.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libpard_oracle.so")
+_SRC = [os.path.join(_HERE, "pard_oracle.cpp"), os.path.join(_HERE, "pard_oracle.h")]
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ -O2 if the shared object is missing or stale."""
+    stale = (not os.path.exists(_SO)
+             or any(os.path.getmtime(s) > os.path.getmtime(_SO) for s in _SRC))
+    if force or stale:
+        tmp = _SO + ".tmp%d" % os.getpid()
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC",
+                               "-o", tmp, _SRC[0]])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+class _Pipeline(C.Structure):
+    _fields_ = [("n_stages", C.c_int32), ("sub_offsets", C.c_void_p),
+                ("sub_ids", C.c_void_p), ("bmax", C.c_void_p),
+                ("lat_offsets", C.c_void_p), ("lat_us", C.c_void_p)]
+
+
+class _State(C.Structure):
+    _fields_ = [("stage_stride", C.c_int32), ("slot_stride", C.c_int32),
+                ("pipeline_of_ctx", C.c_void_p), ("now_us", C.c_void_p),
+                ("batch", C.c_void_p), ("free_at_us", C.c_void_p),
+                ("q_us", C.c_void_p), ("w_us", C.c_void_p), ("workers", C.c_void_p)]
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.oracle_count_paths.restype = C.c_int64
+        _lib.oracle_count_paths.argtypes = [C.c_void_p, C.c_int32]
+        _lib.oracle_slot_base.restype = C.c_int64
+        _lib.oracle_slot_base.argtypes = [C.c_void_p, C.c_int32]
+        _lib.oracle_lsub.restype = C.c_int64
+        _lib.oracle_lsub.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib.oracle_plan.restype = C.c_int
+        _lib.oracle_plan.argtypes = ([C.c_void_p, C.c_int32, C.c_void_p, C.c_uint64,
+                                      C.c_void_p, C.c_uint32, C.c_uint32] + [C.c_void_p] * 9)
+    return _lib
+
+
+def _arr(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data
+
+
+class _Keep:
+    """Holds converted arrays alive next to the C struct that points at them."""
+
+    def __init__(self):
+        self.refs = []
+
+    def add(self, a, dtype):
+        if a is None:
+            return None
+        a = _arr(a, dtype)
+        self.refs.append(a)
+        return a.ctypes.data
+
+
+def _c_pipeline(p, keep: _Keep) -> _Pipeline:
+    return _Pipeline(int(p.n_stages), keep.add(p.sub_offsets, np.int32),
+                     keep.add(p.sub_ids, np.int32), keep.add(p.bmax, np.int32),
+                     keep.add(p.lat_offsets, np.int64), keep.add(p.lat_us, np.int64))
+
+
+def count_paths(p, stage: int) -> int:
+    k = _Keep()
+    cp = _c_pipeline(p, k)
+    return int(lib().oracle_count_paths(C.addressof(cp), stage))
+
+
+def slot_base(p, stage: int) -> int:
+    k = _Keep()
+    cp = _c_pipeline(p, k)
+    return int(lib().oracle_slot_base(C.addressof(cp), stage))
+
+
+def lsub(p, stage: int, batch_row, q_row, w_row=None) -> int:
+    k = _Keep()
+    cp = _c_pipeline(p, k)
+    return int(lib().oracle_lsub(C.addressof(cp), stage, k.add(batch_row, np.int32),
+                                 k.add(q_row, np.int64), k.add(w_row, np.int64)))
+
+
+def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:
+    """Runs the oracle planner; returns a dict of numpy outputs."""
+    k = _Keep()
+    cps = (_Pipeline * len(pipelines))(*[_c_pipeline(p, k) for p in pipelines])
+    req = np.ascontiguousarray(requests)
+    assert req.dtype.itemsize == 16
+    n = int(req.shape[0])
+    S = int(state.stage_stride)
+    cst = _State(S, int(state.slot_stride),
+                 k.add(state.pipeline_of_ctx, np.int32), k.add(state.now_us, np.int64),
+                 k.add(state.batch, np.int32), k.add(state.free_at_us, np.int64),
+                 k.add(state.q_us, np.int64), k.add(state.w_us, np.int64),
+                 k.add(state.workers, np.int32))
+    out = {
+        "keep": np.zeros(n, np.uint8), "est_us": np.zeros(n, np.int64),
+        "perm": np.zeros(n, np.uint32), "kept_idx": np.zeros(n, np.uint32),
+        "n_kept": np.zeros(1, np.uint64),
+        "seg_offsets": np.zeros(n_ctx * S + 1, np.uint32),
+        "seg_kept": np.zeros(n_ctx * S, np.uint32),
+        "ctx_total": np.zeros(n_ctx, np.int64), "ctx_kept": np.zeros(n_ctx, np.int64),
+    }
+    rc = lib().oracle_plan(C.addressof(cps), len(pipelines), req.ctypes.data, n,
+                           C.addressof(cst), n_ctx, mode,
+                           *[out[key].ctypes.data for key in
+                             ("keep", "est_us", "perm", "kept_idx", "n_kept",
+                              "seg_offsets", "seg_kept", "ctx_total", "ctx_kept")])
+    if rc != 0:
+        raise ValueError("oracle_plan: input out of range")
+    out["n_kept"] = int(out["n_kept"][0])
+    out["kept_idx"] = out["kept_idx"][:out["n_kept"]]
+    return out

@@ -1,0 +1,192 @@
+/*
+ * pard_oracle.cpp -- CPU oracle of the PARD drop planner.
+ *
+ * TEST INFRASTRUCTURE ONLY: plain, slow, single-threaded, written from the
+ * paper so that a reader can check it by eye.  It shares nothing with the CUDA
+ * library and no product path may call it.
+ *
+ * What it follows:
+ *   Eq. 1   L = L_pre + L_cur + L_sub                          (Sec. 4.2)
+ *   Eq. 2   Lat_k = Q_k + W_k + D_k                            (Sec. 4.2)
+ *   Eq. 3   L = (t_e - t_s + d_k) + (sum q_i + sum d_i + w_k)  (Sec. 4.2)
+ *   DAG:    the estimate is taken along every subsequent path and the
+ *           maximum is used                                     (Sec. 4.2, 5.1)
+ *   Order:  low budget first = smallest remaining budget first  (Sec. 4.3)
+ *   Rule:   drop when the estimate exceeds the latency objective (Sec. 5.3)
+ *   Counts: goodput / drop rate                                 (Sec. 5.1)
+ *
+ * Readings where the paper is silent (each also listed in the design notes):
+ *   - Snapshot: the Request Broker loop is run over the whole queue at the
+ *     instant `now`; batches of a stage run back to back, batch j starting at
+ *     base + j*d with base = max(now, free_at) (t_e chained forward).
+ *   - A dropped request never enters a batch, so the position that decides the
+ *     batch index counts kept requests only (mode 0).  Mode 1 counts all.
+ *   - d_k is the profile at the stage's current batch size for every batch.
+ *   - est == deadline is kept; equal deadlines are served in index order.
+ *   - w covers the stages after k; one value per (stage, downstream path).
+ *   - m identical workers drain one queue: a batch round starts B*m requests.
+ */
+#include "pard_oracle.h"
+
+#include <algorithm>
+#include <vector>
+
+namespace {
+
+int64_t profile_at(const oracle_pipeline_t* p, int32_t stage, int32_t b) {
+  return p->lat_us[p->lat_offsets[stage] + b - 1];
+}
+
+std::vector<int32_t> successors_ascending(const oracle_pipeline_t* p, int32_t stage) {
+  std::vector<int32_t> s(p->sub_ids + p->sub_offsets[stage],
+                         p->sub_ids + p->sub_offsets[stage + 1]);
+  std::sort(s.begin(), s.end());
+  return s;
+}
+
+/* Number of stage sequences that start at `stage` and end at a sink. */
+int64_t count_from(const oracle_pipeline_t* p, int32_t stage) {
+  std::vector<int32_t> s = successors_ascending(p, stage);
+  if (s.empty()) return 1;
+  int64_t c = 0;
+  for (int32_t j : s) c += count_from(p, j);
+  return c;
+}
+
+/* Walks every path that continues through `stage`.  `acc` is the sum of
+ * q_i + d_i(B_i) over the path's stages before this one.  Each time a sink is
+ * reached one complete path has been seen; paths are met in lexicographic
+ * order of their stage sequence, so the running counter `slot` is the path's
+ * w index. */
+int64_t walk(const oracle_pipeline_t* p, int32_t stage, int64_t acc,
+             const int32_t* batch_row, const int64_t* q_row,
+             const int64_t* w_row, int64_t* slot) {
+  acc += q_row[stage] + profile_at(p, stage, batch_row[stage]);
+  std::vector<int32_t> s = successors_ascending(p, stage);
+  if (s.empty()) {
+    int64_t w = w_row ? w_row[*slot] : 0;
+    *slot += 1;
+    return acc + w;
+  }
+  bool first = true;
+  int64_t best = 0;
+  for (int32_t j : s) {
+    int64_t v = walk(p, j, acc, batch_row, q_row, w_row, slot);
+    if (first || v > best) best = v;
+    first = false;
+  }
+  return best;
+}
+
+}  // namespace
+
+extern "C" int64_t oracle_count_paths(const oracle_pipeline_t* p, int32_t stage) {
+  std::vector<int32_t> s = successors_ascending(p, stage);
+  int64_t c = 0;
+  for (int32_t j : s) c += count_from(p, j);
+  return c;
+}
+
+extern "C" int64_t oracle_slot_base(const oracle_pipeline_t* p, int32_t stage) {
+  int64_t base = 0;
+  for (int32_t k = 0; k < stage; ++k) base += oracle_count_paths(p, k);
+  return base;
+}
+
+extern "C" int64_t oracle_lsub(const oracle_pipeline_t* p, int32_t stage,
+                               const int32_t* batch_row, const int64_t* q_row,
+                               const int64_t* w_row) {
+  std::vector<int32_t> s = successors_ascending(p, stage);
+  if (s.empty()) return 0;                       /* nothing after a sink */
+  int64_t slot = oracle_slot_base(p, stage);
+  bool first = true;
+  int64_t best = 0;
+  for (int32_t j : s) {
+    int64_t v = walk(p, j, 0, batch_row, q_row, w_row, &slot);
+    if (first || v > best) best = v;
+    first = false;
+  }
+  return best;
+}
+
+extern "C" int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                           const oracle_request_t* requests, uint64_t n,
+                           const oracle_state_t* st, uint32_t n_ctx, uint32_t mode,
+                           uint8_t* keep, int64_t* est_us, uint32_t* perm,
+                           uint32_t* kept_idx, uint64_t* n_kept,
+                           uint32_t* seg_offsets, uint32_t* seg_kept,
+                           int64_t* ctx_total, int64_t* ctx_kept) {
+  const int64_t S = st->stage_stride;
+  /* one queue per (ctx, stage), filled in arrival (index) order */
+  std::vector<std::vector<uint32_t>> queue((size_t)n_ctx * S);
+  for (uint64_t i = 0; i < n; ++i) {
+    const oracle_request_t& r = requests[i];
+    if (r.ctx >= n_ctx) return -1;
+    int32_t pi = st->pipeline_of_ctx ? st->pipeline_of_ctx[r.ctx] : 0;
+    if (pi < 0 || pi >= n_pipelines) return -1;
+    if (r.stage >= pipelines[pi].n_stages) return -1;
+    queue[(size_t)r.ctx * S + r.stage].push_back((uint32_t)i);
+  }
+
+  uint64_t pos = 0;        /* position in service order */
+  uint64_t kept_all = 0;
+  for (uint32_t c = 0; c < n_ctx; ++c) {
+    int32_t pi = st->pipeline_of_ctx ? st->pipeline_of_ctx[c] : 0;
+    if (pi < 0 || pi >= n_pipelines) return -1;
+    const oracle_pipeline_t* p = &pipelines[pi];
+    const int32_t* batch_row = st->batch + (size_t)c * S;
+    const int64_t* q_row = st->q_us + (size_t)c * S;
+    const int64_t* free_row = st->free_at_us + (size_t)c * S;
+    const int64_t* w_row = st->w_us ? st->w_us + (size_t)c * st->slot_stride : nullptr;
+    const int32_t* m_row = st->workers ? st->workers + (size_t)c * S : nullptr;
+    int64_t total_c = 0, kept_c = 0;
+
+    for (int32_t k = 0; k < S; ++k) {
+      std::vector<uint32_t>& qk = queue[(size_t)c * S + k];
+      if (seg_offsets) seg_offsets[(size_t)c * S + k] = (uint32_t)pos;
+      if (k >= p->n_stages) {                    /* padding column of the row */
+        if (seg_kept) seg_kept[(size_t)c * S + k] = 0;
+        continue;
+      }
+      int32_t B = batch_row[k];
+      if (B < 1 || B > p->bmax[k]) return -1;
+      int64_t m = m_row ? m_row[k] : 1;
+      if (m < 1) return -1;
+      int64_t d = profile_at(p, k, B);           /* D_k = d_k at the current batch size */
+      int64_t cap = (int64_t)B * m;
+      int64_t base = std::max(st->now_us[c], free_row[k]);   /* t_e of the next batch */
+      int64_t lsub = oracle_lsub(p, k, batch_row, q_row, w_row);
+
+      /* low budget first: smallest deadline first, ties in index order */
+      std::stable_sort(qk.begin(), qk.end(), [&](uint32_t a, uint32_t b) {
+        return requests[a].deadline_us < requests[b].deadline_us;
+      });
+
+      int64_t kept = 0, raw = 0;
+      for (uint32_t i : qk) {                    /* the Request Broker, one request at a time */
+        int64_t ahead = (mode & 1u) ? raw : kept;
+        int64_t t_e = base + (ahead / cap) * d;  /* its batch starts when the previous one ends */
+        int64_t est = t_e + d + lsub;            /* t_s + L of Eq. 3 */
+        bool k_ = est <= requests[i].deadline_us;
+        if (keep) keep[pos] = k_ ? 1 : 0;
+        if (est_us) est_us[pos] = est;
+        if (perm) perm[pos] = i;
+        if (k_) {
+          if (kept_idx) kept_idx[kept_all] = i;
+          ++kept_all;
+          ++kept;
+        }
+        ++raw;
+        ++pos;
+      }
+      if (seg_kept) seg_kept[(size_t)c * S + k] = (uint32_t)kept;
+      total_c += raw;
+      kept_c += kept;
+    }
+    if (ctx_total) ctx_total[c] = total_c;
+    if (ctx_kept) ctx_kept[c] = kept_c;
+  }
+  if (seg_offsets) seg_offsets[(size_t)n_ctx * S] = (uint32_t)pos;
+  if (n_kept) *n_kept = kept_all;
+  return 0;
+}

@@ -1,0 +1,85 @@
+/*
+ * pard_oracle.h -- interface of the CPU oracle for the PARD drop planner.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, single-threaded statement
+ * of what the planner computes, written from the paper (Sec. 4.2 Eq. 1-3,
+ * Sec. 4.3, Sec. 5.1).  It exists so that tests can compare the CUDA library
+ * with it; it shares no code, header or table with that library, and no
+ * product path may call it.
+ *
+ * All pointers are host pointers.  Times are int64 microseconds.
+ */
+#ifndef PARD_ORACLE_H_
+#define PARD_ORACLE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* One pipeline: the stage graph (successor lists, CSR) and the offline
+ * latency profile d_k(b), b = 1..bmax[k] (Sec. 5.1, Implementation). */
+typedef struct oracle_pipeline {
+  int32_t        n_stages;
+  const int32_t* sub_offsets;   /* [n_stages+1] */
+  const int32_t* sub_ids;       /* successors   */
+  const int32_t* bmax;          /* [n_stages]   */
+  const int64_t* lat_offsets;   /* [n_stages+1] */
+  const int64_t* lat_us;        /* d_k(b) at lat_offsets[k] + b - 1 */
+} oracle_pipeline_t;
+
+/* A queued request: deadline = send time t_s + SLO. 16 bytes. */
+typedef struct oracle_request {
+  int64_t  deadline_us;
+  uint32_t ctx;
+  uint16_t stage;
+  uint16_t flags;
+} oracle_request_t;
+
+/* Runtime state, row-major per ctx; rows have stage_stride / slot_stride
+ * entries.  pipeline_of_ctx, w_us and workers may be NULL (=> 0, 0, 1). */
+typedef struct oracle_state {
+  int32_t        stage_stride;
+  int32_t        slot_stride;
+  const int32_t* pipeline_of_ctx;
+  const int64_t* now_us;
+  const int32_t* batch;
+  const int64_t* free_at_us;
+  const int64_t* q_us;
+  const int64_t* w_us;
+  const int32_t* workers;
+} oracle_state_t;
+
+/* Number of downstream paths of `stage` (0 for a sink). */
+int64_t oracle_count_paths(const oracle_pipeline_t* p, int32_t stage);
+
+/* First w slot of `stage`: downstream paths of all stages before it. */
+int64_t oracle_slot_base(const oracle_pipeline_t* p, int32_t stage);
+
+/* L_sub of Eq. 3 for one (ctx row, stage): the maximum over the stage's
+ * downstream paths of sum (q_i + d_i(B_i)) + w[slot]; 0 at a sink.
+ * batch_row/q_row have n_stages entries, w_row is the ctx's slot row or NULL. */
+int64_t oracle_lsub(const oracle_pipeline_t* p, int32_t stage,
+                    const int32_t* batch_row, const int64_t* q_row,
+                    const int64_t* w_row);
+
+/* The planner.  mode bit 0: 0 = a dropped request takes no batch slot,
+ * 1 = every request ahead takes one.  Outputs (any may be NULL):
+ *   keep[n], est_us[n], perm[n]      in service order
+ *   kept_idx[n], *n_kept             original indices of kept requests
+ *   seg_offsets[n_ctx*stage_stride+1], seg_kept[n_ctx*stage_stride]
+ *   ctx_total[n_ctx], ctx_kept[n_ctx]
+ * Returns 0, or -1 when an input is out of range. */
+int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                const oracle_request_t* requests, uint64_t n,
+                const oracle_state_t* state, uint32_t n_ctx, uint32_t mode,
+                uint8_t* keep, int64_t* est_us, uint32_t* perm,
+                uint32_t* kept_idx, uint64_t* n_kept,
+                uint32_t* seg_offsets, uint32_t* seg_kept,
+                int64_t* ctx_total, int64_t* ctx_kept);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* PARD_ORACLE_H_ */

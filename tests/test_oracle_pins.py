@@ -150,6 +150,17 @@ def test_batches_of_B_share_a_start_time():
     assert list(o["est_us"]) == [100] * 8 + [200] * 2
 
 
+def test_duration_is_the_profile_at_the_current_batch_size():
+    """D_k = d_k at the current batch size (Sec. 4.2 Request Broker, third
+    bullet), for the stage itself as well as downstream."""
+    p = inputs.make_pipeline([], 1, [4], [np.array([100, 150, 200, 250])])
+    r = util.requests(10**6 + np.arange(7))
+    for B, d in ((1, 100), (3, 200), (4, 250)):
+        st = util.state(1, 1, 0, 0, B, free_at=0)
+        o = oracle.plan([p], r, st, 1)
+        assert list(o["est_us"]) == [d * (i // B + 1) for i in range(7)]
+
+
 def test_drop_wrong_set_example():
     """Sec. 3.2 Observation #2: W = t_e - t_b; and a dropped request takes no
     batch slot, so dropping R1..R4 lets R5..R8 ride the first batch."""

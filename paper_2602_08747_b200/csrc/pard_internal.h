@@ -1,0 +1,55 @@
+/* Internal declarations shared by the translation units of libpard. */
+#ifndef PARD_INTERNAL_H_
+#define PARD_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "pard.h"
+
+/* Device-resident tables of one pipeline.  The struct itself is the first
+ * bytes of the pipeline's single device allocation; its pointers point into
+ * the same allocation. */
+struct PardPipeDev {
+  int32_t n_stages;
+  int32_t n_slots;
+  const int32_t* bmax;            /* [S]                                        */
+  const int64_t* lat_offsets;     /* [S+1]                                      */
+  const int64_t* lat_us;          /* profile entries                            */
+  const int32_t* stage_slot_off;  /* [S+1] slots of stage k: [off[k], off[k+1]) */
+  const int32_t* path_off;        /* [n_slots+1] into path_stage                */
+  const int32_t* path_stage;      /* concatenated stage ids of all paths        */
+};
+
+struct pard_pipeline {
+  int32_t n_stages = 0;
+  int32_t n_slots = 0;
+  std::vector<int32_t> bmax;
+  std::vector<int64_t> lat_offsets;
+  std::vector<int64_t> lat_us;
+  std::vector<int32_t> stage_slot_off;          /* [S+1]                        */
+  std::vector<int32_t> path_off;                /* [n_slots+1], global offsets  */
+  std::vector<int32_t> path_stage;
+  std::vector<std::vector<int32_t>> local_off;  /* per stage, offsets rebased to 0 */
+  int device = -1;                              /* -1: host only                */
+  void* d_blob = nullptr;                       /* PardPipeDev + tables         */
+};
+
+/* Per-segment constants (Eq. 3 terms that do not depend on the request). */
+struct __align__(16) PardSegConst {
+  int64_t A;        /* base + d_k(B_k) + L_sub : estimate of a request at position 0 */
+  int64_t A_rel;    /* A - (smallest deadline of the segment's ctx)                  */
+  int64_t d;        /* d_k(B_k)                                                      */
+  uint32_t cap;     /* min(B_k * m_k, 2^30)                                          */
+  uint32_t pad;
+};
+
+#define PARD_CUDA_OK(expr)                    \
+  do {                                        \
+    cudaError_t e__ = (expr);                 \
+    if (e__ != cudaSuccess) return PARD_ECUDA; \
+  } while (0)
+
+#endif  /* PARD_INTERNAL_H_ */

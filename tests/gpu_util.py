@@ -1,0 +1,52 @@
+"""Runs a workload through the C-ABI CUDA library and returns numpy outputs."""
+from __future__ import annotations
+
+import numpy as np
+
+from paper_2602_08747_b200 import binding as pb
+from paper_2602_08747_b200 import build as pbuild
+
+
+def run_library(wl, mode=0, check=True):
+    import torch
+    pbuild.build()
+    assert torch.cuda.is_available()
+    dev = "cuda:0"
+    pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
+    S = wl.state.stage_stride
+    n_seg = wl.n_ctx * S
+    d_req = pb.device_requests(wl.requests, dev)
+    d_state = pb.device_state(wl.state, dev)
+    out = pb.alloc_out(wl.n, n_seg, dev)
+    ws = pb.alloc_workspace(pb.pard_plan_workspace_bytes(wl.n, wl.n_ctx, S), dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    rc = pb.pard_plan(pipes, d_req, wl.n, d_state, wl.n_ctx, mode, out, ws, stream=stream, check=check)
+    if rc != pb.PARD_OK:
+        return rc, None
+    total = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
+    kept = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
+    pb.pard_goodput(out.keep, out.seg_offsets, wl.n, wl.n_ctx, S, total, kept, stream=stream)
+    torch.cuda.synchronize()
+    res = pb.out_to_numpy(out, wl.n)
+    res["ctx_total"] = total.cpu().numpy()
+    res["ctx_kept"] = kept.cpu().numpy()
+    for p in pipes:
+        p.free()
+    return rc, res
+
+
+KEYS = ["seg_offsets", "perm", "keep", "est_us", "n_kept", "kept_idx", "seg_kept", "ctx_total", "ctx_kept"]
+
+
+def assert_identical(got, want):
+    """Bit-exact comparison of every output (all of them are integers)."""
+    for k in KEYS:
+        g, w = got[k], want[k]
+        if isinstance(w, (int, np.integer)):
+            assert int(g) == int(w), k
+        else:
+            assert g.shape == w.shape, (k, g.shape, w.shape)
+            if not np.array_equal(g, w):
+                bad = np.flatnonzero(g != w)
+                raise AssertionError("%s differs at %d positions, first %d: got %s want %s"
+                                     % (k, bad.size, bad[0], g[bad[0]], w[bad[0]]))

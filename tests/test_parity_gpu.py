@@ -1,0 +1,216 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle, element
+by element and bit for bit, on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2602_08747_b200 import binding as pb
+from paper_2602_08747_b200 import inputs
+from tests import util
+from tests.gpu_util import assert_identical, run_library
+
+pytestmark = pytest.mark.gpu
+
+
+def both(wl, mode=0):
+    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, mode)
+    rc, got = run_library(wl, mode)
+    assert rc == 0
+    assert_identical(got, want)
+    return got
+
+
+# sizes chosen to span several tiles of both the sort (4096) and the decision
+# pass (2048) and to leave a ragged tail
+@pytest.mark.parametrize("name,kw", [
+    ("C1", {}), ("C1b", {}),
+    ("C1", {"n": 1}), ("C1", {"n": 2047}), ("C1", {"n": 2049}), ("C1b", {"n": 12345}),
+    ("C2", {"n": 100_003}), ("C2b", {"n": 100_003}),
+    ("C3", {"n": 70_001}), ("C3b", {"n": 300_007}),
+    ("C4", {"n_epochs": 37, "per_epoch": 1000}), ("C4b", {"n_epochs": 64, "per_epoch": 8192}),
+    ("C5", {"n_inst": 9, "per_inst": 5001}), ("C5b", {"n_inst": 16, "per_inst": 65536}),
+])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_configs_reduced(name, kw, mode):
+    both(inputs.make(name, **kw), mode)
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_random_small_workloads(seed):
+    rng = np.random.default_rng(900 + seed)
+    n = int(rng.integers(1, 9000))
+    wl = util.random_small_workload(rng, n, n_ctx=int(rng.integers(1, 6)))
+    both(wl, mode=seed & 1)
+
+
+def _one_stage(n, deadline, d=10, B=2, free_at=0, now=0, workers=None):
+    p = util.pipeline([], 1, [d], bmax=max(B, 1))
+    st = util.state(1, 1, 0, now, B, free_at=free_at, workers=workers)
+    return inputs.Workload("edge", [p], util.requests(deadline), st, 1)
+
+
+def test_all_deadlines_equal():
+    both(_one_stage(5000, np.full(5000, 1000)))
+    both(_one_stage(5000, np.full(5000, 10_000)))
+
+
+def test_all_expired_and_all_kept():
+    got = both(_one_stage(6000, np.arange(6000) % 7, now=10_000))
+    assert got["n_kept"] == 0
+    got = both(_one_stage(6000, 10**12 + np.arange(6000)[::-1]))
+    assert got["n_kept"] == 6000
+
+
+def test_batch_one_and_batch_max_and_many_workers():
+    rng = np.random.default_rng(5)
+    dl = rng.integers(0, 40_000, size=9000)
+    both(_one_stage(9000, dl, B=1, d=7))
+    both(_one_stage(9000, dl, B=4096, d=7))
+    both(_one_stage(9000, dl, B=3, d=7, workers=2**31 - 1))
+
+
+def test_threshold_exactly_at_tile_and_warp_boundaries():
+    # u jumps by cap at positions that land on 32, 256, 2048 and 4096
+    for B in (32, 256, 2048, 4096):
+        dl = np.repeat(np.arange(1, 6) * 100, B)     # B requests per batch deadline
+        both(_one_stage(len(dl), dl, d=100, B=B))
+        both(_one_stage(len(dl), dl - 1, d=100, B=B))
+
+
+def test_segment_boundaries_on_tile_boundaries_and_empty_segments():
+    p = util.pipeline(inputs.chain_edges(5), 5, [3, 4, 5, 6, 7], bmax=4)
+    st = util.state(3, 5, inputs.n_slots(p), [100, 200, 300], 2, q=1, w=2)
+    rng = np.random.default_rng(6)
+    # queue lengths that are multiples of the tile sizes, with empty queues and an empty ctx
+    lens = {(0, 0): 2048, (0, 1): 4096, (0, 3): 2048, (2, 0): 6144, (2, 4): 1}
+    dl, stg, ctx = [], [], []
+    for (c, k), m in lens.items():
+        dl.append(rng.integers(0, 4000, size=m)); stg.append(np.full(m, k)); ctx.append(np.full(m, c))
+    order = rng.permutation(sum(lens.values()))
+    r = util.requests(np.concatenate(dl)[order], stage=np.concatenate(stg)[order],
+                      ctx=np.concatenate(ctx)[order])
+    got = both(inputs.Workload("edge", [p], r, st, 3))
+    assert list(got["ctx_total"]) == [8192, 0, 6145]
+
+
+def test_zero_requests():
+    p = util.pipeline(inputs.chain_edges(2), 2, [5, 6])
+    st = util.state(3, 2, 1, 10, 1)
+    got = both(inputs.Workload("edge", [p], util.requests([]), st, 3))
+    assert got["n_kept"] == 0
+
+
+def test_large_times_use_the_64_bit_division():
+    # deadlines and durations beyond 2^32 us
+    d = (1 << 35) + 12345
+    p = util.pipeline([], 1, [d], bmax=2)
+    now = 1 << 50
+    st = util.state(1, 1, 0, now, 2, free_at=now + 17)
+    rng = np.random.default_rng(7)
+    dl = now + rng.integers(0, 40 * d, size=7000)
+    both(inputs.Workload("edge", [p], util.requests(dl), st, 1))
+
+
+def test_wide_deadline_span():
+    # 2^44 us between the earliest and the latest deadline: 6 radix passes
+    rng = np.random.default_rng(8)
+    dl = rng.integers(0, 1 << 44, size=20_000)
+    both(_one_stage(20_000, dl, d=1 << 30, B=4, now=0))
+
+
+def test_multiple_pipelines_and_padded_rows():
+    rng = np.random.default_rng(9)
+    pa = util.pipeline(inputs.chain_edges(2), 2, [30, 40])
+    pbig = util.pipeline([(0, 1), (0, 2), (1, 3), (2, 3)], 4, [10, 20, 50, 5])
+    n_ctx = 5
+    poc = [1, 0, 1, 1, 0]
+    S, R = 6, 9                                    # wider rows than any pipeline needs
+    st = util.state(n_ctx, S, R, rng.integers(100, 200, size=n_ctx), 2,
+                    free_at=rng.integers(100, 300, size=(n_ctx, S)),
+                    q=rng.integers(0, 9, size=(n_ctx, S)), w=rng.integers(0, 30, size=(n_ctx, R)), poc=poc)
+    n = 30_000
+    ctx = rng.integers(0, n_ctx, size=n)
+    stage = np.where(np.asarray(poc)[ctx] == 0, rng.integers(0, 2, size=n), rng.integers(0, 4, size=n))
+    r = util.requests(rng.integers(100, 3000, size=n), stage=stage, ctx=ctx)
+    both(inputs.Workload("edge", [pa, pbig], r, st, n_ctx))
+
+
+def test_device_detected_errors():
+    p = util.pipeline(inputs.chain_edges(2), 2, [5, 6])
+    good = util.requests(np.arange(3000) + 100)
+    st = util.state(1, 2, 1, 10, 1)
+    for bad_field, bad_val in (("stage", 2), ("ctx", 1), ("deadline_us", -5), ("deadline_us", 1 << 60)):
+        r = good.copy()
+        r[bad_field][1234] = bad_val
+        rc, _ = run_library(inputs.Workload("bad", [p], r, st, 1), check=False)
+        assert rc == pb.PARD_EDATA, bad_field
+    rc, _ = run_library(inputs.Workload("bad", [p], good, util.state(1, 2, 1, 10, 5), 1), check=False)
+    assert rc == pb.PARD_EDATA
+    rc, _ = run_library(inputs.Workload("bad", [p], good, util.state(1, 2, 1, 10, 1, workers=0), 1), check=False)
+    assert rc == pb.PARD_EDATA
+    # a request queued at a stage its pipeline does not have (row is wider than the pipeline)
+    r = good.copy()
+    r["stage"][7] = 2
+    rc, _ = run_library(inputs.Workload("bad", [p], r, util.state(1, 3, 1, 10, 1), 1), check=False)
+    assert rc == pb.PARD_EDATA
+    # the context still works afterwards
+    both(inputs.Workload("ok", [p], good, st, 1))
+
+
+def test_key_wider_than_64_bits_is_reported():
+    # 2^59 span * 2^14 requests * 64 segments does not fit one 64-bit sort element
+    p = util.pipeline(inputs.chain_edges(2), 2, [5, 6])
+    n = 10_000
+    dl = np.arange(n, dtype=np.int64)
+    dl[-1] = (1 << 59)
+    st = util.state(32, 2, 1, 10, 1)
+    rc, _ = run_library(inputs.Workload("wide", [p], util.requests(dl), st, 32), check=False)
+    assert rc == pb.PARD_ERANGE
+
+
+def test_workspace_too_small_and_foreign_handle():
+    import torch
+    wl = inputs.make("C1")
+    pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
+    need = pb.pard_plan_workspace_bytes(wl.n, 1, 3)
+    ws = pb.alloc_workspace(need)
+    out = pb.alloc_out(wl.n, 3)
+    d_req, d_st = pb.device_requests(wl.requests), pb.device_state(wl.state)
+    assert pb.pard_plan(pipes, d_req, wl.n, d_st, 1, 0, out, ws, workspace_bytes=need - 1,
+                        check=False) == pb.PARD_EWORKSPACE
+    host_only = pb.pard_load_pipeline(wl.pipelines[0], host_only=True)
+    assert pb.pard_plan([host_only], d_req, wl.n, d_st, 1, 0, out, ws, check=False) == pb.PARD_EINVAL
+    torch.cuda.synchronize()
+
+
+def test_host_buffer_entry_point_matches():
+    import torch
+    wl = inputs.make("C2b", n=150_001)
+    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
+    pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
+    st = wl.state
+    S, R = st.stage_stride, st.slot_stride
+    n_seg = wl.n_ctx * S
+    hs = pb.QueueStateArrays(S, R, st.now_us, st.batch, st.free_at_us, st.q_us, st.w_us, st.workers,
+                             st.pipeline_of_ctx)
+    out = pb.PlanOut(np.zeros(wl.n, np.uint8), np.zeros(wl.n, np.int64), np.zeros(wl.n, np.uint32),
+                     np.zeros(wl.n, np.uint32), np.zeros(1, np.uint64),
+                     np.zeros(n_seg + 1, np.uint32), np.zeros(n_seg, np.uint32))
+    ws = pb.alloc_workspace(pb.pard_plan_host_workspace_bytes(wl.n, wl.n_ctx, S, R))
+    req = np.ascontiguousarray(wl.requests)
+    pb.pard_plan_host(pipes, req, wl.n, hs, wl.n_ctx, 0, out, ws,
+                      stream=torch.cuda.current_stream().cuda_stream)
+    nk = int(out.n_kept[0])
+    assert nk == want["n_kept"]
+    assert np.array_equal(out.keep, want["keep"])
+    assert np.array_equal(out.est_us, want["est_us"])
+    assert np.array_equal(out.perm, want["perm"])
+    assert np.array_equal(out.kept_idx[:nk], want["kept_idx"])
+    assert np.array_equal(out.seg_offsets, want["seg_offsets"])
+    assert np.array_equal(out.seg_kept, want["seg_kept"])
+
+
+# full sizes, in the launch configuration the benchmark times
+@pytest.mark.parametrize("name", ["C2", "C3", "C3b", "C4", "C5"])
+def test_configs_full_size(name):
+    both(inputs.make(name))

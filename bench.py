@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the PARD drop planner on B200.
+
+One step = one pass of the whole hot path (pard_plan + pard_goodput) over one
+snapshot of the 16-stage / 12-path / 2^24-request workload ("C3").  Prints ONE
+JSON line.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_08747_b200 import inputs  # noqa: E402
+
+METRIC = "requests_planned_per_sec"
+UNIT = "requests/s"
+WORKLOAD = "C3"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index, period_s=0.01):
+        super().__init__(daemon=True)
+        self.index, self.period, self.stop_flag = index, period_s, threading.Event()
+        self.sm, self.reasons, self.max_mhz, self.err = [], set(), None, None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+                getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            }
+            get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            while not self.stop_flag.is_set():
+                self.sm.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                bits = get(h)
+                for bit, name in names.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception as e:  # NVML missing: report it, do not fail the bench
+            self.err = repr(e)
+
+    def result(self):
+        self.stop_flag.set()
+        self.join(timeout=2)
+        out = {"sm_mhz": statistics.median(self.sm) if self.sm else None,
+               "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.sm)}
+        if self.err:
+            out["error"] = self.err
+        return out
+
+
+def physical_gpu_index(local):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# --------------------------------------------------------------------------
+def time_oracle(wl, repeats):
+    from oracle import oracle
+    best = None
+    for _ in range(repeats):
+        t = time.perf_counter()
+        o = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
+        dt = time.perf_counter() - t
+        best = dt if best is None else min(best, dt)
+    return best, o
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores; each step plans a bounded
+    sample (a smaller draw of the same workload)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n = 1 << 22 if args.steps + args.warmup <= 100 else 1 << 20
+    wl = inputs.make(WORKLOAD, n=n)
+    from oracle import oracle
+    for _ in range(args.warmup):
+        oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
+    dt = time.perf_counter() - t0
+    value = wl.n * args.steps / dt
+    sample = "%s workload drawn at n=%d requests per step" % (WORKLOAD, n)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "requests_per_step": n, "stages": 16, "paths": 12,
+                   "note": "CPU oracle (single thread) on a bounded sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": os.cpu_count()},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------
+class DevicePlan:
+    """Device-resident workload, outputs and workspace for repeated planning."""
+
+    def __init__(self, wl, dev):
+        import torch
+        from paper_2602_08747_b200 import binding as pb
+        self.pb, self.torch, self.wl, self.dev = pb, torch, wl, dev
+        self.S = wl.state.stage_stride
+        self.n_seg = wl.n_ctx * self.S
+        self.pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
+        self.d_req = pb.device_requests(wl.requests, dev)
+        self.d_state = pb.device_state(wl.state, dev)
+        self.out = pb.alloc_out(wl.n, self.n_seg, dev)
+        self.ws = pb.alloc_workspace(pb.pard_plan_workspace_bytes(wl.n, wl.n_ctx, self.S), dev)
+        self.total = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
+        self.kept = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
+        self.stream = torch.cuda.current_stream().cuda_stream
+        self.launches = pb.pard_plan_kernel_launches(wl.n, wl.n_ctx, self.S) + 2
+
+    def step(self, nowait=True):
+        pb, wl = self.pb, self.wl
+        pb.pard_plan(self.pipes, self.d_req, wl.n, self.d_state, wl.n_ctx,
+                     pb.PARD_MODE_NOWAIT if nowait else 0, self.out, self.ws, stream=self.stream)
+        pb.pard_goodput(self.out.keep, self.out.seg_offsets, wl.n, wl.n_ctx, self.S, self.total,
+                        self.kept, stream=self.stream)
+
+    def status(self):
+        return self.pb.pard_plan_status(self.ws, self.stream)
+
+
+def timed_steps(plan, steps, warmup, dist, profile_every=None):
+    """K steps between two CUDA events on the launching stream; returns seconds
+    (max over ranks) and the phase profile."""
+    torch, pb = plan.torch, plan.pb
+    for _ in range(warmup):
+        plan.step()
+    plan.status()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    if profile_every:
+        pb.pard_profile_begin(profile_every, max(1, steps // profile_every + 1))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        plan.step()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    plan.status()
+    prof = pb.pard_profile_end() if profile_every else None
+    sec = e0.elapsed_time(e1) / 1e3
+    if dist is not None:
+        t = torch.tensor([sec], dtype=torch.float64, device=plan.dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+    return sec, prof
+
+
+def kernel_table(prof, n, keep_frac, peak):
+    """Per-kernel average duration and achieved algorithmic GB/s from the phase events."""
+    k = prof["n_samples"]
+    ms = prof["ms"]
+    sort_names = [s for s in ms if s.startswith("sort")]
+    sort_active = [s for s in sort_names if ms[s] / k > 0.02]       # passes that really ran
+    rows = {}
+
+    def add(name, total_ms, launches, bytes_per_req):
+        if launches == 0:
+            return
+        per = total_ms / k / launches
+        gbs = bytes_per_req * n / (per * 1e-3) / 1e9 if per > 0 else None
+        rows[name] = {"launches_per_step": launches, "ms_per_launch": per,
+                      "algorithmic_bytes_per_request": bytes_per_req, "achieved_gbs": gbs,
+                      "frac": gbs / peak if gbs else None, "ms_per_step": total_ms / k}
+    add("k_prepass", ms["prepass"], 1, 16.0)
+    add("k_pack", ms["pack"], 1, 24.0)
+    add("k_sort_pass", sum(ms[s] for s in sort_active), len(sort_active), 16.0)
+    add("k_decide", ms["decide"], 1, 21.0 + 4.0 * keep_frac)
+    other = ms["clear"] + ms["segments"] + sum(ms[s] for s in sort_names if s not in sort_active)
+    rows["other"] = {"ms_per_step": other / k}
+    return rows
+
+
+def run_e2e(wl, dev, steps, dist):
+    """The same metric through pard_plan_host: pinned host inputs and outputs,
+    copies inside the timed region."""
+    import torch
+    from paper_2602_08747_b200 import binding as pb
+    st = wl.state
+    S, R = st.stage_stride, st.slot_stride
+    n, n_seg = wl.n, wl.n_ctx * S
+    pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
+
+    def pin(a, dt):
+        if a is None:
+            return None
+        t = torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).pin_memory()
+        return t
+
+    req = torch.from_numpy(np.ascontiguousarray(wl.requests).view(np.uint8).reshape(-1, 16)).pin_memory()
+    hs = pb.QueueStateArrays(S, R, pin(st.now_us, np.int64), pin(st.batch, np.int32),
+                             pin(st.free_at_us, np.int64), pin(st.q_us, np.int64),
+                             pin(st.w_us, np.int64), pin(st.workers, np.int32),
+                             pin(st.pipeline_of_ctx, np.int32))
+
+    def pinned(shape, dt):
+        return torch.empty(shape, dtype=dt).pin_memory()
+
+    out = pb.PlanOut(pinned(n, torch.uint8), pinned(n, torch.int64), pinned(n, torch.int32),
+                     pinned(n, torch.int32), pinned(1, torch.int64), pinned(n_seg + 1, torch.int32),
+                     pinned(n_seg, torch.int32))
+    ws = pb.alloc_workspace(pb.pard_plan_host_workspace_bytes(n, wl.n_ctx, S, R), dev)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step():
+        pb.pard_plan_host(pipes, req, n, hs, wl.n_ctx, 0, out, ws, stream=stream)
+
+    for _ in range(3):
+        step()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) / 1e3
+    if dist is not None:
+        t = torch.tensor([sec], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+    nk = int(out.n_kept[0])
+    state_bytes = sum(t.numel() * t.element_size() for t in
+                      (hs.now_us, hs.batch, hs.free_at_us, hs.q_us, hs.w_us, hs.workers,
+                       hs.pipeline_of_ctx) if t is not None)
+    h2d = 16 * n + state_bytes
+    d2h = n + 8 * n + 4 * n + 4 * nk + 8 + 4 * (n_seg + 1) + 4 * n_seg
+    return sec, h2d, d2h
+
+
+def run_ours(args):
+    import torch
+    from paper_2602_08747_b200 import build as pbuild
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the planner has no CPU path")
+    pbuild.build()
+    torch.cuda.set_device(local)
+    dev = "cuda:%d" % local
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device(dev))
+        dist = dist_mod
+
+    # every rank plans its own, independently drawn snapshot (contexts are
+    # independent planning problems: no data-path collective)
+    wl = inputs.make(WORKLOAD, seed=2 + rank)
+    plan = DevicePlan(wl, dev)
+    plan.step(nowait=False)
+    keep_frac = float(plan.out.n_kept.cpu()[0]) / wl.n
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    # warm-up first so that the sampler only sees the timed region
+    for _ in range(args.warmup):
+        plan.step()
+    plan.status()
+    sampler.start()
+    sec, prof = timed_steps(plan, args.steps, 0, dist, profile_every=8)
+    clocks = sampler.result()
+
+    peak, peak_kind = measured_peaks()
+    n_total = wl.n * world
+    value = n_total * args.steps / sec
+    e2e_steps = max(3, min(args.steps, 20))
+    e2e_sec, h2d, d2h = run_e2e(wl, dev, e2e_steps, dist)
+
+    if rank == 0:
+        kernels = kernel_table(prof, wl.n, keep_frac, peak)
+        timed = {k: v for k, v in kernels.items() if k != "other"}
+        top = max(timed, key=lambda k: timed[k]["ms_per_step"])
+        traffic = None
+        roofline = {"bound": "hbm", "kernel": top, "achieved": timed[top]["achieved_gbs"], "peak": peak,
+                    "unit": "GB/s", "frac": timed[top]["frac"], "traffic": traffic,
+                    "peak_kind": "of " + peak_kind,
+                    "algorithmic_bytes_per_launch": timed[top]["algorithmic_bytes_per_request"] * wl.n,
+                    "kernels": kernels}
+        # the balanced variant (about half of the requests kept) as a second data point
+        variants = {}
+        if not args.no_variants:
+            wlb = inputs.make(WORKLOAD + "b", seed=2)
+            pl2 = DevicePlan(wlb, dev)
+            pl2.step(nowait=False)
+            kf = float(pl2.out.n_kept.cpu()[0]) / wlb.n
+            s2, prof2 = timed_steps(pl2, max(10, args.steps // 4), 5, None, profile_every=4)
+            variants[WORKLOAD + "b"] = {"value": wlb.n * max(10, args.steps // 4) / s2, "unit": UNIT,
+                                        "keep_fraction": kf,
+                                        "kernels": kernel_table(prof2, wlb.n, kf, peak)}
+            del pl2
+        t_cpu, _ = time_oracle(wl, 2)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "requests_per_gpu": wl.n, "stages": 16, "paths": 12,
+                       "contexts": wl.n_ctx, "keep_fraction": keep_frac,
+                       "l2": "inputs (256 MiB) and sort buffers (2 x 128 MiB) exceed the 126 MB L2",
+                       "parallelism": "independent snapshot per GPU, no collective"},
+            "clocks": clocks,
+            "e2e": {"value": n_total * e2e_steps / e2e_sec, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "ms_per_step": 1e3 * e2e_sec / e2e_steps},
+            "gpu_launches": plan.launches * args.steps,
+            "gpu_launches_per_step": plan.launches,
+            "roofline": roofline,
+            "cpu_baseline": {"value": wl.n / t_cpu, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": "the full %s snapshot (%d requests), best of 2 runs" % (WORKLOAD, wl.n),
+                             "host_cores": os.cpu_count()},
+            "variants": variants,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-variants", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

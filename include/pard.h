@@ -148,6 +148,9 @@ typedef struct pard_plan_out {
 
 #define PARD_MODE_ADMITTED 0u   /* a dropped request takes no batch slot (default)   */
 #define PARD_MODE_RAW      1u   /* every queued request ahead takes a batch slot     */
+#define PARD_MODE_NOWAIT   2u   /* pard_plan returns once its work is enqueued and
+                                   reads no status back; the status word stays in the
+                                   workspace until pard_plan_status fetches it        */
 
 /* Device scratch pard_plan needs for n requests in n_ctx contexts. */
 int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
@@ -178,6 +181,18 @@ int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
               const pard_plan_out_t* out,
               void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
 
+/* For PARD_MODE_NOWAIT: waits for `cuda_stream`, then returns the status that
+ * the most recent pard_plan call on this workspace left there (PARD_OK,
+ * PARD_EDATA, PARD_ERANGE or PARD_ETIMEOUT).  The workspace must not have been
+ * reused for anything else in between. */
+int pard_plan_status(const void* d_workspace, void* cuda_stream);
+
+/* Number of kernels one pard_plan call enqueues for these sizes (memsets and
+ * copies not counted).  Radix passes beyond the key width found on the device
+ * are launched and return at once; they are included. */
+int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
+                              uint32_t* launches);
+
 /* Same computation with HOST inputs and outputs: `requests`, the arrays of
  * `state` and the members of `out` are host pointers (pinned memory makes the
  * copies asynchronous).  Inputs are copied to the device, planned, and the
@@ -201,6 +216,20 @@ int pard_plan_host(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines
 int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets,
                  uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                  int64_t* d_out_total, int64_t* d_out_kept, void* cuda_stream);
+
+/* ---- optional device timing of the planner's phases ----------------------
+ * For benchmarks.  Between pard_profile_begin and pard_profile_end every
+ * `every`-th pard_plan call of the process (at most max_samples of them)
+ * records CUDA events on its stream between its phases; the other calls are
+ * untouched.  pard_profile_end waits for the sampled calls, adds up the
+ * elapsed milliseconds per phase into ms_sum[PARD_N_PHASES] and returns the
+ * number of sampled calls.  Process-wide state: do not call begin/end while
+ * another thread is inside pard_plan.  The paper has no counterpart. */
+#define PARD_N_PHASES 13
+int pard_profile_begin(uint32_t every, uint32_t max_samples);
+int pard_profile_end(float* ms_sum, uint32_t* n_samples);
+/* "clear", "prepass", "segments", "pack", "sort0".."sort7", "decide" */
+const char* pard_profile_phase_name(uint32_t phase);
 
 #ifdef __cplusplus
 }

@@ -21,11 +21,14 @@ PARD_OK = 0
 PARD_EINVAL, PARD_ECYCLE, PARD_ERANGE, PARD_ENOMEM = -1, -2, -3, -4
 PARD_EWORKSPACE, PARD_ETIMEOUT, PARD_ECUDA, PARD_EDATA = -5, -6, -7, -8
 PARD_LOAD_HOST_ONLY = 1
-PARD_MODE_ADMITTED, PARD_MODE_RAW = 0, 1
+PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT = 0, 1, 2
+PARD_N_PHASES = 13
 
 EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pipeline_n_stages",
            "pard_pipeline_n_slots", "pard_pipeline_paths", "pard_plan_workspace_bytes", "pard_plan",
-           "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput"]
+           "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput", "pard_plan_status",
+           "pard_plan_kernel_launches", "pard_profile_begin", "pard_profile_end",
+           "pard_profile_phase_name"]
 
 
 class PardError(RuntimeError):
@@ -81,8 +84,14 @@ def library() -> C.CDLL:
         lib.pard_plan_host.argtypes = plan_args
         lib.pard_goodput.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.pard_plan_status.argtypes = [C.c_void_p, C.c_void_p]
+        lib.pard_plan_kernel_launches.argtypes = [C.c_uint64, C.c_uint32, C.c_int32, C.c_void_p]
+        lib.pard_profile_begin.argtypes = [C.c_uint32, C.c_uint32]
+        lib.pard_profile_end.argtypes = [C.c_void_p, C.c_void_p]
+        lib.pard_profile_phase_name.restype = C.c_char_p
+        lib.pard_profile_phase_name.argtypes = [C.c_uint32]
         for name in EXPORTS:
-            if name != "pard_strerror":
+            if name not in ("pard_strerror", "pard_profile_phase_name"):
                 getattr(lib, name).restype = C.c_int
         _lib = lib
     return _lib
@@ -239,6 +248,33 @@ def pard_plan_host(pipelines: Sequence[Pipeline], requests, n: int, state: Queue
     if check:
         _check(rc, "pard_plan_host")
     return rc
+
+
+def pard_plan_status(d_workspace, stream: int = 0, check: bool = True) -> int:
+    rc = library().pard_plan_status(_ptr(d_workspace), stream or None)
+    if check:
+        _check(rc, "pard_plan_status")
+    return rc
+
+
+def pard_plan_kernel_launches(n: int, n_ctx: int, stage_stride: int) -> int:
+    v = C.c_uint32()
+    _check(library().pard_plan_kernel_launches(n, n_ctx, stage_stride, C.byref(v)),
+           "pard_plan_kernel_launches")
+    return v.value
+
+
+def pard_profile_begin(every: int, max_samples: int) -> None:
+    _check(library().pard_profile_begin(every, max_samples), "pard_profile_begin")
+
+
+def pard_profile_end() -> dict:
+    """{"n_samples": k, "ms": {phase name: milliseconds summed over the k sampled calls}}"""
+    ms = (C.c_float * PARD_N_PHASES)()
+    k = C.c_uint32()
+    _check(library().pard_profile_end(ms, C.byref(k)), "pard_profile_end")
+    names = [library().pard_profile_phase_name(i).decode() for i in range(PARD_N_PHASES)]
+    return {"n_samples": k.value, "ms": {names[i]: float(ms[i]) for i in range(PARD_N_PHASES)}}
 
 
 def pard_goodput(d_keep, d_seg_offsets, n: int, n_ctx: int, stage_stride: int, d_out_total,

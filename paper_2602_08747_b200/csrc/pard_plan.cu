@@ -13,6 +13,7 @@
  */
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 
 #include "pard_internal.h"
 
@@ -737,6 +738,26 @@ k_decide(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
   }
 }
 
+/* ---- optional phase timing (process-wide) ---- */
+constexpr int kEventsPerSample = PARD_N_PHASES + 1;
+static_assert(PARD_N_PHASES == 4 + kMaxPasses + 1, "phase list");
+struct Profiler {
+  std::mutex mu;
+  bool on = false;
+  uint32_t every = 1, max_samples = 0, calls = 0, n_samples = 0;
+  std::vector<cudaEvent_t> ev;
+};
+Profiler g_prof;
+
+/* events of this call if it is a sampled one, else nullptr */
+cudaEvent_t* profile_acquire() {
+  std::lock_guard<std::mutex> lock(g_prof.mu);
+  if (!g_prof.on) return nullptr;
+  uint32_t call = g_prof.calls++;
+  if (call % g_prof.every != 0 || g_prof.n_samples >= g_prof.max_samples) return nullptr;
+  return g_prof.ev.data() + (size_t)(g_prof.n_samples++) * kEventsPerSample;
+}
+
 int check_state(const pard_queue_state_t* st, uint32_t n_ctx) {
   if (!st) return PARD_EINVAL;
   if (st->stage_stride < 1) return PARD_EINVAL;
@@ -768,7 +789,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   /* ---- host-side checks, nothing launched before they pass ---- */
   if (!pipelines || n_pipelines < 1 || !out) return PARD_EINVAL;
   if (n_pipelines > kMaxPipelinesPerCall) return PARD_ERANGE;
-  if (mode & ~PARD_MODE_RAW) return PARD_EINVAL;
+  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT)) return PARD_EINVAL;
   int rc = check_state(state, n_ctx);
   if (rc != PARD_OK) return rc;
   if (n >= PARD_MAX_REQUESTS) return PARD_ERANGE;
@@ -813,6 +834,13 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   const uint32_t ibits = std::max(1u, ceil_log2(n));
   const uint32_t sbits = ceil_log2(L.n_seg);
 
+  cudaEvent_t* evs = profile_acquire();
+  int phase = 0;
+  auto mark = [&]() {                      /* boundary between two phases */
+    if (evs) cudaEventRecord(evs[phase], stream);
+    ++phase;
+  };
+  mark();
   /* ---- clear the scratch that must start at zero ---- */
   PARD_CUDA_OK(cudaMemsetAsync(ws + L.hdr, 0, sizeof(PlanHeader), stream));
   PARD_CUDA_OK(cudaMemsetAsync(ctx_dmin, 0xff, 8ull * n_ctx, stream));
@@ -832,31 +860,107 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const uint4* req4 = (const uint4*)d_requests;
 
+  mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 2047) / 2048, (uint64_t)sms * 8);
     if (L.n_seg <= (uint32_t)kSmemSegs)
       k_prepass<true><<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, L.n_seg, ctx_dmin, ctx_dmax, seg_off, hdr);
     else
       k_prepass<false><<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, L.n_seg, ctx_dmin, ctx_dmax, seg_off, hdr);
-    k_ctx_span<<<(n_ctx + 255) / 256, 256, 0, stream>>>(ctx_dmin, ctx_dmax, n_ctx, hdr);
   }
+  mark();
+  if (n > 0) k_ctx_span<<<(n_ctx + 255) / 256, 256, 0, stream>>>(ctx_dmin, ctx_dmax, n_ctx, hdr);
   k_seg_scan<<<1, 1024, 0, stream>>>(seg_off, L.n_seg, out->d_seg_offsets, sbits, ibits, hdr);
   k_seg_const<<<(L.n_seg + 127) / 128, 128, 0, stream>>>(d_pipes, n_pipelines, *state, n_ctx, ctx_dmin,
                                                          seg_off, ktab, hdr);
+  mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
     k_pack<<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, ctx_dmin, ibits, hdr, buf_a, hist);
-    for (uint32_t p = 0; p < L.max_passes; ++p)
+  }
+  for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
+    mark();
+    if (n > 0 && p < L.max_passes)
       k_sort_pass<<<L.sort_tiles, kSortThreads, 0, stream>>>(
           p, hdr, buf_a, buf_b, hist, lookback + (size_t)p * L.sort_tiles * kBins, n32, ibits);
+  }
+  mark();
+  if (n > 0) {
     k_decide<<<L.dec_tiles, kDecThreads, 0, stream>>>(
         hdr, buf_a, buf_b, n32, ibits, mode, ktab, seg_off, st_min, st_kept, out->d_keep,
         (long long*)out->d_est_us, out->d_perm, out->d_kept_idx,
         (unsigned long long*)out->d_n_kept, out->d_seg_kept);
   }
+  mark();
   PARD_CUDA_OK(cudaGetLastError());
+  if (mode & PARD_MODE_NOWAIT) return PARD_OK;
+  return pard_plan_status(d_workspace, cuda_stream);
+}
+
+extern "C" int pard_plan_status(const void* d_workspace, void* cuda_stream) {
+  if (!d_workspace) return PARD_EINVAL;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
   uint32_t h_status = 0;
-  PARD_CUDA_OK(cudaMemcpyAsync(&h_status, &hdr->status, 4, cudaMemcpyDeviceToHost, stream));
+  PARD_CUDA_OK(cudaMemcpyAsync(&h_status, &((const PlanHeader*)d_workspace)->status, 4,
+                               cudaMemcpyDeviceToHost, stream));
   PARD_CUDA_OK(cudaStreamSynchronize(stream));
   return h_status ? -(int)h_status : PARD_OK;
+}
+
+extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
+                                         uint32_t* launches) {
+  uint64_t bytes;
+  if (!launches) return PARD_EINVAL;
+  int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
+  if (rc != PARD_OK) return rc;
+  /* seg_scan + seg_const always; prepass, ctx_span, pack, passes, decide when n > 0 */
+  *launches = n > 0 ? 2 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 1 : 2;
+  return PARD_OK;
+}
+
+extern "C" int pard_profile_begin(uint32_t every, uint32_t max_samples) {
+  if (every < 1 || max_samples < 1 || max_samples > 65536) return PARD_EINVAL;
+  std::lock_guard<std::mutex> lock(g_prof.mu);
+  if (g_prof.on) return PARD_EINVAL;
+  g_prof.ev.assign((size_t)max_samples * kEventsPerSample, nullptr);
+  for (auto& e : g_prof.ev)
+    if (cudaEventCreate(&e) != cudaSuccess) {
+      for (auto& f : g_prof.ev) if (f) cudaEventDestroy(f);
+      g_prof.ev.clear();
+      return PARD_ECUDA;
+    }
+  g_prof.every = every;
+  g_prof.max_samples = max_samples;
+  g_prof.calls = 0;
+  g_prof.n_samples = 0;
+  g_prof.on = true;
+  return PARD_OK;
+}
+
+extern "C" int pard_profile_end(float* ms_sum, uint32_t* n_samples) {
+  std::lock_guard<std::mutex> lock(g_prof.mu);
+  if (!g_prof.on) return PARD_EINVAL;
+  int rc = PARD_OK;
+  if (ms_sum) for (int i = 0; i < PARD_N_PHASES; ++i) ms_sum[i] = 0.f;
+  for (uint32_t s = 0; s < g_prof.n_samples; ++s) {
+    cudaEvent_t* e = g_prof.ev.data() + (size_t)s * kEventsPerSample;
+    if (cudaEventSynchronize(e[PARD_N_PHASES]) != cudaSuccess) { rc = PARD_ECUDA; break; }
+    for (int i = 0; i < PARD_N_PHASES && ms_sum; ++i) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, e[i], e[i + 1]) != cudaSuccess) rc = PARD_ECUDA;
+      ms_sum[i] += ms;
+    }
+  }
+  if (n_samples) *n_samples = g_prof.n_samples;
+  for (auto& e : g_prof.ev) cudaEventDestroy(e);
+  g_prof.ev.clear();
+  g_prof.on = false;
+  return rc;
+}
+
+extern "C" const char* pard_profile_phase_name(uint32_t phase) {
+  static const char* names[PARD_N_PHASES] = {"clear", "prepass", "segments", "pack", "sort0", "sort1",
+                                              "sort2", "sort3", "sort4", "sort5", "sort6", "sort7",
+                                              "decide"};
+  return phase < PARD_N_PHASES ? names[phase] : "";
 }

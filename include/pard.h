@@ -47,8 +47,10 @@ typedef enum pard_status {
   PARD_EWORKSPACE  = -5,  /* caller's workspace is smaller than required             */
   PARD_ETIMEOUT    = -6,  /* a bounded device-side wait ran out; outputs unspecified */
   PARD_ECUDA       = -7,  /* a CUDA runtime call failed                              */
-  PARD_EDATA       = -8   /* device found ctx, stage or batch size out of range, or
+  PARD_EDATA       = -8,  /* device found ctx, stage or batch size out of range, or
                              a deadline outside [0, 2^60); outputs unspecified       */
+  PARD_ESTATIC     = -9   /* pard_plan_static: the problem needs more scratch than
+                             the library's built-in PARD_STATIC_SCRATCH_BYTES        */
 } pard_status;
 
 const char* pard_strerror(int status);
@@ -192,6 +194,36 @@ int pard_plan_status(const void* d_workspace, void* cuda_stream);
  * are launched and return at once; they are included. */
 int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                               uint32_t* launches);
+
+/* The planner for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a deployment aid).  A drop planner typically runs in
+ * the control loop of an inference server: the serving runtime has often
+ * claimed all device memory at start-up, and a cudaMalloc / cudaFree issued
+ * from that loop takes the driver's allocation lock and may synchronise the
+ * device, stalling the very inference kernels whose queues are being planned.
+ * pard_plan_static computes exactly what pard_plan computes, with the same
+ * arguments minus the workspace: its scratch is a fixed array of
+ * PARD_STATIC_SCRATCH_BYTES of device global memory that is part of the
+ * library image (every GPU that loads the library holds it until the process
+ * exits).  It calls no allocation routine.
+ *  - Size limit: accepted iff pard_plan_workspace_bytes(n, n_ctx, stage_stride)
+ *    <= PARD_STATIC_SCRATCH_BYTES, e.g. 2^18 requests in up to 4,096 segments;
+ *    anything larger returns PARD_ESTATIC and nothing is launched.
+ *  - The first call on each device looks up the array's device address (a
+ *    one-time set-up under a lock); make that first call before any stream
+ *    capture begins on that device.
+ *  - All calls on one device share the one array.  Each call clears the parts
+ *    that must start at zero, so the previous call's contents do not matter,
+ *    but two calls whose GPU work overlaps (different streams, or
+ *    PARD_MODE_NOWAIT calls not ordered by one stream) race on it; so does a
+ *    pard_plan_status on anything but this scratch.  With PARD_MODE_NOWAIT
+ *    there is no way to fetch the status afterwards: use the default mode.
+ * Inputs, outputs, ordering and error codes are otherwise those of pard_plan. */
+#define PARD_STATIC_SCRATCH_BYTES (8u << 20)
+int pard_plan_static(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+                     const pard_request_t* d_requests, uint64_t n,
+                     const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,
+                     const pard_plan_out_t* out, void* cuda_stream);
 
 /* Same computation with HOST inputs and outputs: `requests`, the arrays of
  * `state` and the members of `out` are host pointers (pinned memory makes the

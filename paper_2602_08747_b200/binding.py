@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libpard.so")
 
 PARD_OK = 0
 PARD_EINVAL, PARD_ECYCLE, PARD_ERANGE, PARD_ENOMEM = -1, -2, -3, -4
-PARD_EWORKSPACE, PARD_ETIMEOUT, PARD_ECUDA, PARD_EDATA = -5, -6, -7, -8
+PARD_EWORKSPACE, PARD_ETIMEOUT, PARD_ECUDA, PARD_EDATA, PARD_ESTATIC = -5, -6, -7, -8, -9
+PARD_STATIC_SCRATCH_BYTES = 8 << 20
 PARD_LOAD_HOST_ONLY = 1
 PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT = 0, 1, 2
 PARD_N_PHASES = 13
@@ -28,7 +29,7 @@ EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pi
            "pard_pipeline_n_slots", "pard_pipeline_paths", "pard_plan_workspace_bytes", "pard_plan",
            "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput", "pard_plan_status",
            "pard_plan_kernel_launches", "pard_profile_begin", "pard_profile_end",
-           "pard_profile_phase_name"]
+           "pard_profile_phase_name", "pard_plan_static"]
 
 
 class PardError(RuntimeError):
@@ -84,6 +85,7 @@ def library() -> C.CDLL:
         lib.pard_plan_host.argtypes = plan_args
         lib.pard_goodput.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.pard_plan_static.argtypes = plan_args[:8] + [C.c_void_p]
         lib.pard_plan_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.pard_plan_kernel_launches.argtypes = [C.c_uint64, C.c_uint32, C.c_int32, C.c_void_p]
         lib.pard_profile_begin.argtypes = [C.c_uint32, C.c_uint32]
@@ -247,6 +249,21 @@ def pard_plan_host(pipelines: Sequence[Pipeline], requests, n: int, state: Queue
                                   C.byref(o), _ptr(d_workspace), wb, stream or None)
     if check:
         _check(rc, "pard_plan_host")
+    return rc
+
+
+def pard_plan_static(pipelines: Sequence[Pipeline], d_requests, n: int, state: QueueStateArrays,
+                     n_ctx: int, mode: int, out: PlanOut, stream: int = 0, check: bool = True) -> int:
+    """pard_plan without a workspace argument: the scratch is the library's own
+    fixed device array, for callers that must not allocate device memory
+    (problems up to PARD_STATIC_SCRATCH_BYTES of scratch; larger ones return
+    PARD_ESTATIC).  Calls on one device share that array and must not overlap."""
+    hs = _handles(pipelines)
+    st, o = state.c_struct(), out.c_struct()
+    rc = library().pard_plan_static(hs, len(pipelines), _ptr(d_requests), n, C.byref(st), n_ctx, mode,
+                                    C.byref(o), stream or None)
+    if check:
+        _check(rc, "pard_plan_static")
     return rc
 
 

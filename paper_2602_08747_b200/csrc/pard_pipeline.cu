@@ -244,6 +244,7 @@ extern "C" const char* pard_strerror(int status) {
     case PARD_ETIMEOUT: return "device-side wait ran out";
     case PARD_ECUDA: return "CUDA runtime call failed";
     case PARD_EDATA: return "device found out-of-range request or state data";
+    case PARD_ESTATIC: return "problem exceeds the built-in scratch of pard_plan_static";
     default: return "unknown status";
   }
 }

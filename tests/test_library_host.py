@@ -36,11 +36,11 @@ def test_every_declared_symbol_is_exported():
 
 def test_strerror_covers_all_codes():
     seen = set()
-    for code in range(0, -9, -1):
+    for code in range(0, -10, -1):
         s = pb.pard_strerror(code)
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 9
+    assert len(seen) == 10
     assert pb.pard_strerror(-99) == "unknown status"
 
 

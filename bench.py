@@ -294,6 +294,15 @@ def run_ours(args):
         dist_mod.init_process_group("nccl", device_id=torch.device(dev))
         dist = dist_mod
 
+    if args.only_device:
+        kw = {"n": args.n} if args.n else {}
+        wl = inputs.make(args.workload or WORKLOAD, **kw)
+        plan = DevicePlan(wl, dev)
+        sec, _ = timed_steps(plan, args.steps, args.warmup, None)
+        print(json.dumps({"only_device": True, "workload": wl.name, "n": wl.n,
+                          "ms_per_step": 1e3 * sec / args.steps}))
+        return
+
     # every rank plans its own, independently drawn snapshot (contexts are
     # independent planning problems: no data-path collective)
     wl = inputs.make(WORKLOAD, seed=2 + rank)
@@ -372,6 +381,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-variants", action="store_true")
+    ap.add_argument("--only-device", action="store_true",
+                    help="run warm-up and timed steps of the device path only and print a short line "
+                         "(for use under a profiler; not a bench value)")
+    ap.add_argument("--workload", default=None, help="with --only-device: another workload name, e.g. C3b")
+    ap.add_argument("--n", type=int, default=None, help="with --only-device: number of requests")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -39,10 +39,12 @@ struct pard_pipeline {
 
 /* Per-segment constants (Eq. 3 terms that do not depend on the request). */
 struct __align__(16) PardSegConst {
-  int64_t A;        /* base + d_k(B_k) + L_sub : estimate of a request at position 0 */
-  int64_t A_rel;    /* A - (smallest deadline of the segment's ctx)                  */
-  int64_t d;        /* d_k(B_k)                                                      */
-  uint32_t cap;     /* min(B_k * m_k, 2^30)                                          */
+  int64_t A;         /* base + d_k(B_k) + L_sub : estimate of a request at position 0   */
+  int64_t A_rel;     /* A - (smallest deadline of the segment's ctx)                    */
+  int64_t d;         /* d_k(B_k)                                                        */
+  uint64_t d_magic;  /* floor(2^64 / d) + 1, or 0 when d == 1 or d >= 2^32              */
+  uint64_t cap_magic;/* floor(2^64 / cap) + 1, or 0 when cap == 1                       */
+  uint32_t cap;      /* min(B_k * m_k, 2^30)                                            */
   uint32_t pad;
 };
 

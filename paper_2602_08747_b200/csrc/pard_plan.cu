@@ -31,15 +31,14 @@ constexpr int kSortTile = kSortThreads * kSortItems;
 constexpr int kDecThreads = 256;
 constexpr int kDecItems = 8;
 constexpr int kDecTile = kDecThreads * kDecItems;
+constexpr int kCompactChunk = 4096;                /* indices moved by one block of k_kept_move */
+constexpr int kLookBatch = 16;                     /* earlier tiles inspected per round trip in the sort */
 constexpr int kSmemSegs = 4096;                    /* segment histogram kept in shared memory up to here */
 
 /* look-back word of the sort: [31:30] state, [29:0] count */
 constexpr uint32_t kLbAgg = 1u << 30;
 constexpr uint32_t kLbIncl = 2u << 30;
 constexpr uint32_t kLbMask = (1u << 30) - 1;
-/* look-back words of the decision pass: [63:62] state */
-constexpr unsigned long long kStAgg = 1ull << 62;
-constexpr unsigned long long kStIncl = 2ull << 62;
 
 struct PlanHeader {
   uint32_t status;            /* 0, or the positive value of a pard_status */
@@ -54,8 +53,9 @@ struct PlanHeader {
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
-  uint64_t hdr, pipes, ctx_dmin, ctx_dmax, seg_off, ktab, hist, lookback, st_min, st_kept,
-      buf_a, buf_b, total;
+  /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
+  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, hist, lookback, zero_end,
+      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, kept_tmp, buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes;
 };
 
@@ -82,15 +82,20 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.max_passes = std::min<uint32_t>(kMaxPasses, (std::min(64u - ibits, sbits + 60u) + 7) / 8);
   uint64_t o = 0;
   L.hdr = o;       o = al(o + sizeof(PlanHeader));
-  L.pipes = o;     o = al(o + 8ull * kMaxPipelinesPerCall);
-  L.ctx_dmin = o;  o = al(o + 8ull * n_ctx);
+  L.ctx_dmin = o;  o = al(o + 8ull * n_ctx);          /* complement of the minimum: starts at 0 */
   L.ctx_dmax = o;  o = al(o + 8ull * n_ctx);
   L.seg_off = o;   o = al(o + 4ull * (L.n_seg + 1));
-  L.ktab = o;      o = al(o + sizeof(PardSegConst) * (uint64_t)L.n_seg);
+  L.seg_kept = o;  o = al(o + 4ull * L.n_seg);
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
-  L.lookback = o;  o = al(o + 4ull * kBins * (uint64_t)L.sort_tiles * L.max_passes);
-  L.st_min = o;    o = al(o + 8ull * L.dec_tiles);
-  L.st_kept = o;   o = al(o + 8ull * L.dec_tiles);
+  L.lookback = o;  o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);   /* two arrays, used in turn */
+  L.zero_end = o;
+  L.pipes = o;     o = al(o + 8ull * kMaxPipelinesPerCall);
+  L.ktab = o;      o = al(o + sizeof(PardSegConst) * (uint64_t)L.n_seg);
+  L.kept_base = o; o = al(o + 4ull * (L.n_seg + 1));
+  L.chunk_base = o; o = al(o + 4ull * (L.n_seg + 1));
+  L.tile_agg = o;  o = al(o + 8ull * L.dec_tiles);
+  L.tile_carry = o; o = al(o + 4ull * L.dec_tiles);
+  L.kept_tmp = o;  o = al(o + 4ull * n);
   L.buf_a = o;     o = al(o + 8ull * n);
   L.buf_b = o;     o = al(o + 8ull * n);
   L.total = o;
@@ -101,19 +106,13 @@ __device__ __forceinline__ void set_status(PlanHeader* hdr, int status) {
   atomicCAS(&hdr->status, 0u, (uint32_t)(-status));
 }
 
-__device__ __forceinline__ uint32_t lanemask_lt() {
-  uint32_t m;
-  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
-  return m;
-}
-
 /* ------------------------------------------------------------------------ */
 /* prepass: one coalesced 16-byte read per request                           */
 /* ------------------------------------------------------------------------ */
 template <bool SMEM_HIST>
 __global__ void __launch_bounds__(256)
 k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S, uint32_t n_seg,
-          unsigned long long* __restrict__ ctx_dmin, unsigned long long* __restrict__ ctx_dmax,
+          unsigned long long* __restrict__ ctx_dmin_inv, unsigned long long* __restrict__ ctx_dmax,
           uint32_t* __restrict__ seg_count, PlanHeader* hdr) {
   __shared__ uint32_t s_hist[SMEM_HIST ? kSmemSegs : 1];
   const uint32_t lane = threadIdx.x & 31;
@@ -135,7 +134,7 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
       lmax = b > lmax ? b : lmax;
     }
     if (lane == 0 && lmin <= lmax) {
-      atomicMin(&ctx_dmin[run_ctx], lmin);
+      atomicMax(&ctx_dmin_inv[run_ctx], ~lmin);
       atomicMax(&ctx_dmax[run_ctx], lmax);
     }
     lmin = ~0ull;
@@ -157,11 +156,12 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
         ok = false;
       }
       uint32_t seg = ok ? ctx * S + stage : 0;
-      if (SMEM_HIST) {
-        if (ok) atomicAdd(&s_hist[seg], 1u);
-      } else {
+      {                                       /* one atomic per distinct segment in the warp */
         uint32_t grp = __match_any_sync(0xffffffffu, ok ? seg : 0xffffffffu);
-        if (ok && lane == (uint32_t)(__ffs(grp) - 1)) atomicAdd(&seg_count[seg], (uint32_t)__popc(grp));
+        if (ok && lane == (uint32_t)(__ffs(grp) - 1)) {
+          if (SMEM_HIST) atomicAdd(&s_hist[seg], (uint32_t)__popc(grp));
+          else atomicAdd(&seg_count[seg], (uint32_t)__popc(grp));
+        }
       }
       uint32_t vmask = __ballot_sync(0xffffffffu, ok);
       if (vmask == 0) continue;
@@ -177,7 +177,7 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
           lmax = (unsigned long long)D > lmax ? (unsigned long long)D : lmax;
         }
       } else if (ok) {
-        atomicMin(&ctx_dmin[ctx], (unsigned long long)D);
+        atomicMax(&ctx_dmin_inv[ctx], ~(unsigned long long)D);
         atomicMax(&ctx_dmax[ctx], (unsigned long long)D);
       }
     }
@@ -191,12 +191,12 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
   }
 }
 
-__global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin,
+__global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin_inv,
                            const unsigned long long* __restrict__ ctx_dmax, uint32_t n_ctx,
                            PlanHeader* hdr) {
   uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
   unsigned long long span = 0;
-  if (c < n_ctx && ctx_dmin[c] <= ctx_dmax[c]) span = ctx_dmax[c] - ctx_dmin[c];
+  if (c < n_ctx && ~ctx_dmin_inv[c] <= ctx_dmax[c]) span = ctx_dmax[c] - ~ctx_dmin_inv[c];
   for (int o = 16; o; o >>= 1) {
     unsigned long long a = __shfl_xor_sync(0xffffffffu, span, o);
     span = a > span ? a : span;
@@ -207,8 +207,8 @@ __global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin,
 /* Exclusive scan of the queue lengths by one block; also fixes the key width. */
 __global__ void __launch_bounds__(1024)
 k_seg_scan(uint32_t* __restrict__ seg_off /* in: counts, out: offsets, [n_seg+1] */,
-           uint32_t n_seg, uint32_t* __restrict__ out_seg_off, uint32_t sbits, uint32_t ibits,
-           PlanHeader* hdr) {
+           uint32_t n_seg, uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ out_seg_kept,
+           uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
   __shared__ uint32_t s_warp[32];
   __shared__ uint32_t s_carry;
   if (threadIdx.x == 0) {
@@ -248,6 +248,7 @@ k_seg_scan(uint32_t* __restrict__ seg_off /* in: counts, out: offsets, [n_seg+1]
     if (i <= n_seg) {
       seg_off[i] = excl;
       if (out_seg_off) out_seg_off[i] = excl;
+      if (out_seg_kept && i < n_seg) out_seg_kept[i] = 0;
     }
     __syncthreads();
     if (threadIdx.x == 1023) s_carry = excl + v;
@@ -255,18 +256,29 @@ k_seg_scan(uint32_t* __restrict__ seg_off /* in: counts, out: offsets, [n_seg+1]
   }
 }
 
-/* Per-segment constants; one thread per (ctx, stage). */
-__global__ void k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
-                            pard_queue_state_t st, uint32_t n_ctx,
-                            const unsigned long long* __restrict__ ctx_dmin,
-                            const uint32_t* __restrict__ seg_off, PardSegConst* __restrict__ ktab,
-                            PlanHeader* hdr) {
+/* floor(2^64 / d) + 1 for d >= 2 */
+__device__ __forceinline__ unsigned long long magic64(unsigned long long d) {
+  unsigned long long q = ~0ull / d;
+  if (~0ull % d == d - 1) ++q;          /* d divides 2^64 */
+  return q + 1;
+}
+
+/* Per-segment constants; one warp per (ctx, stage), lanes over the stage's
+ * downstream paths (the path table of the pipeline lists, for every stage,
+ * each stage sequence from a successor to a sink). */
+__global__ void __launch_bounds__(128)
+k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
+            pard_queue_state_t st, uint32_t n_ctx,
+            const unsigned long long* __restrict__ ctx_dmin_inv,
+            const uint32_t* __restrict__ seg_off, PardSegConst* __restrict__ ktab,
+            PlanHeader* hdr) {
   const uint32_t S = (uint32_t)st.stage_stride;
-  uint32_t seg = blockIdx.x * blockDim.x + threadIdx.x;
-  if (seg >= n_ctx * S) return;
-  uint32_t c = seg / S, k = seg % S;
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t seg = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (seg >= n_ctx * S) return;                          /* whole warps leave together */
+  const uint32_t c = seg / S, k = seg % S;
   PardSegConst out;
-  out.A = 0; out.A_rel = 0; out.d = 1; out.cap = 1; out.pad = 0;
+  out.A = 0; out.A_rel = 0; out.d = 1; out.cap = 1; out.pad = 0; out.d_magic = 0; out.cap_magic = 0;
   int32_t pi = st.d_pipeline_of_ctx ? st.d_pipeline_of_ctx[c] : 0;
   bool bad = false;
   if (pi < 0 || (uint32_t)pi >= n_pipelines) {
@@ -285,10 +297,10 @@ __global__ void k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32
           fa >= PARD_TIME_LIMIT_US) {
         bad = true;
       } else {
-        int64_t d = p->lat_us[p->lat_offsets[k] + B - 1];
-        int64_t lsub = 0;
+        const int64_t d = p->lat_us[p->lat_offsets[k] + B - 1];
         const int32_t s0 = p->stage_slot_off[k], s1 = p->stage_slot_off[k + 1];
-        for (int32_t s = s0; s < s1; ++s) {             /* every downstream path */
+        long long lsub = -1;                              /* every path sum is >= 1 */
+        for (int32_t s = s0 + (int32_t)lane; s < s1; s += 32) {
           int64_t acc = st.d_w_us ? st.d_w_us[(size_t)c * st.slot_stride + s] : 0;
           if (acc < 0 || acc >= PARD_TIME_LIMIT_US) { bad = true; acc = 0; }
           for (int32_t e = p->path_off[s]; e < p->path_off[s + 1]; ++e) {
@@ -298,25 +310,32 @@ __global__ void k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32
             if (Bi < 1 || Bi > p->bmax[i] || qi < 0 || qi >= PARD_TIME_LIMIT_US) { bad = true; Bi = 1; qi = 0; }
             acc += qi + p->lat_us[p->lat_offsets[i] + Bi - 1];
           }
-          lsub = (s == s0 || acc > lsub) ? acc : lsub;
+          lsub = acc > lsub ? acc : lsub;
         }
+        for (int o = 16; o; o >>= 1) {                    /* maximum over the paths */
+          long long t = __shfl_xor_sync(0xffffffffu, lsub, o);
+          lsub = t > lsub ? t : lsub;
+        }
+        if (lsub < 0) lsub = 0;                           /* a sink: nothing downstream */
         int64_t base = now > fa ? now : fa;
         int64_t cap = (int64_t)B * m;
         out.d = d;
         out.cap = (uint32_t)(cap > (int64_t)(1u << 30) ? (int64_t)(1u << 30) : cap);
         out.A = base + d + lsub;
-        out.A_rel = out.A - (int64_t)ctx_dmin[c];
+        out.A_rel = out.A - (int64_t)(~ctx_dmin_inv[c]);
+        out.d_magic = (d >= 2 && d < ((int64_t)1 << 32)) ? magic64((uint64_t)d) : 0;
+        out.cap_magic = out.cap >= 2 ? magic64(out.cap) : 0;
       }
     }
   }
   if (bad) set_status(hdr, PARD_EDATA);
-  ktab[seg] = out;
+  if (lane == 0) ktab[seg] = out;
 }
 
 /* request -> sort element; digit histograms of every pass */
 __global__ void __launch_bounds__(256)
 k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
-       const unsigned long long* __restrict__ ctx_dmin, uint32_t ibits,
+       const unsigned long long* __restrict__ ctx_dmin_inv, uint32_t ibits,
        const PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
        uint32_t* __restrict__ hist) {
   __shared__ uint32_t s_hist[kMaxPasses * kBins];
@@ -332,7 +351,7 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
     uint32_t ctx = r.z, stage = r.w & 0xffffu;
     unsigned long long e;
     if (ctx < n_ctx && stage < S) {
-      unsigned long long off = (D - ctx_dmin[ctx]) & dmask;
+      unsigned long long off = (D - ~ctx_dmin_inv[ctx]) & dmask;
       e = ((((unsigned long long)(ctx * S + stage) << dbits) | off) << ibits) | j;
     } else {
       e = j;                                  /* flagged by the prepass; keep indices in range */
@@ -349,12 +368,16 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
 /* ------------------------------------------------------------------------ */
 /* one LSD radix pass (8 bits), stable, tile prefixes by decoupled look-back */
 /* ------------------------------------------------------------------------ */
-__global__ void __launch_bounds__(kSortThreads)
+__global__ void __launch_bounds__(kSortThreads, 3)
 k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf_a,
             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ hist,
-            uint32_t* __restrict__ lookback, uint32_t n, uint32_t ibits) {
+            uint32_t* __restrict__ lookback, uint32_t* __restrict__ lookback_next, uint32_t n,
+            uint32_t ibits) {
   constexpr int WARPS = kSortThreads / 32;
-  __shared__ unsigned long long s_keys[kSortTile];
+  /* the match words are only used while ranking, the key buffer only afterwards */
+  __shared__ __align__(16) unsigned long long s_keys[kSortTile];
+  uint32_t (*s_match)[kBins] = reinterpret_cast<uint32_t (*)[kBins]>(s_keys);
+  static_assert(sizeof(uint32_t) * WARPS * kBins <= sizeof(unsigned long long) * kSortTile, "alias fits");
   __shared__ uint32_t s_whist[WARPS][kBins];
   __shared__ uint32_t s_dstart[kBins];
   __shared__ uint32_t s_gofs[kBins];
@@ -371,7 +394,8 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
     s_tile = atomicAdd(&hdr->ticket[pass], 1u);
     s_abort = 0;
   }
-  for (int w = 0; w < WARPS; ++w) s_whist[w][tid] = 0;
+  for (int w = 0; w < WARPS; ++w) { s_whist[w][tid] = 0; s_match[w][tid] = 0; }
+  const uint32_t lanebit = 1u << lane;
   __syncthreads();
   const uint32_t tile = s_tile;
   const uint64_t base = (uint64_t)tile * kSortTile;
@@ -387,15 +411,20 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
 #pragma unroll
   for (int i = 0; i < kSortItems; ++i) {
     uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
-    uint32_t grp = __match_any_sync(0xffffffffu, d);
-    uint32_t leader = __ffs(grp) - 1;
-    uint32_t old = 0;
-    if (lane == leader) {
-      old = s_whist[warp][d];
+    /* lanes of the warp that hold the same digit meet in a shared word: every
+     * lane ORs its bit into the word of its digit and reads the union back
+     * (the hardware match instruction and eight votes both cost far more) */
+    atomicOr(&s_match[warp][d], lanebit);
+    __syncwarp();
+    const uint32_t grp = s_match[warp][d];
+    const uint32_t below = grp & (lanebit - 1);
+    const uint32_t old = s_whist[warp][d];               /* same word for the whole group */
+    __syncwarp();
+    if (below == 0) {                                    /* lowest lane of the group */
       s_whist[warp][d] = old + __popc(grp);
+      s_match[warp][d] = 0;
     }
-    old = __shfl_sync(0xffffffffu, old, leader);
-    rank[i] = old + __popc(grp & lanemask_lt());
+    rank[i] = old + __popc(below);
     __syncwarp();
   }
   __syncthreads();
@@ -427,19 +456,37 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   const uint32_t gstart = wg + g - gh;         /* first global position of digit tid */
   s_dstart[tid] = dstart;
 
-  /* publish the tile's count, then sum the counts of all earlier tiles */
+  /* publish the tile's count, then sum the counts of all earlier tiles.  The
+   * words of kLookBatch earlier tiles are requested together, so a long run
+   * of tiles that have only published their own count costs one memory round
+   * trip per batch instead of one per tile. */
   volatile uint32_t* lb = lookback;            /* this pass's array */
   lb[(size_t)tile * kBins + tid] = cnt | kLbAgg;
-  uint32_t excl = 0;
-  for (int64_t t = (int64_t)tile - 1; t >= 0; --t) {
-    uint32_t v, spins = 0;
-    while (((v = lb[(size_t)t * kBins + tid]) >> 30) == 0) {
-      if (++spins > kSpinLimit) { s_abort = 1; break; }
-      __nanosleep(20);
+  lookback_next[(size_t)tile * kBins + tid] = 0;          /* the array of the pass after this one */
+  uint32_t excl = 0, spins = 0;
+  int64_t t = (int64_t)tile - 1;
+  bool done = t < 0;
+  while (!done) {
+    uint32_t v[kLookBatch];
+#pragma unroll
+    for (int k = 0; k < kLookBatch; ++k)
+      v[k] = (t - k >= 0) ? lb[(size_t)(t - k) * kBins + tid] : +kLbIncl;   /* before tile 0: nothing */
+    int used = 0;
+#pragma unroll
+    for (int k = 0; k < kLookBatch; ++k) {
+      if (!done && used == k) {
+        if ((v[k] >> 30) != 0) {
+          excl += v[k] & kLbMask;
+          used = k + 1;
+          if (v[k] & kLbIncl) done = true;
+        }
+      }
     }
-    if ((v >> 30) == 0) break;
-    excl += v & kLbMask;
-    if (v & kLbIncl) break;
+    t -= used;
+    if (!done && used < kLookBatch) {          /* met a tile that has not published yet */
+      if (++spins > kSpinLimit) { s_abort = 1; break; }
+      __nanosleep(40);
+    }
   }
   lb[(size_t)tile * kBins + tid] = ((excl + cnt) & kLbMask) | kLbIncl;
   s_gofs[tid] = gstart + excl - dstart;
@@ -466,179 +513,355 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
 /* ------------------------------------------------------------------------ */
 /* decision pass over the sorted elements                                    */
 /* ------------------------------------------------------------------------ */
-struct SegMin {            /* value of a segmented running minimum */
-  int32_t m;               /* minimum of u_t - t since the last queue head (or since the span's start) */
+struct SegVal {            /* value of a segmented running reduction */
+  int32_t m;               /* admitted mode: minimum of u_t - t; raw mode: number of kept requests;
+                              over the elements since the last queue head (or since the span's start) */
   uint32_t head;           /* a queue head lies inside the span */
 };
 
-__device__ __forceinline__ SegMin seg_combine(SegMin left, SegMin right) {
-  SegMin r;
-  r.m = right.head ? right.m : min(left.m, right.m);
+template <bool RAW>
+__device__ __forceinline__ SegVal seg_identity() {
+  SegVal a;
+  a.m = RAW ? 0 : 0x7fffffff;
+  a.head = 0;
+  return a;
+}
+
+template <bool RAW>
+__device__ __forceinline__ SegVal seg_combine(SegVal left, SegVal right) {
+  SegVal r;
+  r.m = right.head ? right.m : (RAW ? left.m + right.m : min(left.m, right.m));
   r.head = left.head | right.head;
   return r;
 }
 
-__device__ __forceinline__ unsigned long long pack_min(SegMin a, unsigned long long state) {
+__device__ __forceinline__ unsigned long long pack_val(SegVal a, unsigned long long state) {
   return state | ((unsigned long long)a.head << 32) | (uint32_t)a.m;
 }
-__device__ __forceinline__ SegMin unpack_min(unsigned long long w) {
-  SegMin a;
+__device__ __forceinline__ SegVal unpack_val(unsigned long long w) {
+  SegVal a;
   a.m = (int32_t)(uint32_t)w;
   a.head = (uint32_t)(w >> 32) & 1u;
   return a;
 }
 
-__device__ __forceinline__ uint32_t threshold_u(int64_t X, int64_t d, uint32_t cap) {
+/* floor(x / d) for 32-bit x, with M = floor(2^64 / d) + 1 (d >= 2): exact
+ * whenever x * d < 2^64, i.e. for every 32-bit x and d */
+__device__ __forceinline__ uint32_t div_magic32(uint32_t x, unsigned long long M) {
+  unsigned long long p0 = (unsigned long long)x * (uint32_t)M;
+  unsigned long long p1 = (unsigned long long)x * (uint32_t)(M >> 32) + (p0 >> 32);
+  return (uint32_t)(p1 >> 32);
+}
+
+__device__ __forceinline__ uint32_t threshold_u(int64_t X, const PardSegConst& K) {
   /* number of requests that may be admitted ahead of or at this one while it
    * still completes by its deadline: 0 if even position 0 is late, else
    * cap * (floor(X / d) + 1), saturated */
   if (X < 0) return 0;
   unsigned long long q;
-  if (((unsigned long long)X | (unsigned long long)d) >> 32)
-    q = (unsigned long long)X / (unsigned long long)d;
+  if (((unsigned long long)X >> 32) == 0 && K.d_magic)
+    q = div_magic32((uint32_t)X, K.d_magic);
   else
-    q = (uint32_t)X / (uint32_t)d;
+    q = (unsigned long long)X / (unsigned long long)K.d;    /* d == 1 or operands beyond 32 bits */
   if (q >= kUClamp) return kUClamp;
-  unsigned long long u = (q + 1) * cap;
+  unsigned long long u = (q + 1) * K.cap;
   return u > kUClamp ? kUClamp : (uint32_t)u;
 }
 
-__global__ void __launch_bounds__(kDecThreads)
-k_decide(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
-         const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t mode,
-         const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-         unsigned long long* st_min, unsigned long long* st_kept,
-         uint8_t* __restrict__ out_keep, long long* __restrict__ out_est,
-         uint32_t* __restrict__ out_perm, uint32_t* __restrict__ out_kept_idx,
-         unsigned long long* __restrict__ out_n_kept, uint32_t* __restrict__ out_seg_kept) {
-  constexpr int WARPS = kDecThreads / 32;
-  __shared__ uint32_t s_tile;
-  __shared__ uint32_t s_abort;
-  __shared__ int32_t s_wm[WARPS];
-  __shared__ uint32_t s_wh[WARPS];
-  __shared__ uint32_t s_wk[WARPS];
-  __shared__ int32_t s_carry_m;
-  __shared__ uint32_t s_carry_k;
+/* 32 bytes with one access; p is 32-byte aligned */
+__device__ __forceinline__ void load4(const unsigned long long* p, unsigned long long* v) {
+  asm volatile("ld.global.nc.v4.u64 {%0, %1, %2, %3}, [%4];"
+               : "=l"(v[0]), "=l"(v[1]), "=l"(v[2]), "=l"(v[3]) : "l"(p));
+}
+__device__ __forceinline__ void store4(void* p, unsigned long long a, unsigned long long b,
+                                       unsigned long long c, unsigned long long d) {
+  asm volatile("st.global.v4.u64 [%0], {%1, %2, %3, %4};" :: "l"(p), "l"(a), "l"(b), "l"(c), "l"(d) : "memory");
+}
 
-  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (hdr->wide) return;
-  if (tid == 0) {
-    s_tile = atomicAdd(&hdr->ticket[kMaxPasses], 1u);
-    s_abort = 0;
+/* First half of the decision pass for one thread's kDecItems consecutive
+ * sorted elements: decode, admission threshold u, position r inside the own
+ * queue, and the thread's running segmented reduction (admitted mode: minimum
+ * of u_t - t; raw mode: number of kept requests). */
+struct TileCtx {
+  const unsigned long long* src;
+  const PardSegConst* ktab;
+  const uint32_t* seg_off;
+  uint32_t n, ibits, imask, kshift;
+  unsigned long long dmask;
+};
+
+template <bool RAW>
+__device__ __forceinline__ void tile_first_half(const TileCtx& T, uint64_t base, unsigned long long (&e)[kDecItems],
+                                                uint32_t (&idx)[kDecItems], uint32_t (&u)[kDecItems],
+                                                uint32_t (&r)[kDecItems], int32_t (&lv)[kDecItems],
+                                                uint32_t& lheadbits, SegVal& run, PardSegConst& K,
+                                                uint32_t& sstart, uint32_t& seg_first, bool& one_seg) {
+  static_assert(kDecItems == 8, "two 32-byte loads per thread");
+  const bool full = base + kDecItems <= T.n;
+  if (full) {
+    load4(T.src + base, e);
+    load4(T.src + base + 4, e + 4);
+  } else {
+#pragma unroll
+    for (int i = 0; i < kDecItems; ++i) e[i] = base + i < T.n ? T.src[base + i] : 0;
   }
-  __syncthreads();
-  const uint32_t tile = s_tile;
-  const uint32_t npass = hdr->npass, dbits = hdr->dbits;
-  const unsigned long long* src = (npass & 1) ? buf_b : buf_a;
-  const uint64_t base = (uint64_t)tile * kDecTile + (uint64_t)tid * kDecItems;
-  const unsigned long long imask = (1ull << ibits) - 1;
-  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
-  const bool raw = mode & PARD_MODE_RAW;
-  constexpr int32_t kInf = 0x7fffffff;
-
-  uint32_t idx[kDecItems], u[kDecItems], r[kDecItems], seg[kDecItems];
-  int32_t lv[kDecItems];        /* min of u_t - t over this thread's earlier items of the same queue */
-  bool lhead[kDecItems];        /* the item's queue head is one of this thread's items up to it      */
-
-  SegMin run; run.m = kInf; run.head = 0;
+  seg_first = (uint32_t)(e[0] >> T.kshift);
+  /* most threads see one queue only: its constants are then loaded once */
+  one_seg = full && seg_first == (uint32_t)(e[kDecItems - 1] >> T.kshift);
+  K = T.ktab[seg_first];
+  sstart = T.seg_off[seg_first];
+  uint32_t cur_seg = seg_first;
+  lheadbits = 0;
+  run = seg_identity<RAW>();
 #pragma unroll
   for (int i = 0; i < kDecItems; ++i) {
-    uint64_t j = base + i;
-    if (j < n) {
-      unsigned long long e = src[j];
-      idx[i] = (uint32_t)(e & imask);
-      unsigned long long off = (e >> ibits) & dmask;
-      seg[i] = (uint32_t)((e >> ibits) >> dbits);
-      const PardSegConst K = ktab[seg[i]];
-      r[i] = (uint32_t)j - seg_off[seg[i]];
-      u[i] = threshold_u((int64_t)off - K.A_rel, K.d, K.cap);
+    const uint64_t j = base + i;
+    if (j < T.n) {
+      idx[i] = (uint32_t)e[i] & T.imask;
+      const unsigned long long off = (e[i] >> T.ibits) & T.dmask;
+      if (!one_seg) {
+        const uint32_t sg = (uint32_t)(e[i] >> T.kshift);
+        if (sg != cur_seg) {
+          cur_seg = sg;
+          K = T.ktab[sg];
+          sstart = T.seg_off[sg];
+        }
+      }
+      r[i] = (uint32_t)j - sstart;
+      u[i] = threshold_u((int64_t)off - K.A_rel, K);
     } else {
-      idx[i] = 0; seg[i] = 0; r[i] = 0; u[i] = kUClamp;     /* acts as a head, never read */
+      idx[i] = 0; r[i] = 0; u[i] = kUClamp;                    /* acts as a head, never read */
     }
-    if (r[i] == 0) { run.m = kInf; run.head = 1; }
+    if (r[i] == 0) { run = seg_identity<RAW>(); run.head = 1; }
     lv[i] = run.m;
-    lhead[i] = run.head;
-    run.m = min(run.m, (int32_t)u[i] - (int32_t)r[i]);
+    lheadbits |= run.head << i;
+    if (RAW) run.m += (r[i] < u[i] && j < T.n) ? 1 : 0;
+    else run.m = min(run.m, (int32_t)u[i] - (int32_t)r[i]);
   }
+}
 
-  /* exclusive segmented scan of the threads' aggregates: warp, then block, then tiles */
-  SegMin inc = run;
+__device__ __forceinline__ TileCtx make_tile_ctx(const PlanHeader* hdr, const unsigned long long* buf_a,
+                                                 const unsigned long long* buf_b, uint32_t n, uint32_t ibits,
+                                                 const PardSegConst* ktab, const uint32_t* seg_off) {
+  TileCtx T;
+  const uint32_t dbits = hdr->dbits;
+  T.src = (hdr->npass & 1) ? buf_b : buf_a;
+  T.ktab = ktab;
+  T.seg_off = seg_off;
+  T.n = n;
+  T.ibits = ibits;
+  T.imask = (1u << ibits) - 1;                                 /* ibits <= 30 */
+  T.kshift = ibits + dbits;                                    /* < 64 */
+  T.dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  return T;
+}
+
+/* Inclusive segmented warp scan of the threads' values (in lane order). */
+template <bool RAW>
+__device__ __forceinline__ SegVal warp_scan(SegVal v, uint32_t lane) {
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    SegMin l;
-    l.m = __shfl_up_sync(0xffffffffu, inc.m, o);
-    l.head = __shfl_up_sync(0xffffffffu, inc.head, o);
-    if (lane >= (uint32_t)o) inc = seg_combine(l, inc);
+    SegVal l;
+    l.m = __shfl_up_sync(0xffffffffu, v.m, o);
+    l.head = __shfl_up_sync(0xffffffffu, v.head, o);
+    if (lane >= (uint32_t)o) v = seg_combine<RAW>(l, v);
   }
-  SegMin exc;
-  exc.m = __shfl_up_sync(0xffffffffu, inc.m, 1);
-  exc.head = __shfl_up_sync(0xffffffffu, inc.head, 1);
-  if (lane == 0) { exc.m = kInf; exc.head = 0; }
+  return v;
+}
+
+/* Tile aggregates: the segmented reduction over each tile of kDecTile sorted
+ * elements.  Tiles are independent; k_tile_scan turns the aggregates into the
+ * value carried into every tile, so that the decision kernel never waits on
+ * another block. */
+template <bool RAW>
+__global__ void __launch_bounds__(kDecThreads)
+k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+           const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
+           const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+           unsigned long long* __restrict__ tile_agg) {
+  constexpr int WARPS = kDecThreads / 32;
+  __shared__ int32_t s_wm[WARPS];
+  __shared__ uint32_t s_wh[WARPS];
+  if (hdr->wide) return;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
+  const uint64_t base = (uint64_t)blockIdx.x * kDecTile + (uint64_t)tid * kDecItems;
+  unsigned long long e[kDecItems];
+  uint32_t idx[kDecItems], u[kDecItems], r[kDecItems], lheadbits, sstart, seg_first;
+  int32_t lv[kDecItems];
+  SegVal run;
+  PardSegConst K;
+  bool one_seg;
+  tile_first_half<RAW>(T, base, e, idx, u, r, lv, lheadbits, run, K, sstart, seg_first, one_seg);
+  const SegVal inc = warp_scan<RAW>(run, lane);
   if (lane == 31) { s_wm[warp] = inc.m; s_wh[warp] = inc.head; }
   __syncthreads();
-  SegMin wprefix; wprefix.m = kInf; wprefix.head = 0;
-  SegMin tile_agg; tile_agg.m = kInf; tile_agg.head = 0;
+  if (tid == 0) {
+    SegVal agg = seg_identity<RAW>();
 #pragma unroll
-  for (int w = 0; w < WARPS; ++w) {
-    SegMin a; a.m = s_wm[w]; a.head = s_wh[w];
-    if (w < (int)warp) wprefix = seg_combine(wprefix, a);
-    tile_agg = seg_combine(tile_agg, a);
+    for (int w = 0; w < WARPS; ++w) {
+      SegVal a; a.m = s_wm[w]; a.head = s_wh[w];
+      agg = seg_combine<RAW>(agg, a);
+    }
+    tile_agg[blockIdx.x] = pack_val(agg, 0);
   }
-  exc = seg_combine(wprefix, exc);
+}
 
-  if (!raw) {
-    if (tid == 0) {
-      volatile unsigned long long* st = st_min;
-      st[tile] = pack_min(tile_agg, kStAgg);
-      SegMin carry; carry.m = kInf; carry.head = 0;
-      bool first = true;
-      for (int64_t t = (int64_t)tile - 1; t >= 0; --t) {
-        unsigned long long w;
-        uint32_t spins = 0;
-        while (((w = st[t]) >> 62) == 0) {
-          if (++spins > kSpinLimit) { s_abort = 1; break; }
-          __nanosleep(20);
-        }
-        if ((w >> 62) == 0) break;
-        SegMin a = unpack_min(w);
-        carry = first ? a : seg_combine(a, carry);
-        first = false;
-        if ((w >> 62) == 2 || carry.head) break;     /* nothing before a queue head matters */
-      }
-      SegMin incl = seg_combine(carry, tile_agg);
-      st[tile] = pack_min(incl, kStIncl);
-      s_carry_m = carry.m;
+/* Exclusive segmented scan of the tile aggregates by one block, eight tiles
+ * per thread and round: carry[t] is the reduction over the elements that
+ * precede tile t in the queue that is open at the start of tile t. */
+template <bool RAW>
+__global__ void __launch_bounds__(1024)
+k_tile_scan(const unsigned long long* __restrict__ tile_agg, uint32_t n_tiles, int32_t* __restrict__ carry) {
+  constexpr int PER = 8;
+  __shared__ int32_t s_wm[32];
+  __shared__ uint32_t s_wh[32];
+  __shared__ int32_t s_cm;
+  __shared__ uint32_t s_ch;
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) { s_cm = seg_identity<RAW>().m; s_ch = 0; }
+  __syncthreads();
+  for (uint32_t b = 0; b < n_tiles; b += 1024 * PER) {
+    const uint32_t t0 = b + threadIdx.x * PER;
+    SegVal v[PER];
+    SegVal run = seg_identity<RAW>();
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      v[k] = t0 + k < n_tiles ? unpack_val(tile_agg[t0 + k]) : seg_identity<RAW>();
+      run = seg_combine<RAW>(run, v[k]);
+    }
+    const SegVal inc = warp_scan<RAW>(run, lane);
+    SegVal exc;
+    exc.m = __shfl_up_sync(0xffffffffu, inc.m, 1);
+    exc.head = __shfl_up_sync(0xffffffffu, inc.head, 1);
+    if (lane == 0) exc = seg_identity<RAW>();
+    if (lane == 31) { s_wm[warp] = inc.m; s_wh[warp] = inc.head; }
+    __syncthreads();
+    if (warp == 0) {                        /* scan of the 32 warp aggregates, led by the carry */
+      SegVal a; a.m = s_wm[lane]; a.head = s_wh[lane];
+      SegVal ai = warp_scan<RAW>(a, lane);
+      SegVal ae;
+      ae.m = __shfl_up_sync(0xffffffffu, ai.m, 1);
+      ae.head = __shfl_up_sync(0xffffffffu, ai.head, 1);
+      if (lane == 0) ae = seg_identity<RAW>();
+      SegVal c0; c0.m = s_cm; c0.head = s_ch;
+      ae = seg_combine<RAW>(c0, ae);
+      const SegVal all = seg_combine<RAW>(c0, ai);
+      s_wm[lane] = ae.m; s_wh[lane] = ae.head;
+      __syncwarp();
+      if (lane == 31) { s_cm = all.m; s_ch = all.head; }
     }
     __syncthreads();
-    if (s_abort) {
-      if (tid == 0) set_status(hdr, PARD_ETIMEOUT);
-      return;
+    SegVal pre; pre.m = s_wm[warp]; pre.head = s_wh[warp];
+    pre = seg_combine<RAW>(pre, exc);
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      if (t0 + k < n_tiles) carry[t0 + k] = pre.m;
+      pre = seg_combine<RAW>(pre, v[k]);
     }
-    if (!exc.head) exc.m = min(exc.m, s_carry_m);
+    __syncthreads();
   }
+}
+
+/* Decision pass; one tile of kDecTile sorted elements per block, a thread owns
+ * kDecItems consecutive elements.
+ *
+ * Admitted mode: c_r = min(r, r-1 + min_{t<r}(u_t - t)) by a segmented
+ * exclusive prefix-min; raw mode: c_r = r, and the kept requests ahead in the
+ * queue are counted by a segmented exclusive prefix-sum.  Either way the
+ * number k_r of kept requests ahead in the own queue is known per request, and
+ * a kept request's index goes to kept_tmp[first position of its queue + k_r]:
+ * every queue's survivors end up contiguous, k_kept_move packs the queues. */
+template <bool RAW>
+__global__ void __launch_bounds__(kDecThreads)
+k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+         const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
+         const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+         const int32_t* __restrict__ carry, uint8_t* __restrict__ out_keep,
+         long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
+         uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept) {
+  constexpr int WARPS = kDecThreads / 32;
+  __shared__ int32_t s_wm[WARPS];
+  __shared__ uint32_t s_wh[WARPS];
+  if (hdr->wide) return;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
+  const uint32_t tile = blockIdx.x;
+  const uint64_t base = (uint64_t)tile * kDecTile + (uint64_t)tid * kDecItems;
+  const bool full = base + kDecItems <= n;
+  const int32_t tile_carry = carry[tile];
+
+  unsigned long long e[kDecItems];
+  uint32_t idx[kDecItems], u[kDecItems], r[kDecItems], lheadbits, sstart, seg_first;
+  int32_t lv[kDecItems];     /* reduction over this thread's earlier items of the same queue */
+  SegVal run;
+  PardSegConst K;
+  bool one_seg;
+  tile_first_half<RAW>(T, base, e, idx, u, r, lv, lheadbits, run, K, sstart, seg_first, one_seg);
+
+  /* exclusive segmented scan of the threads' aggregates: warp, block, then the tile's carry */
+  const SegVal inc = warp_scan<RAW>(run, lane);
+  SegVal exc;
+  exc.m = __shfl_up_sync(0xffffffffu, inc.m, 1);
+  exc.head = __shfl_up_sync(0xffffffffu, inc.head, 1);
+  if (lane == 0) exc = seg_identity<RAW>();
+  if (lane == 31) { s_wm[warp] = inc.m; s_wh[warp] = inc.head; }
+  __syncthreads();
+  SegVal wprefix; wprefix.m = tile_carry; wprefix.head = 0;
+#pragma unroll
+  for (int w = 0; w < WARPS; ++w) {
+    SegVal a; a.m = s_wm[w]; a.head = s_wh[w];
+    if (w < (int)warp) wprefix = seg_combine<RAW>(wprefix, a);
+  }
+  exc = seg_combine<RAW>(wprefix, exc);
 
   /* admitted position, estimate, decision */
   uint32_t keepbits = 0;
   long long est[kDecItems];
-  uint32_t cpos[kDecItems];
+  uint32_t cur_seg = seg_first;
+  uint32_t send = seg_off[seg_first + 1];
+  if (!one_seg) {
+    K = ktab[seg_first];
+    sstart = seg_off[seg_first];
+  }
 #pragma unroll
   for (int i = 0; i < kDecItems; ++i) {
-    uint32_t c;
-    if (raw || r[i] == 0) {
-      c = r[i];
-    } else {
-      int32_t pm = lhead[i] ? lv[i] : min(lv[i], exc.m);   /* min over t < r of (u_t - t) */
-      int64_t cc = (int64_t)r[i] - 1 + pm;
-      c = cc < (int64_t)r[i] ? (uint32_t)cc : r[i];
+    const bool valid = base + i < n;
+    if (!one_seg && valid) {
+      const uint32_t sg = (uint32_t)(e[i] >> T.kshift);
+      if (sg != cur_seg) {
+        cur_seg = sg;
+        K = ktab[sg];
+        sstart = seg_off[sg];
+        send = seg_off[sg + 1];
+      }
     }
-    cpos[i] = c;
-    const PardSegConst K = ktab[seg[i]];
-    est[i] = K.A + (long long)(c / K.cap) * K.d;
-    if (c < u[i] && base + i < n) keepbits |= 1u << i;
+    /* reduction over the earlier requests of the same queue */
+    const bool local = (lheadbits >> i) & 1u;
+    const int32_t pre = local ? lv[i] : (RAW ? lv[i] + exc.m : min(lv[i], exc.m));
+    uint32_t c, ahead;            /* batch-slot position; kept requests ahead in the queue */
+    if (RAW) {
+      c = r[i];
+      ahead = r[i] == 0 ? 0u : (uint32_t)pre;
+    } else {
+      if (r[i] == 0) {
+        c = 0;
+      } else {
+        const int64_t cc = (int64_t)r[i] - 1 + pre;               /* r-1 + min over t < r of (u_t - t) */
+        c = cc < (int64_t)r[i] ? (uint32_t)cc : r[i];
+      }
+      ahead = c;
+    }
+    const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;     /* floor(c / cap) */
+    est[i] = K.A + (long long)round * K.d;
+    const uint32_t kept = (c < u[i] && valid) ? 1u : 0u;
+    keepbits |= kept << i;
+    if (kept && kept_tmp) kept_tmp[sstart + ahead] = idx[i];
+    /* the last request of a queue knows the queue's kept count */
+    if (valid && (uint32_t)(base + i) + 1 == send) seg_kept[cur_seg] = ahead + kept;
   }
 
-  const uint64_t nrem = base < n ? (uint64_t)n - base : 0;
-  if (nrem >= kDecItems) {
+  if (full) {
     if (out_keep) {
       unsigned long long kb = 0;
 #pragma unroll
@@ -646,96 +869,84 @@ k_decide(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
       *reinterpret_cast<unsigned long long*>(out_keep + base) = kb;
     }
     if (out_est) {
-#pragma unroll
-      for (int i = 0; i < kDecItems; i += 2)
-        *reinterpret_cast<longlong2*>(out_est + base + i) = make_longlong2(est[i], est[i + 1]);
+      store4(out_est + base, est[0], est[1], est[2], est[3]);
+      store4(out_est + base + 4, est[4], est[5], est[6], est[7]);
     }
-    if (out_perm) {
-#pragma unroll
-      for (int i = 0; i < kDecItems; i += 4)
-        *reinterpret_cast<uint4*>(out_perm + base + i) = make_uint4(idx[i], idx[i + 1], idx[i + 2], idx[i + 3]);
-    }
+    if (out_perm)
+      store4(out_perm + base, idx[0] | ((unsigned long long)idx[1] << 32),
+             idx[2] | ((unsigned long long)idx[3] << 32), idx[4] | ((unsigned long long)idx[5] << 32),
+             idx[6] | ((unsigned long long)idx[7] << 32));
   } else {
-    for (int i = 0; i < (int)nrem; ++i) {
-      if (out_keep) out_keep[base + i] = (keepbits >> i) & 1u;
-      if (out_est) out_est[base + i] = est[i];
-      if (out_perm) out_perm[base + i] = idx[i];
-    }
-  }
-  if (out_seg_kept && !raw) {
-    /* the last request of a queue knows the queue's kept count */
 #pragma unroll
     for (int i = 0; i < kDecItems; ++i)
-      if (base + i < n && (uint32_t)(base + i) + 1 == seg_off[seg[i] + 1])
-        out_seg_kept[seg[i]] = cpos[i] + ((keepbits >> i) & 1u);
-  }
-  if (out_seg_kept && raw) {
-    /* kept requests are not a running count here: add them up per queue */
-    const bool one_seg = nrem >= kDecItems && seg[0] == seg[kDecItems - 1];
-    const uint32_t s0 = __shfl_sync(0xffffffffu, seg[0], 0);
-    if (__all_sync(0xffffffffu, one_seg && seg[0] == s0)) {
-      uint32_t x = __popc(keepbits);
-      for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-      if (lane == 0 && x) atomicAdd(&out_seg_kept[s0], x);
-    } else {
-      uint32_t run = 0;
-      for (int i = 0; i < kDecItems && base + i < n; ++i) {
-        run += (keepbits >> i) & 1u;
-        if (i + 1 == kDecItems || base + i + 1 >= n || seg[i + 1] != seg[i]) {
-          if (run) atomicAdd(&out_seg_kept[seg[i]], run);
-          run = 0;
-        }
+      if (base + i < n) {
+        if (out_keep) out_keep[base + i] = (keepbits >> i) & 1u;
+        if (out_est) out_est[base + i] = est[i];
+        if (out_perm) out_perm[base + i] = idx[i];
       }
-    }
   }
+}
 
-  /* compaction: positions of the kept requests among all kept requests */
-  if (out_kept_idx || out_n_kept) {
-    uint32_t mine = __popc(keepbits), x = mine;
-#pragma unroll
+/* Kept requests per queue -> first output slot of every queue, the number of
+ * kCompactChunk-sized copy jobs before every queue, and the total.  One block. */
+__global__ void __launch_bounds__(1024)
+k_kept_scan(const uint32_t* __restrict__ seg_kept, uint32_t n_seg, uint32_t* __restrict__ kept_base,
+            uint32_t* __restrict__ chunk_base, uint32_t* __restrict__ out_seg_kept,
+            unsigned long long* __restrict__ out_n_kept) {
+  __shared__ uint32_t s_a[32], s_b[32];
+  __shared__ uint32_t s_ca, s_cb;
+  if (threadIdx.x == 0) { s_ca = 0; s_cb = 0; }
+  __syncthreads();
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (uint32_t base = 0; base < n_seg + 1; base += 1024) {
+    const uint32_t i = base + threadIdx.x;
+    const uint32_t v = i < n_seg ? seg_kept[i] : 0;
+    const uint32_t c = (v + kCompactChunk - 1) / kCompactChunk;
+    if (out_seg_kept && i < n_seg) out_seg_kept[i] = v;
+    uint32_t x = v, y = c;
     for (int o = 1; o < 32; o <<= 1) {
-      uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= (uint32_t)o) x += y;
+      uint32_t p = __shfl_up_sync(0xffffffffu, x, o), q = __shfl_up_sync(0xffffffffu, y, o);
+      if (lane >= (uint32_t)o) { x += p; y += q; }
     }
-    if (lane == 31) s_wk[warp] = x;
+    if (lane == 31) { s_a[warp] = x; s_b[warp] = y; }
     __syncthreads();
-    uint32_t wpre = 0, total = 0;
-#pragma unroll
-    for (int w = 0; w < WARPS; ++w) {
-      if (w < (int)warp) wpre += s_wk[w];
-      total += s_wk[w];
-    }
-    if (tid == 0) {
-      volatile unsigned long long* st = st_kept;
-      st[tile] = kStAgg | total;
-      unsigned long long excl = 0;
-      for (int64_t t = (int64_t)tile - 1; t >= 0; --t) {
-        unsigned long long w;
-        uint32_t spins = 0;
-        while (((w = st[t]) >> 62) == 0) {
-          if (++spins > kSpinLimit) { s_abort = 1; break; }
-          __nanosleep(20);
-        }
-        if ((w >> 62) == 0) break;
-        excl += w & 0xffffffffull;
-        if ((w >> 62) == 2) break;
+    if (warp == 0) {
+      uint32_t a = s_a[lane], b = s_b[lane], ta = a, tb = b;
+      for (int o = 1; o < 32; o <<= 1) {
+        uint32_t p = __shfl_up_sync(0xffffffffu, ta, o), q = __shfl_up_sync(0xffffffffu, tb, o);
+        if (lane >= (uint32_t)o) { ta += p; tb += q; }
       }
-      st[tile] = kStIncl | (excl + total);
-      s_carry_k = (uint32_t)excl;
-      if (out_n_kept && (uint64_t)(tile + 1) * kDecTile >= n) *out_n_kept = excl + total;
+      s_a[lane] = ta - a;
+      s_b[lane] = tb - b;
     }
     __syncthreads();
-    if (s_abort) {
-      if (tid == 0) set_status(hdr, PARD_ETIMEOUT);
-      return;
-    }
-    if (out_kept_idx) {
-      uint32_t pos = s_carry_k + wpre + x - mine;
-#pragma unroll
-      for (int i = 0; i < kDecItems; ++i)
-        if ((keepbits >> i) & 1u) out_kept_idx[pos++] = idx[i];
-    }
+    const uint32_t ea = s_ca + s_a[warp] + x - v, eb = s_cb + s_b[warp] + y - c;
+    if (i <= n_seg) { kept_base[i] = ea; chunk_base[i] = eb; }
+    __syncthreads();
+    if (threadIdx.x == 1023) { s_ca = ea + v; s_cb = eb + c; }
+    __syncthreads();
   }
+  if (threadIdx.x == 0 && out_n_kept) *out_n_kept = s_ca;
+}
+
+/* Packs the queues' survivors: copy job b moves up to kCompactChunk indices of one queue. */
+__global__ void __launch_bounds__(256)
+k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ seg_off,
+            const uint32_t* __restrict__ seg_kept, const uint32_t* __restrict__ kept_base,
+            const uint32_t* __restrict__ chunk_base, uint32_t n_seg, uint32_t* __restrict__ out_kept_idx) {
+  const uint32_t job = blockIdx.x;
+  if (job >= chunk_base[n_seg]) return;
+  uint32_t lo = 0, hi = n_seg;                 /* last queue whose first job is <= job */
+  while (hi - lo > 1) {
+    const uint32_t mid = lo + (hi - lo) / 2;
+    if (chunk_base[mid] <= job) lo = mid; else hi = mid;
+  }
+  const uint32_t s = lo;
+  const uint32_t first = (job - chunk_base[s]) * kCompactChunk;
+  const uint32_t count = min((uint32_t)kCompactChunk, seg_kept[s] - first);
+  const uint32_t* src = kept_tmp + seg_off[s] + first;
+  uint32_t* dst = out_kept_idx + kept_base[s] + first;
+  for (uint32_t i = threadIdx.x; i < count; i += blockDim.x) dst[i] = src[i];
 }
 
 /* ---- optional phase timing (process-wide) ---- */
@@ -825,8 +1036,13 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   PardSegConst* ktab = (PardSegConst*)(ws + L.ktab);
   uint32_t* hist = (uint32_t*)(ws + L.hist);
   uint32_t* lookback = (uint32_t*)(ws + L.lookback);
-  unsigned long long* st_min = (unsigned long long*)(ws + L.st_min);
-  unsigned long long* st_kept = (unsigned long long*)(ws + L.st_kept);
+  const size_t lb_words = (size_t)L.sort_tiles * kBins;
+  unsigned long long* tile_agg = (unsigned long long*)(ws + L.tile_agg);
+  int32_t* tile_carry = (int32_t*)(ws + L.tile_carry);
+  uint32_t* seg_kept = (uint32_t*)(ws + L.seg_kept);
+  uint32_t* kept_base = (uint32_t*)(ws + L.kept_base);
+  uint32_t* chunk_base = (uint32_t*)(ws + L.chunk_base);
+  uint32_t* kept_tmp = (uint32_t*)(ws + L.kept_tmp);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -841,19 +1057,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     ++phase;
   };
   mark();
-  /* ---- clear the scratch that must start at zero ---- */
-  PARD_CUDA_OK(cudaMemsetAsync(ws + L.hdr, 0, sizeof(PlanHeader), stream));
-  PARD_CUDA_OK(cudaMemsetAsync(ctx_dmin, 0xff, 8ull * n_ctx, stream));
-  PARD_CUDA_OK(cudaMemsetAsync(ctx_dmax, 0, 8ull * n_ctx, stream));
-  PARD_CUDA_OK(cudaMemsetAsync(seg_off, 0, 4ull * (L.n_seg + 1), stream));
-  PARD_CUDA_OK(cudaMemsetAsync(hist, 0, 4ull * kMaxPasses * kBins, stream));
-  if (n > 0) {
-    PARD_CUDA_OK(cudaMemsetAsync(lookback, 0, 4ull * kBins * (uint64_t)L.sort_tiles * L.max_passes, stream));
-    PARD_CUDA_OK(cudaMemsetAsync(st_min, 0, 8ull * L.dec_tiles, stream));
-    PARD_CUDA_OK(cudaMemsetAsync(st_kept, 0, 8ull * L.dec_tiles, stream));
-  }
-  if (out->d_seg_kept) PARD_CUDA_OK(cudaMemsetAsync(out->d_seg_kept, 0, 4ull * L.n_seg, stream));
-  if (out->d_n_kept) PARD_CUDA_OK(cudaMemsetAsync(out->d_n_kept, 0, 8, stream));
+  /* ---- clear the scratch that must start at zero: one contiguous region ---- */
+  PARD_CUDA_OK(cudaMemsetAsync(ws + L.hdr, 0, n > 0 ? L.zero_end : L.lookback, stream));
   PARD_CUDA_OK(cudaMemcpyAsync(d_pipes, h_pipes.data(), 8ull * n_pipelines, cudaMemcpyHostToDevice, stream));
 
   int sms = 148;
@@ -870,8 +1075,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   }
   mark();
   if (n > 0) k_ctx_span<<<(n_ctx + 255) / 256, 256, 0, stream>>>(ctx_dmin, ctx_dmax, n_ctx, hdr);
-  k_seg_scan<<<1, 1024, 0, stream>>>(seg_off, L.n_seg, out->d_seg_offsets, sbits, ibits, hdr);
-  k_seg_const<<<(L.n_seg + 127) / 128, 128, 0, stream>>>(d_pipes, n_pipelines, *state, n_ctx, ctx_dmin,
+  k_seg_scan<<<1, 1024, 0, stream>>>(seg_off, L.n_seg, out->d_seg_offsets, out->d_seg_kept, sbits, ibits, hdr);
+  k_seg_const<<<(L.n_seg + 3) / 4, 128, 0, stream>>>(d_pipes, n_pipelines, *state, n_ctx, ctx_dmin,
                                                          seg_off, ktab, hdr);
   mark();
   if (n > 0) {
@@ -882,15 +1087,31 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     mark();
     if (n > 0 && p < L.max_passes)
       k_sort_pass<<<L.sort_tiles, kSortThreads, 0, stream>>>(
-          p, hdr, buf_a, buf_b, hist, lookback + (size_t)p * L.sort_tiles * kBins, n32, ibits);
+          p, hdr, buf_a, buf_b, hist, lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words,
+          n32, ibits);
   }
   mark();
   if (n > 0) {
-    k_decide<<<L.dec_tiles, kDecThreads, 0, stream>>>(
-        hdr, buf_a, buf_b, n32, ibits, mode, ktab, seg_off, st_min, st_kept, out->d_keep,
-        (long long*)out->d_est_us, out->d_perm, out->d_kept_idx,
-        (unsigned long long*)out->d_n_kept, out->d_seg_kept);
+    uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
+    if (mode & PARD_MODE_RAW) {
+      k_tile_agg<true><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
+      k_tile_scan<true><<<1, 1024, 0, stream>>>(tile_agg, L.dec_tiles, tile_carry);
+      k_decide<true><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+                                                              out->d_keep, (long long*)out->d_est_us, out->d_perm,
+                                                              tmp, seg_kept);
+    } else {
+      k_tile_agg<false><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
+      k_tile_scan<false><<<1, 1024, 0, stream>>>(tile_agg, L.dec_tiles, tile_carry);
+      k_decide<false><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+                                                               out->d_keep, (long long*)out->d_est_us, out->d_perm,
+                                                               tmp, seg_kept);
+    }
   }
+  k_kept_scan<<<1, 1024, 0, stream>>>(seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+                                      (unsigned long long*)out->d_n_kept);
+  if (n > 0 && out->d_kept_idx)
+    k_kept_move<<<(uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg, 256, 0, stream>>>(
+        kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
   mark();
   PARD_CUDA_OK(cudaGetLastError());
   if (mode & PARD_MODE_NOWAIT) return PARD_OK;
@@ -913,8 +1134,9 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* seg_scan + seg_const always; prepass, ctx_span, pack, passes, decide when n > 0 */
-  *launches = n > 0 ? 2 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 1 : 2;
+  /* seg_scan, seg_const, kept_scan always; prepass, ctx_span, pack, passes, decide and
+   * tile_agg, tile_scan and kept_move (when the compacted indices are requested) when n > 0 */
+  *launches = n > 0 ? 3 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 4 : 3;
   return PARD_OK;
 }
 

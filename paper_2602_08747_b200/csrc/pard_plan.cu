@@ -25,7 +25,7 @@ constexpr uint32_t kUClamp = (1u << 30) - 1;       /* >= any request count      
 constexpr uint32_t kMaxPipelinesPerCall = 65536;
 constexpr uint32_t kSpinLimit = 1u << 22;          /* polls before giving up    */
 
-constexpr int kSortThreads = 256;
+constexpr int kSortThreads = 512;
 constexpr int kSortItems = 16;
 constexpr int kSortTile = kSortThreads * kSortItems;
 constexpr int kDecThreads = 256;
@@ -368,145 +368,179 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
 /* ------------------------------------------------------------------------ */
 /* one LSD radix pass (8 bits), stable, tile prefixes by decoupled look-back */
 /* ------------------------------------------------------------------------ */
-__global__ void __launch_bounds__(kSortThreads, 3)
+/* Tile = kSortTile elements, warp w owns the consecutive elements
+ * [w*32*kSortItems, (w+1)*32*kSortItems) and visits them 32 at a time, so the
+ * tile order is (warp, round, lane).
+ *   1. every warp counts its digits (shared atomics, order irrelevant);
+ *   2. thread d turns the counts of digit d into the first tile-local slot of
+ *      every (warp, digit) and publishes the tile's count for the look-back;
+ *   3. the lower part of the block adds up the counts of all earlier tiles
+ *      (look-back, kLookBatch tiles per memory round trip) while the other
+ *      warps already rank;
+ *   4. ranking: the lanes that hold the same digit find each other through a
+ *      shared word (atomic OR), take consecutive slots in lane order and drop
+ *      their elements into the shared tile buffer, now sorted by digit;
+ *   5. the buffer is written out, run by run, to the digit's global range.
+ * Large tiles keep the number of tiles in flight, and with it the depth of the
+ * look-back, small. */
+/* loads and stores of look-back words: relaxed, device scope (other blocks write them) */
+__device__ __forceinline__ uint32_t ld_relaxed(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_relaxed(uint32_t* p, uint32_t v) {
+  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+
+struct SortSmem {
+  unsigned long long keys[kSortTile];
+  uint32_t slot[kSortThreads / 32][kBins];    /* counts, then next free tile-local slot per (warp, digit) */
+  uint32_t match[kSortThreads / 32][kBins];   /* lanes currently holding the digit */
+  uint32_t dstart[kBins];
+  uint32_t gofs[kBins];
+  uint32_t scan[2][kSortThreads / 32];
+  uint32_t tile;
+  uint32_t abort;
+};
+
+__global__ void __launch_bounds__(kSortThreads, 2)
 k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf_a,
             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ hist,
             uint32_t* __restrict__ lookback, uint32_t* __restrict__ lookback_next, uint32_t n,
             uint32_t ibits) {
   constexpr int WARPS = kSortThreads / 32;
-  /* the match words are only used while ranking, the key buffer only afterwards */
-  __shared__ __align__(16) unsigned long long s_keys[kSortTile];
-  uint32_t (*s_match)[kBins] = reinterpret_cast<uint32_t (*)[kBins]>(s_keys);
-  static_assert(sizeof(uint32_t) * WARPS * kBins <= sizeof(unsigned long long) * kSortTile, "alias fits");
-  __shared__ uint32_t s_whist[WARPS][kBins];
-  __shared__ uint32_t s_dstart[kBins];
-  __shared__ uint32_t s_gofs[kBins];
-  __shared__ uint32_t s_scan[WARPS];
-  __shared__ uint32_t s_tile;
-  __shared__ uint32_t s_abort;
+  static_assert(kSortThreads >= kBins && kSortThreads % 32 == 0, "one thread per digit in the lower part");
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  SortSmem& S = *reinterpret_cast<SortSmem*>(smem_raw);
 
   if (pass >= hdr->npass) return;
   const unsigned long long* src = (pass & 1) ? buf_b : buf_a;
   unsigned long long* dst = (pass & 1) ? buf_a : buf_b;
   hist += pass * kBins;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) {
-    s_tile = atomicAdd(&hdr->ticket[pass], 1u);
-    s_abort = 0;
-  }
-  for (int w = 0; w < WARPS; ++w) { s_whist[w][tid] = 0; s_match[w][tid] = 0; }
   const uint32_t lanebit = 1u << lane;
+  if (tid == 0) {
+    S.tile = atomicAdd(&hdr->ticket[pass], 1u);
+    S.abort = 0;
+  }
+  for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) {
+    (&S.slot[0][0])[i] = 0;
+    (&S.match[0][0])[i] = 0;
+  }
+  const uint32_t gh = tid < kBins ? hist[tid] : 0;     /* global count of digit tid, needed in step 2 */
   __syncthreads();
-  const uint32_t tile = s_tile;
+  const uint32_t tile = S.tile;
   const uint64_t base = (uint64_t)tile * kSortTile;
   const uint32_t shift = ibits + 8 * pass;
 
+  /* 1. load and count */
   unsigned long long key[kSortItems];
-  uint32_t rank[kSortItems];
 #pragma unroll
   for (int i = 0; i < kSortItems; ++i) {
-    uint64_t j = base + warp * (32 * kSortItems) + i * 32 + lane;
+    const uint64_t j = base + warp * (32 * kSortItems) + i * 32 + lane;
     key[i] = j < n ? src[j] : ~0ull;
   }
 #pragma unroll
-  for (int i = 0; i < kSortItems; ++i) {
-    uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
-    /* lanes of the warp that hold the same digit meet in a shared word: every
-     * lane ORs its bit into the word of its digit and reads the union back
-     * (the hardware match instruction and eight votes both cost far more) */
-    atomicOr(&s_match[warp][d], lanebit);
-    __syncwarp();
-    const uint32_t grp = s_match[warp][d];
-    const uint32_t below = grp & (lanebit - 1);
-    const uint32_t old = s_whist[warp][d];               /* same word for the whole group */
-    __syncwarp();
-    if (below == 0) {                                    /* lowest lane of the group */
-      s_whist[warp][d] = old + __popc(grp);
-      s_match[warp][d] = 0;
+  for (int i = 0; i < kSortItems; ++i) atomicAdd(&S.slot[warp][(uint32_t)(key[i] >> shift) & 255u], 1u);
+  __syncthreads();
+
+  /* 2. thread d owns digit d */
+  uint32_t cnt = 0, x = 0, g = 0;
+  if (tid < kBins) {
+#pragma unroll
+    for (int w = 0; w < WARPS; ++w) {
+      const uint32_t t = S.slot[w][tid];
+      S.slot[w][tid] = cnt;                            /* exclusive over the warps */
+      cnt += t;
     }
-    rank[i] = old + __popc(below);
-    __syncwarp();
+    x = cnt;
+    g = gh;
+    for (int o = 1; o < 32; o <<= 1) {                 /* scans over the 256 digits */
+      const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+      const uint32_t z = __shfl_up_sync(0xffffffffu, g, o);
+      if (lane >= (uint32_t)o) { x += y; g += z; }
+    }
+    if (lane == 31) { S.scan[0][warp] = x; S.scan[1][warp] = g; }
+    /* the tile's count is all that later tiles need from this one for now */
+    st_relaxed(lookback + (size_t)tile * kBins + tid, cnt | kLbAgg);
+    lookback_next[(size_t)tile * kBins + tid] = 0;     /* the array of the pass after this one */
+  }
+  __syncthreads();
+  uint32_t dstart = 0, gstart = 0;
+  if (tid < kBins) {
+    uint32_t wx = 0, wg = 0;
+#pragma unroll
+    for (int w = 0; w < kBins / 32; ++w)
+      if (w < (int)warp) { wx += S.scan[0][w]; wg += S.scan[1][w]; }
+    dstart = wx + x - cnt;                             /* first tile-local slot of digit tid  */
+    gstart = wg + g - gh;                              /* first global position of digit tid  */
+    S.dstart[tid] = dstart;
+#pragma unroll
+    for (int w = 0; w < WARPS; ++w) S.slot[w][tid] += dstart;
   }
   __syncthreads();
 
-  /* thread d owns digit d: counts across warps -> exclusive warp offsets */
-  uint32_t cnt = 0;
+  /* 3. look-back by the lower part of the block; the other warps go on */
+  if (tid < kBins) {
+    const uint32_t* lb = lookback;
+    uint32_t excl = 0, spins = 0;
+    int64_t t = (int64_t)tile - 1;
+    bool done = t < 0;
+    while (!done) {
+      uint32_t v[kLookBatch];
 #pragma unroll
-  for (int w = 0; w < WARPS; ++w) {
-    uint32_t t = s_whist[w][tid];
-    s_whist[w][tid] = cnt;
-    cnt += t;
-  }
-  /* exclusive scans over the 256 digits: the tile's counts and the global histogram */
-  uint32_t gh = hist[tid];
-  uint32_t x = cnt, g = gh;
-  for (int o = 1; o < 32; o <<= 1) {
-    uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
-    uint32_t z = __shfl_up_sync(0xffffffffu, g, o);
-    if (lane >= (uint32_t)o) { x += y; g += z; }
-  }
-  __shared__ uint32_t s_scan_g[WARPS];
-  if (lane == 31) { s_scan[warp] = x; s_scan_g[warp] = g; }
-  __syncthreads();
-  uint32_t wx = 0, wg = 0;
+      for (int k = 0; k < kLookBatch; ++k)
+        v[k] = (t - k >= 0) ? ld_relaxed(lb + (size_t)(t - k) * kBins + tid) : +kLbIncl;   /* before tile 0: nothing */
+      int used = 0;
 #pragma unroll
-  for (int w = 0; w < WARPS; ++w)
-    if (w < (int)warp) { wx += s_scan[w]; wg += s_scan_g[w]; }
-  const uint32_t dstart = wx + x - cnt;        /* first local position of digit tid  */
-  const uint32_t gstart = wg + g - gh;         /* first global position of digit tid */
-  s_dstart[tid] = dstart;
-
-  /* publish the tile's count, then sum the counts of all earlier tiles.  The
-   * words of kLookBatch earlier tiles are requested together, so a long run
-   * of tiles that have only published their own count costs one memory round
-   * trip per batch instead of one per tile. */
-  volatile uint32_t* lb = lookback;            /* this pass's array */
-  lb[(size_t)tile * kBins + tid] = cnt | kLbAgg;
-  lookback_next[(size_t)tile * kBins + tid] = 0;          /* the array of the pass after this one */
-  uint32_t excl = 0, spins = 0;
-  int64_t t = (int64_t)tile - 1;
-  bool done = t < 0;
-  while (!done) {
-    uint32_t v[kLookBatch];
-#pragma unroll
-    for (int k = 0; k < kLookBatch; ++k)
-      v[k] = (t - k >= 0) ? lb[(size_t)(t - k) * kBins + tid] : +kLbIncl;   /* before tile 0: nothing */
-    int used = 0;
-#pragma unroll
-    for (int k = 0; k < kLookBatch; ++k) {
-      if (!done && used == k) {
-        if ((v[k] >> 30) != 0) {
+      for (int k = 0; k < kLookBatch; ++k) {
+        if (!done && used == k && (v[k] >> 30) != 0) {
           excl += v[k] & kLbMask;
           used = k + 1;
           if (v[k] & kLbIncl) done = true;
         }
       }
+      t -= used;
+      if (!done && used < kLookBatch) {                /* met a tile that has not published yet */
+        if (++spins > kSpinLimit) { S.abort = 1; break; }
+        __nanosleep(40);
+      }
     }
-    t -= used;
-    if (!done && used < kLookBatch) {          /* met a tile that has not published yet */
-      if (++spins > kSpinLimit) { s_abort = 1; break; }
-      __nanosleep(40);
-    }
+    st_relaxed(lookback + (size_t)tile * kBins + tid, ((excl + cnt) & kLbMask) | kLbIncl);
+    S.gofs[tid] = gstart + excl - dstart;
   }
-  lb[(size_t)tile * kBins + tid] = ((excl + cnt) & kLbMask) | kLbIncl;
-  s_gofs[tid] = gstart + excl - dstart;
+
+  /* 4. rank and drop into the tile buffer */
+#pragma unroll
+  for (int i = 0; i < kSortItems; ++i) {
+    const uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
+    atomicOr(&S.match[warp][d], lanebit);
+    __syncwarp();
+    const uint32_t grp = S.match[warp][d];
+    const uint32_t below = grp & (lanebit - 1);
+    const uint32_t first = S.slot[warp][d];            /* same word for the whole group */
+    __syncwarp();
+    if (below == 0) {                                  /* lowest lane of the group */
+      S.slot[warp][d] = first + __popc(grp);
+      S.match[warp][d] = 0;
+    }
+    S.keys[first + __popc(below)] = key[i];
+    __syncwarp();
+  }
   __syncthreads();
-  if (s_abort) {
+  if (S.abort) {
     if (tid == 0) set_status(hdr, PARD_ETIMEOUT);
     return;
   }
 
-#pragma unroll
-  for (int i = 0; i < kSortItems; ++i) {
-    uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
-    s_keys[s_dstart[d] + s_whist[warp][d] + rank[i]] = key[i];
-  }
-  __syncthreads();
+  /* 5. write out */
   const uint32_t nvalid = (uint32_t)min((uint64_t)kSortTile, (uint64_t)n - base);
+#pragma unroll 4
   for (uint32_t pos = tid; pos < nvalid; pos += kSortThreads) {
-    unsigned long long k = s_keys[pos];
-    uint32_t d = (uint32_t)(k >> shift) & 255u;
-    dst[s_gofs[d] + pos] = k;
+    const unsigned long long k = S.keys[pos];
+    const uint32_t d = (uint32_t)(k >> shift) & 255u;
+    dst[S.gofs[d] + pos] = k;
   }
 }
 
@@ -969,6 +1003,20 @@ cudaEvent_t* profile_acquire() {
   return g_prof.ev.data() + (size_t)(g_prof.n_samples++) * kEventsPerSample;
 }
 
+/* the sort pass needs more dynamic shared memory than the default limit: opt in once per device */
+int allow_sort_smem(int dev) {
+  static std::mutex mu;
+  static bool done[64];
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev < 0 || dev >= 64) return PARD_ERANGE;
+  if (!done[dev]) {
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(SortSmem)));
+    done[dev] = true;
+  }
+  return PARD_OK;
+}
+
 int check_state(const pard_queue_state_t* st, uint32_t n_ctx) {
   if (!st) return PARD_EINVAL;
   if (st->stage_stride < 1) return PARD_EINVAL;
@@ -1063,6 +1111,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
 
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  rc = allow_sort_smem(dev);
+  if (rc != PARD_OK) return rc;
   const uint4* req4 = (const uint4*)d_requests;
 
   mark();
@@ -1086,7 +1136,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
     if (n > 0 && p < L.max_passes)
-      k_sort_pass<<<L.sort_tiles, kSortThreads, 0, stream>>>(
+      k_sort_pass<<<L.sort_tiles, kSortThreads, sizeof(SortSmem), stream>>>(
           p, hdr, buf_a, buf_b, hist, lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words,
           n32, ibits);
   }

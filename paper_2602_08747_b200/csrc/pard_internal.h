@@ -45,8 +45,12 @@ struct __align__(16) PardSegConst {
   uint64_t d_magic;  /* floor(2^64 / d) + 1, or 0 when d == 1 or d >= 2^32              */
   uint64_t cap_magic;/* floor(2^64 / cap) + 1, or 0 when cap == 1                       */
   uint32_t cap;      /* min(B_k * m_k, 2^30)                                            */
-  uint32_t pad;
+  uint32_t narrow;   /* 1: 2 <= d < 2^31 and |A_rel| < 2^29, the 32-bit fields below apply */
+  int32_t a_rel32;   /* A_rel                                                           */
+  uint32_t d32;      /* d                                                               */
+  uint32_t pad[2];
 };
+static_assert(sizeof(PardSegConst) == 64, "one 64-byte line per segment");
 
 #define PARD_CUDA_OK(expr)                    \
   do {                                        \

@@ -278,7 +278,8 @@ k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
   if (seg >= n_ctx * S) return;                          /* whole warps leave together */
   const uint32_t c = seg / S, k = seg % S;
   PardSegConst out;
-  out.A = 0; out.A_rel = 0; out.d = 1; out.cap = 1; out.pad = 0; out.d_magic = 0; out.cap_magic = 0;
+  out.A = 0; out.A_rel = 0; out.d = 1; out.cap = 1; out.d_magic = 0; out.cap_magic = 0;
+  out.narrow = 0; out.a_rel32 = 0; out.d32 = 1; out.pad[0] = out.pad[1] = 0;
   int32_t pi = st.d_pipeline_of_ctx ? st.d_pipeline_of_ctx[c] : 0;
   bool bad = false;
   if (pi < 0 || (uint32_t)pi >= n_pipelines) {
@@ -325,6 +326,10 @@ k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
         out.A_rel = out.A - (int64_t)(~ctx_dmin_inv[c]);
         out.d_magic = (d >= 2 && d < ((int64_t)1 << 32)) ? magic64((uint64_t)d) : 0;
         out.cap_magic = out.cap >= 2 ? magic64(out.cap) : 0;
+        const int64_t lim = (int64_t)1 << 29;
+        out.narrow = (out.d_magic != 0 && d < ((int64_t)1 << 31) && out.A_rel > -lim && out.A_rel < lim) ? 1u : 0u;
+        out.a_rel32 = (int32_t)out.A_rel;
+        out.d32 = (uint32_t)d;
       }
     }
   }
@@ -622,6 +627,7 @@ struct TileCtx {
   const uint32_t* seg_off;
   uint32_t n, ibits, imask, kshift;
   unsigned long long dmask;
+  bool narrow;               /* deadline offsets have at most 29 bits */
 };
 
 template <bool RAW>
@@ -647,6 +653,26 @@ __device__ __forceinline__ void tile_first_half(const TileCtx& T, uint64_t base,
   uint32_t cur_seg = seg_first;
   lheadbits = 0;
   run = seg_identity<RAW>();
+  if (one_seg && T.narrow && K.narrow) {
+    /* one queue, and every quantity fits 32 bits: the common case */
+    const uint32_t r0 = (uint32_t)base - sstart;
+#pragma unroll
+    for (int i = 0; i < kDecItems; ++i) {
+      const uint32_t lo = (uint32_t)e[i], hi = (uint32_t)(e[i] >> 32);
+      idx[i] = lo & T.imask;
+      const uint32_t off = __funnelshift_r(lo, hi, T.ibits) & (uint32_t)T.dmask;
+      const int32_t X = (int32_t)off - K.a_rel32;
+      const unsigned long long uu = (unsigned long long)(div_magic32((uint32_t)X, K.d_magic) + 1u) * K.cap;
+      u[i] = X < 0 ? 0u : (uu > kUClamp ? kUClamp : (uint32_t)uu);
+      r[i] = r0 + i;
+      if (r[i] == 0) { run = seg_identity<RAW>(); run.head = 1; }
+      lv[i] = run.m;
+      lheadbits |= run.head << i;
+      if (RAW) run.m += r[i] < u[i] ? 1 : 0;
+      else run.m = min(run.m, (int32_t)u[i] - (int32_t)r[i]);
+    }
+    return;
+  }
 #pragma unroll
   for (int i = 0; i < kDecItems; ++i) {
     const uint64_t j = base + i;
@@ -687,6 +713,7 @@ __device__ __forceinline__ TileCtx make_tile_ctx(const PlanHeader* hdr, const un
   T.imask = (1u << ibits) - 1;                                 /* ibits <= 30 */
   T.kshift = ibits + dbits;                                    /* < 64 */
   T.dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  T.narrow = dbits <= 29;
   return T;
 }
 
@@ -858,6 +885,28 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
     K = ktab[seg_first];
     sstart = seg_off[seg_first];
   }
+  const bool fast = one_seg && T.narrow && K.narrow;
+  if (fast) {
+#pragma unroll
+    for (int i = 0; i < kDecItems; ++i) {
+      const bool local = (lheadbits >> i) & 1u;
+      const int32_t pre = local ? lv[i] : (RAW ? lv[i] + exc.m : min(lv[i], exc.m));
+      uint32_t c, ahead;
+      if (RAW) {
+        c = r[i];
+        ahead = r[i] == 0 ? 0u : (uint32_t)pre;
+      } else {
+        c = r[i] == 0 ? 0u : (uint32_t)min((int32_t)r[i] - 1 + pre, (int32_t)r[i]);   /* both below 2^31 */
+        ahead = c;
+      }
+      const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;
+      est[i] = K.A + (long long)((unsigned long long)round * K.d32);
+      const uint32_t kept = c < u[i] ? 1u : 0u;
+      keepbits |= kept << i;
+      if (kept && kept_tmp) kept_tmp[sstart + ahead] = idx[i];
+      if ((uint32_t)(base + i) + 1 == send) seg_kept[cur_seg] = ahead + kept;
+    }
+  } else
 #pragma unroll
   for (int i = 0; i < kDecItems; ++i) {
     const bool valid = base + i < n;
@@ -897,10 +946,10 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
 
   if (full) {
     if (out_keep) {
-      unsigned long long kb = 0;
-#pragma unroll
-      for (int i = 0; i < kDecItems; ++i) kb |= (unsigned long long)((keepbits >> i) & 1u) << (8 * i);
-      *reinterpret_cast<unsigned long long*>(out_keep + base) = kb;
+      /* bit k of a nibble -> byte k of a word */
+      const uint32_t klo = ((keepbits & 15u) * 0x00204081u) & 0x01010101u;
+      const uint32_t khi = (((keepbits >> 4) & 15u) * 0x00204081u) & 0x01010101u;
+      *reinterpret_cast<uint2*>(out_keep + base) = make_uint2(klo, khi);
     }
     if (out_est) {
       store4(out_est + base, est[0], est[1], est[2], est[3]);

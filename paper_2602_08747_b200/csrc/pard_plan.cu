@@ -33,7 +33,6 @@ constexpr int kDecItems = 8;
 constexpr int kDecTile = kDecThreads * kDecItems;
 constexpr int kCompactChunk = 4096;                /* indices moved by one block of k_kept_move */
 constexpr int kLookBatch = 16;                     /* earlier tiles inspected per round trip in the sort */
-constexpr int kSmemSegs = 4096;                    /* segment histogram kept in shared memory up to here */
 
 /* look-back word of the sort: [31:30] state, [29:0] count */
 constexpr uint32_t kLbAgg = 1u << 30;
@@ -109,86 +108,71 @@ __device__ __forceinline__ void set_status(PlanHeader* hdr, int status) {
 /* ------------------------------------------------------------------------ */
 /* prepass: one coalesced 16-byte read per request                           */
 /* ------------------------------------------------------------------------ */
-template <bool SMEM_HIST>
+/* Range checks and the smallest / largest deadline of every ctx.  A thread
+ * follows the ctx of the requests it reads and only touches global memory
+ * when that ctx changes; requests of one ctx normally sit together, so this
+ * is rare.  (ctx_dmin_inv holds the complement of the minimum, so that both
+ * arrays start from zero and grow by atomicMax.) */
 __global__ void __launch_bounds__(256)
-k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S, uint32_t n_seg,
+k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
           unsigned long long* __restrict__ ctx_dmin_inv, unsigned long long* __restrict__ ctx_dmax,
-          uint32_t* __restrict__ seg_count, PlanHeader* hdr) {
-  __shared__ uint32_t s_hist[SMEM_HIST ? kSmemSegs : 1];
-  const uint32_t lane = threadIdx.x & 31;
-  if (SMEM_HIST) {
-    for (uint32_t s = threadIdx.x; s < n_seg; s += blockDim.x) s_hist[s] = 0;
-    __syncthreads();
-  }
+          PlanHeader* hdr) {
   constexpr uint32_t kNone = 0xffffffffu;
-  uint32_t run_ctx = kNone;                 /* warp-uniform */
+  const uint32_t lane = threadIdx.x & 31;
+  uint32_t run_ctx = kNone;
   unsigned long long lmin = ~0ull, lmax = 0;
   bool bad_seen = false;
-
   auto flush = [&]() {
-    if (run_ctx == kNone) return;
-    for (int o = 16; o; o >>= 1) {
-      unsigned long long a = __shfl_xor_sync(0xffffffffu, lmin, o);
-      unsigned long long b = __shfl_xor_sync(0xffffffffu, lmax, o);
-      lmin = a < lmin ? a : lmin;
-      lmax = b > lmax ? b : lmax;
-    }
-    if (lane == 0 && lmin <= lmax) {
+    if (run_ctx != kNone) {
       atomicMax(&ctx_dmin_inv[run_ctx], ~lmin);
       atomicMax(&ctx_dmax[run_ctx], lmax);
     }
-    lmin = ~0ull;
-    lmax = 0;
   };
-
   const uint64_t chunk = (uint64_t)blockDim.x * 8;
   for (uint64_t base = (uint64_t)blockIdx.x * chunk; base < n; base += (uint64_t)gridDim.x * chunk) {
-#pragma unroll 4
+    uint4 r[8];
+    uint32_t have = 0;
+#pragma unroll
     for (int i = 0; i < 8; ++i) {
-      uint64_t j = base + (uint64_t)i * blockDim.x + threadIdx.x;
-      bool ok = j < n;
-      uint4 r = make_uint4(0, 0, 0, 0);
-      if (ok) r = __ldg(&req[j]);
-      long long D = (long long)(((unsigned long long)r.y << 32) | r.x);
-      uint32_t ctx = r.z, stage = r.w & 0xffffu;
-      if (ok && (D < 0 || D >= PARD_TIME_LIMIT_US || ctx >= n_ctx || stage >= S)) {
-        bad_seen = true;
-        ok = false;
-      }
-      uint32_t seg = ok ? ctx * S + stage : 0;
-      {                                       /* one atomic per distinct segment in the warp */
-        uint32_t grp = __match_any_sync(0xffffffffu, ok ? seg : 0xffffffffu);
-        if (ok && lane == (uint32_t)(__ffs(grp) - 1)) {
-          if (SMEM_HIST) atomicAdd(&s_hist[seg], (uint32_t)__popc(grp));
-          else atomicAdd(&seg_count[seg], (uint32_t)__popc(grp));
-        }
-      }
-      uint32_t vmask = __ballot_sync(0xffffffffu, ok);
-      if (vmask == 0) continue;
-      uint32_t c0 = __shfl_sync(0xffffffffu, ctx, __ffs(vmask) - 1);
-      bool uniform = __all_sync(0xffffffffu, !ok || ctx == c0);
-      if (uniform) {
-        if (run_ctx != c0) {
-          flush();
-          run_ctx = c0;
-        }
-        if (ok) {
-          lmin = (unsigned long long)D < lmin ? (unsigned long long)D : lmin;
-          lmax = (unsigned long long)D > lmax ? (unsigned long long)D : lmax;
-        }
-      } else if (ok) {
-        atomicMax(&ctx_dmin_inv[ctx], ~(unsigned long long)D);
-        atomicMax(&ctx_dmax[ctx], (unsigned long long)D);
+      const uint64_t j = base + (uint64_t)i * blockDim.x + threadIdx.x;
+      if (j < n) {
+        r[i] = __ldg(&req[j]);
+        have |= 1u << i;
       }
     }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (!((have >> i) & 1u)) continue;
+      const unsigned long long D = ((unsigned long long)r[i].y << 32) | r[i].x;
+      const uint32_t ctx = r[i].z, stage = r[i].w & 0xffffu;
+      if (D >= (unsigned long long)PARD_TIME_LIMIT_US || ctx >= n_ctx || stage >= S) {
+        bad_seen = true;
+        continue;
+      }
+      if (ctx != run_ctx) {
+        flush();
+        run_ctx = ctx;
+        lmin = ~0ull;
+        lmax = 0;
+      }
+      lmin = D < lmin ? D : lmin;
+      lmax = D > lmax ? D : lmax;
+    }
   }
-  flush();
+  /* one atomic pair per warp when the whole warp ended in the same ctx */
+  const uint32_t c0 = __shfl_sync(0xffffffffu, run_ctx, 0);
+  if (__all_sync(0xffffffffu, run_ctx == c0)) {
+    for (int o = 16; o; o >>= 1) {
+      const unsigned long long a = __shfl_xor_sync(0xffffffffu, lmin, o);
+      const unsigned long long b = __shfl_xor_sync(0xffffffffu, lmax, o);
+      lmin = a < lmin ? a : lmin;
+      lmax = b > lmax ? b : lmax;
+    }
+    if (lane == 0) flush();
+  } else {
+    flush();
+  }
   if (bad_seen) set_status(hdr, PARD_EDATA);
-  if (SMEM_HIST) {
-    __syncthreads();
-    for (uint32_t s = threadIdx.x; s < n_seg; s += blockDim.x)
-      if (s_hist[s]) atomicAdd(&seg_count[s], s_hist[s]);
-  }
 }
 
 __global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin_inv,
@@ -204,55 +188,48 @@ __global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin_inv,
   if ((threadIdx.x & 31) == 0 && span) atomicMax(&hdr->span_max, span);
 }
 
-/* Exclusive scan of the queue lengths by one block; also fixes the key width. */
-__global__ void __launch_bounds__(1024)
-k_seg_scan(uint32_t* __restrict__ seg_off /* in: counts, out: offsets, [n_seg+1] */,
-           uint32_t n_seg, uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ out_seg_kept,
-           uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
-  __shared__ uint32_t s_warp[32];
-  __shared__ uint32_t s_carry;
-  if (threadIdx.x == 0) {
-    s_carry = 0;
-    uint32_t dbits = bit_width64(hdr->span_max);
-    hdr->dbits = dbits;
-    hdr->keybits = sbits + dbits;
-    hdr->npass = (sbits + dbits + 7) / 8;
-    if (sbits + dbits + ibits > 64) {
-      hdr->npass = 0;
-      hdr->wide = 1;
-      set_status(hdr, PARD_ERANGE);
+/* Width of the sort key, once the widest deadline span is known. */
+__global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
+  const uint32_t dbits = bit_width64(hdr->span_max);
+  hdr->dbits = dbits;
+  hdr->keybits = sbits + dbits;
+  hdr->npass = (sbits + dbits + 7) / 8;
+  if (sbits + dbits + ibits > 64) {
+    hdr->npass = 0;
+    hdr->wide = 1;
+    set_status(hdr, PARD_ERANGE);
+  }
+}
+
+/* First position of every segment in the sorted elements: one warp per
+ * segment searches for the segment id in the elements' upper bits, probing 32
+ * positions per step. */
+__global__ void __launch_bounds__(256)
+k_seg_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+             const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t n_seg,
+             uint32_t* __restrict__ seg_off, uint32_t* __restrict__ out_seg_off) {
+  const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t lane = threadIdx.x & 31;
+  if (s > n_seg) return;                         /* whole warps leave together */
+  uint32_t lo = 0;
+  if (!hdr->wide && n > 0) {
+    const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
+    const uint32_t kshift = ibits + hdr->dbits;
+    uint32_t hi = n;                             /* answer: first element whose segment id is >= s */
+    while (lo < hi) {
+      const uint32_t span = hi - lo;
+      const uint32_t p = lo + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);   /* lo <= p < hi, non-decreasing in lane */
+      const bool less = (uint32_t)(__ldg(src + p) >> kshift) < s;
+      const uint32_t k = __popc(__ballot_sync(0xffffffffu, less));   /* lanes 0..k-1 saw a smaller id */
+      const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
+      const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
+      if (k > 0) lo = p_below + 1;
+      if (k < 32) hi = p_at;
     }
   }
-  __syncthreads();
-  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t base = 0; base < n_seg + 1; base += 1024) {
-    uint32_t i = base + threadIdx.x;
-    uint32_t v = (i < n_seg) ? seg_off[i] : 0;
-    uint32_t x = v;
-    for (int o = 1; o < 32; o <<= 1) {
-      uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= (uint32_t)o) x += y;
-    }
-    if (lane == 31) s_warp[warp] = x;
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t w = s_warp[lane], t = w;
-      for (int o = 1; o < 32; o <<= 1) {
-        uint32_t y = __shfl_up_sync(0xffffffffu, t, o);
-        if (lane >= (uint32_t)o) t += y;
-      }
-      s_warp[lane] = t - w;
-    }
-    __syncthreads();
-    uint32_t excl = s_carry + s_warp[warp] + x - v;
-    if (i <= n_seg) {
-      seg_off[i] = excl;
-      if (out_seg_off) out_seg_off[i] = excl;
-      if (out_seg_kept && i < n_seg) out_seg_kept[i] = 0;
-    }
-    __syncthreads();
-    if (threadIdx.x == 1023) s_carry = excl + v;
-    __syncthreads();
+  if (lane == 0) {
+    seg_off[s] = lo;
+    if (out_seg_off) out_seg_off[s] = lo;
   }
 }
 
@@ -269,8 +246,7 @@ __device__ __forceinline__ unsigned long long magic64(unsigned long long d) {
 __global__ void __launch_bounds__(128)
 k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
             pard_queue_state_t st, uint32_t n_ctx,
-            const unsigned long long* __restrict__ ctx_dmin_inv,
-            const uint32_t* __restrict__ seg_off, PardSegConst* __restrict__ ktab,
+            const unsigned long long* __restrict__ ctx_dmin_inv, PardSegConst* __restrict__ ktab,
             PlanHeader* hdr) {
   const uint32_t S = (uint32_t)st.stage_stride;
   const uint32_t lane = threadIdx.x & 31;
@@ -289,7 +265,7 @@ k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
     const int64_t* qrow = st.d_q_us + (size_t)c * S;
     const int32_t* brow = st.d_batch + (size_t)c * S;
     if (k >= (uint32_t)p->n_stages) {
-      if (seg_off[seg + 1] != seg_off[seg]) bad = true;   /* requests queued at a stage that does not exist */
+      out.narrow = 2;            /* no such stage: a request found in this queue is an input error */
     } else {
       int32_t B = brow[k];
       int64_t m = st.d_workers ? st.d_workers[(size_t)c * S + k] : 1;
@@ -628,6 +604,7 @@ struct TileCtx {
   uint32_t n, ibits, imask, kshift;
   unsigned long long dmask;
   bool narrow;               /* deadline offsets have at most 29 bits */
+  PlanHeader* hdr;
 };
 
 template <bool RAW>
@@ -653,7 +630,8 @@ __device__ __forceinline__ void tile_first_half(const TileCtx& T, uint64_t base,
   uint32_t cur_seg = seg_first;
   lheadbits = 0;
   run = seg_identity<RAW>();
-  if (one_seg && T.narrow && K.narrow) {
+  if ((K.narrow & 2u) && base < T.n) set_status(T.hdr, PARD_EDATA);   /* queue of a stage the pipeline lacks */
+  if (one_seg && T.narrow && K.narrow == 1) {
     /* one queue, and every quantity fits 32 bits: the common case */
     const uint32_t r0 = (uint32_t)base - sstart;
 #pragma unroll
@@ -685,6 +663,7 @@ __device__ __forceinline__ void tile_first_half(const TileCtx& T, uint64_t base,
           cur_seg = sg;
           K = T.ktab[sg];
           sstart = T.seg_off[sg];
+          if (K.narrow & 2u) set_status(T.hdr, PARD_EDATA);
         }
       }
       r[i] = (uint32_t)j - sstart;
@@ -714,6 +693,7 @@ __device__ __forceinline__ TileCtx make_tile_ctx(const PlanHeader* hdr, const un
   T.kshift = ibits + dbits;                                    /* < 64 */
   T.dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
   T.narrow = dbits <= 29;
+  T.hdr = const_cast<PlanHeader*>(hdr);
   return T;
 }
 
@@ -834,7 +814,7 @@ k_tile_scan(const unsigned long long* __restrict__ tile_agg, uint32_t n_tiles, i
  * a kept request's index goes to kept_tmp[first position of its queue + k_r]:
  * every queue's survivors end up contiguous, k_kept_move packs the queues. */
 template <bool RAW>
-__global__ void __launch_bounds__(kDecThreads)
+__global__ void __launch_bounds__(kDecThreads, 3)
 k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
          const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
          const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
@@ -885,7 +865,7 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
     K = ktab[seg_first];
     sstart = seg_off[seg_first];
   }
-  const bool fast = one_seg && T.narrow && K.narrow;
+  const bool fast = one_seg && T.narrow && K.narrow == 1;
   if (fast) {
 #pragma unroll
     for (int i = 0; i < kDecItems; ++i) {
@@ -1167,16 +1147,12 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 2047) / 2048, (uint64_t)sms * 8);
-    if (L.n_seg <= (uint32_t)kSmemSegs)
-      k_prepass<true><<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, L.n_seg, ctx_dmin, ctx_dmax, seg_off, hdr);
-    else
-      k_prepass<false><<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, L.n_seg, ctx_dmin, ctx_dmax, seg_off, hdr);
+    k_prepass<<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, hdr);
   }
   mark();
   if (n > 0) k_ctx_span<<<(n_ctx + 255) / 256, 256, 0, stream>>>(ctx_dmin, ctx_dmax, n_ctx, hdr);
-  k_seg_scan<<<1, 1024, 0, stream>>>(seg_off, L.n_seg, out->d_seg_offsets, out->d_seg_kept, sbits, ibits, hdr);
-  k_seg_const<<<(L.n_seg + 3) / 4, 128, 0, stream>>>(d_pipes, n_pipelines, *state, n_ctx, ctx_dmin,
-                                                         seg_off, ktab, hdr);
+  k_key_width<<<1, 1, 0, stream>>>(sbits, ibits, hdr);
+  k_seg_const<<<(L.n_seg + 3) / 4, 128, 0, stream>>>(d_pipes, n_pipelines, *state, n_ctx, ctx_dmin, ktab, hdr);
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
@@ -1190,6 +1166,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
           n32, ibits);
   }
   mark();
+  k_seg_bounds<<<(L.n_seg + 1 + 7) / 8, 256, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, L.n_seg, seg_off,
+                                                             out->d_seg_offsets);
   if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
     if (mode & PARD_MODE_RAW) {
@@ -1233,9 +1211,9 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* seg_scan, seg_const, kept_scan always; prepass, ctx_span, pack, passes, decide and
+  /* key_width, seg_const, seg_bounds, kept_scan always; prepass, ctx_span, pack, passes, decide and
    * tile_agg, tile_scan and kept_move (when the compacted indices are requested) when n > 0 */
-  *launches = n > 0 ? 3 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 4 : 3;
+  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 4 : 4;
   return PARD_OK;
 }
 

@@ -19,64 +19,93 @@ __global__ void k_goodput_init(const uint32_t* __restrict__ seg_off, uint32_t n_
   out_kept[c] = 0;
 }
 
-/* Each thread sums 16 keep flags read as one vector; sums of one ctx are
- * combined in the warp, then in the block, before one atomic per (block, ctx). */
+/* last ctx whose start is <= o (empty ctxs share a start; the last one owns the byte) */
+__device__ __forceinline__ uint32_t ctx_of(const uint32_t* __restrict__ seg_off, uint32_t n_ctx, uint32_t S,
+                                           uint64_t o) {
+  uint32_t lo = 0, hi = n_ctx;                   /* start(lo) <= o; start(hi) > o or hi == n_ctx */
+  while (hi - lo > 1) {
+    const uint32_t mid = lo + (hi - lo) / 2;
+    if (ctx_start(seg_off, mid, S) <= o) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+/* A block counts the keep flags of kChunk consecutive requests, read as
+ * 16-byte vectors.  If the chunk lies inside one ctx (the usual case) the
+ * block reduces its count and issues one atomic; otherwise every thread finds
+ * the ctx of its own 16 flags and counts per ctx. */
+constexpr uint32_t kVecs = 4;                                  /* vectors per thread */
+constexpr uint32_t kChunk = kThreads * kVecs * 16;             /* flags per block    */
+
 __global__ void __launch_bounds__(kThreads)
 k_goodput_count(const uint8_t* __restrict__ keep, const uint32_t* __restrict__ seg_off, uint32_t n,
                 uint32_t n_ctx, uint32_t S, unsigned long long* __restrict__ out_kept) {
   constexpr int WARPS = kThreads / 32;
-  __shared__ uint32_t s_ctx[WARPS];
   __shared__ uint32_t s_sum[WARPS];
+  __shared__ uint32_t s_ctx0, s_end0;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint64_t o = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) * 16;
-  constexpr uint32_t kNone = 0xffffffffu;
-  uint32_t my_ctx = kNone, my_sum = 0;
-  if (o < n) {
-    /* last ctx whose start is <= o (empty ctxs share a start; the last one owns the byte) */
-    uint32_t lo = 0, hi = n_ctx;               /* invariant: start(lo) <= o, start(hi) > o or hi == n_ctx */
-    while (hi - lo > 1) {
-      uint32_t mid = lo + (hi - lo) / 2;
-      if (ctx_start(seg_off, mid, S) <= o) lo = mid; else hi = mid;
-    }
-    uint32_t c = lo;
-    uint32_t cend = ctx_start(seg_off, c + 1, S);
-    if (o + 16 <= n && o + 16 <= cend) {
-      uint4 v = __ldg(reinterpret_cast<const uint4*>(keep + o));
-      my_ctx = c;
-      my_sum = __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
-    } else {
-      /* a ctx boundary or the end of the array inside these 16 flags */
-      uint32_t run = 0;
-      for (uint32_t b = 0; b < 16 && o + b < n; ++b) {
-        while (o + b >= cend) {
-          if (run) atomicAdd(&out_kept[c], (unsigned long long)run);
-          run = 0;
-          ++c;
-          cend = ctx_start(seg_off, c + 1, S);
-        }
-        run += keep[o + b] & 1u;
-      }
-      my_ctx = c;
-      my_sum = run;
-    }
-  }
-  /* warp: threads usually share one ctx */
-  uint32_t c0 = __shfl_sync(0xffffffffu, my_ctx, 0);
-  if (__all_sync(0xffffffffu, my_ctx == c0)) {
-    for (int k = 16; k; k >>= 1) my_sum += __shfl_xor_sync(0xffffffffu, my_sum, k);
-    if (lane == 0) { s_ctx[warp] = c0; s_sum[warp] = my_sum; }
-  } else {
-    if (my_ctx != kNone && my_sum) atomicAdd(&out_kept[my_ctx], (unsigned long long)my_sum);
-    if (lane == 0) { s_ctx[warp] = kNone; s_sum[warp] = 0; }
+  const uint64_t c0 = (uint64_t)blockIdx.x * kChunk;
+  const uint64_t c1 = c0 + kChunk < n ? c0 + kChunk : n;
+  if (threadIdx.x == 0) {
+    const uint32_t c = ctx_of(seg_off, n_ctx, S, c0);
+    s_ctx0 = c;
+    s_end0 = ctx_start(seg_off, c + 1, S);
   }
   __syncthreads();
-  if (warp == 0) {
-    uint32_t c = lane < WARPS ? s_ctx[lane] : kNone;
-    uint32_t s = lane < WARPS ? s_sum[lane] : 0;
-    uint32_t grp = __match_any_sync(0xffffffffu, c);
-    uint32_t tot = 0;
-    for (uint32_t m = grp; m; m &= m - 1) tot += __shfl_sync(grp, s, __ffs(m) - 1);
-    if (c != kNone && tot && lane == (uint32_t)(__ffs(grp) - 1)) atomicAdd(&out_kept[c], (unsigned long long)tot);
+  if (s_end0 >= c1) {
+    /* one ctx: plain block reduction */
+    uint32_t sum = 0;
+#pragma unroll
+    for (uint32_t k = 0; k < kVecs; ++k) {
+      const uint64_t o = c0 + ((uint64_t)k * kThreads + threadIdx.x) * 16;
+      if (o + 16 <= c1) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(keep + o));
+        sum += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+      } else {
+        for (uint64_t b = o; b < c1; ++b) sum += keep[b] & 1u;
+      }
+    }
+    for (int k = 16; k; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+    if (lane == 0) s_sum[warp] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t tot = 0;
+      for (int w = 0; w < WARPS; ++w) tot += s_sum[w];
+      if (tot) atomicAdd(&out_kept[s_ctx0], (unsigned long long)tot);
+    }
+    return;
+  }
+  /* ctx boundaries inside the chunk */
+  constexpr uint32_t kNone = 0xffffffffu;
+  for (uint32_t k = 0; k < kVecs; ++k) {
+    const uint64_t o = c0 + ((uint64_t)k * kThreads + threadIdx.x) * 16;
+    uint32_t c = kNone, run = 0;
+    if (o < c1) {
+      c = ctx_of(seg_off, n_ctx, S, o);
+      uint32_t cend = ctx_start(seg_off, c + 1, S);
+      if (o + 16 <= c1 && o + 16 <= cend) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(keep + o));
+        run = __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+      } else {
+        for (uint32_t b = 0; b < 16 && o + b < c1; ++b) {
+          while (o + b >= cend) {
+            if (run) atomicAdd(&out_kept[c], (unsigned long long)run);
+            run = 0;
+            ++c;
+            cend = ctx_start(seg_off, c + 1, S);
+          }
+          run += keep[o + b] & 1u;
+        }
+      }
+    }
+    /* a warp whose 32 vectors end in one ctx adds once */
+    const uint32_t w0 = __shfl_sync(0xffffffffu, c, 0);
+    if (__all_sync(0xffffffffu, c == w0)) {
+      for (int q = 16; q; q >>= 1) run += __shfl_xor_sync(0xffffffffu, run, q);
+      if (lane == 0 && w0 != kNone && run) atomicAdd(&out_kept[w0], (unsigned long long)run);
+    } else if (c != kNone && run) {
+      atomicAdd(&out_kept[c], (unsigned long long)run);
+    }
   }
 }
 
@@ -94,7 +123,7 @@ extern "C" int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets
   k_goodput_init<<<(n_ctx + 255) / 256, 256, 0, stream>>>(d_seg_offsets, n_ctx, (uint32_t)stage_stride,
                                                           (long long*)d_out_total, (long long*)d_out_kept);
   if (n > 0) {
-    uint32_t blocks = (uint32_t)((n + (uint64_t)kThreads * 16 - 1) / ((uint64_t)kThreads * 16));
+    uint32_t blocks = (uint32_t)((n + kChunk - 1) / kChunk);
     k_goodput_count<<<blocks, kThreads, 0, stream>>>(d_keep, d_seg_offsets, (uint32_t)n, n_ctx,
                                                      (uint32_t)stage_stride,
                                                      (unsigned long long*)d_out_kept);

@@ -210,6 +210,23 @@ def test_host_buffer_entry_point_matches():
     assert np.array_equal(out.seg_kept, want["seg_kept"])
 
 
+def test_sharded_plans_concatenate_to_the_whole_job():
+    """Sharding by ctx (the multi-GPU path) needs no exchange: the shards'
+    outputs, planned one after the other on this GPU, concatenate to the oracle's
+    plan of the whole job."""
+    from paper_2602_08747_b200 import sharding
+    wl = inputs.make("C4b", n_epochs=12, per_epoch=3000)
+    whole = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
+    parts = []
+    for rank in range(3):
+        rc, got = run_library(sharding.shard_workload(wl, 3, rank))
+        assert rc == 0
+        parts.append(got)
+    for key in ("keep", "est_us", "ctx_total", "ctx_kept", "seg_kept"):
+        assert np.array_equal(np.concatenate([p[key] for p in parts]), whole[key]), key
+    assert sum(p["n_kept"] for p in parts) == whole["n_kept"]
+
+
 # full sizes, in the launch configuration the benchmark times
 @pytest.mark.parametrize("name", ["C2", "C3", "C3b", "C4", "C5"])
 def test_configs_full_size(name):

@@ -153,6 +153,10 @@ typedef struct pard_plan_out {
 #define PARD_MODE_NOWAIT   2u   /* pard_plan returns once its work is enqueued and
                                    reads no status back; the status word stays in the
                                    workspace until pard_plan_status fetches it        */
+#define PARD_MODE_SCAN     4u   /* take the decision by the scan kernels even when the
+                                   batch-window tables would do (same results; the scan
+                                   is otherwise the fallback for queues with thousands
+                                   of batch windows)                                  */
 
 /* Device scratch pard_plan needs for n requests in n_ctx contexts. */
 int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,

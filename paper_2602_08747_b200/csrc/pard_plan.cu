@@ -47,15 +47,16 @@ struct PlanHeader {
   unsigned long long span_max;
   uint32_t ticket[kMaxPasses + 1];
   uint32_t wide;              /* 1: segment, deadline and index bits exceed 64; nothing is sorted */
-  uint32_t pad[64 - 7 - (kMaxPasses + 1)];
+  uint32_t use_scan;          /* 1: too many batch windows for the window tables: decide by scanning */
+  uint32_t pad[64 - 8 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
   uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, hist, lookback, zero_end,
-      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, kept_tmp, buf_a, buf_b, total;
-  uint32_t n_seg, sort_tiles, dec_tiles, max_passes;
+      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, wtab, kept_tmp, buf_a, buf_b, total;
+  uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
 };
 
 __host__ __device__ inline uint32_t bit_width64(unsigned long long x) {
@@ -94,6 +95,9 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.chunk_base = o; o = al(o + 4ull * (L.n_seg + 1));
   L.tile_agg = o;  o = al(o + 8ull * L.dec_tiles);
   L.tile_carry = o; o = al(o + 4ull * L.dec_tiles);
+  L.win_capacity = (uint32_t)(n / 32 + 4ull * L.n_seg + 1024);
+  L.win_off = o;   o = al(o + 4ull * (L.n_seg + 1));
+  L.wtab = o;      o = al(o + 16ull * L.win_capacity);
   L.kept_tmp = o;  o = al(o + 4ull * n);
   L.buf_a = o;     o = al(o + 8ull * n);
   L.buf_b = o;     o = al(o + 8ull * n);
@@ -723,10 +727,12 @@ k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restr
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide) return;
+  if (hdr->wide || !hdr->use_scan) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
-  const uint64_t base = (uint64_t)blockIdx.x * kDecTile + (uint64_t)tid * kDecItems;
+  const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
+  for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+  const uint64_t base = (uint64_t)tile * kDecTile + (uint64_t)tid * kDecItems;
   unsigned long long e[kDecItems];
   uint32_t idx[kDecItems], u[kDecItems], r[kDecItems], lheadbits, sstart, seg_first;
   int32_t lv[kDecItems];
@@ -744,7 +750,9 @@ k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restr
       SegVal a; a.m = s_wm[w]; a.head = s_wh[w];
       agg = seg_combine<RAW>(agg, a);
     }
-    tile_agg[blockIdx.x] = pack_val(agg, 0);
+    tile_agg[tile] = pack_val(agg, 0);
+  }
+  __syncthreads();
   }
 }
 
@@ -753,8 +761,10 @@ k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restr
  * precede tile t in the queue that is open at the start of tile t. */
 template <bool RAW>
 __global__ void __launch_bounds__(1024)
-k_tile_scan(const unsigned long long* __restrict__ tile_agg, uint32_t n_tiles, int32_t* __restrict__ carry) {
+k_tile_scan(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ tile_agg,
+            uint32_t n_tiles, int32_t* __restrict__ carry) {
   constexpr int PER = 8;
+  if (hdr->wide || !hdr->use_scan) return;
   __shared__ int32_t s_wm[32];
   __shared__ uint32_t s_wh[32];
   __shared__ int32_t s_cm;
@@ -824,10 +834,11 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide) return;
+  if (hdr->wide || !hdr->use_scan) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
-  const uint32_t tile = blockIdx.x;
+  const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
+  for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
   const uint64_t base = (uint64_t)tile * kDecTile + (uint64_t)tid * kDecItems;
   const bool full = base + kDecItems <= n;
   const int32_t tile_carry = carry[tile];
@@ -927,6 +938,297 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
   if (full) {
     if (out_keep) {
       /* bit k of a nibble -> byte k of a word */
+      const uint32_t klo = ((keepbits & 15u) * 0x00204081u) & 0x01010101u;
+      const uint32_t khi = (((keepbits >> 4) & 15u) * 0x00204081u) & 0x01010101u;
+      *reinterpret_cast<uint2*>(out_keep + base) = make_uint2(klo, khi);
+    }
+    if (out_est) {
+      store4(out_est + base, est[0], est[1], est[2], est[3]);
+      store4(out_est + base + 4, est[4], est[5], est[6], est[7]);
+    }
+    if (out_perm)
+      store4(out_perm + base, idx[0] | ((unsigned long long)idx[1] << 32),
+             idx[2] | ((unsigned long long)idx[3] << 32), idx[4] | ((unsigned long long)idx[5] << 32),
+             idx[6] | ((unsigned long long)idx[7] << 32));
+  } else {
+#pragma unroll
+    for (int i = 0; i < kDecItems; ++i)
+      if (base + i < n) {
+        if (out_keep) out_keep[base + i] = (keepbits >> i) & 1u;
+        if (out_est) out_est[base + i] = est[i];
+        if (out_perm) out_perm[base + i] = idx[i];
+      }
+  }
+  __syncthreads();
+  }
+}
+
+/* ------------------------------------------------------------------------ */
+/* window tables: the decision pass without a scan                           */
+/* ------------------------------------------------------------------------ */
+/* Inside one queue the threshold u is a step function of the deadline: every
+ * request whose deadline falls into the same batch window
+ *     b = floor((D - A) / d)
+ * has u = cap * (b + 1) (requests with D < A have u = 0).  The running minimum
+ * of u_t - t that fixes the admitted position therefore only changes at the
+ * window boundaries: with P[b] = number of requests of the queue whose window
+ * is below b, the minimum over a complete window b is u(b) - (P[b+1] - 1), and
+ *     E[b] = minimum over all complete runs before window b
+ * is a prefix minimum over at most a few thousand windows per queue.  A request
+ * at queue position r in window b then has
+ *     min_{t<r}(u_t - t) = min(E[b], u(b) - (r - 1) if r > P[b])
+ * with no reference to any other request.  P comes from a search in the sorted
+ * elements (one warp per window), E and the raw-mode kept counts Kp from a
+ * per-queue prefix pass over the windows.  Queues with more than kWinMaxPerSeg
+ * windows, or more windows in total than the table holds, make the call fall
+ * back to the scan kernels (same results). */
+struct __align__(16) WinEntry {
+  uint32_t P;      /* requests of the queue in earlier windows (or expired)       */
+  int32_t E;       /* min of u_t - t over those requests, kWinInf if there is none */
+  uint32_t Kp;     /* raw mode: kept requests among them                          */
+  uint32_t pad;
+};
+constexpr int32_t kWinInf = 0x7fffffff;
+constexpr uint32_t kWinMaxPerSeg = 4096;
+
+
+/* u of window b (the saturation of threshold_u) */
+__device__ __forceinline__ uint32_t win_u(uint32_t b, uint32_t cap) {
+  const unsigned long long u = (unsigned long long)(b + 1) * cap;
+  return u > kUClamp ? kUClamp : (uint32_t)u;
+}
+
+/* window of a non-negative X = D - A */
+__device__ __forceinline__ unsigned long long win_of(unsigned long long X, const PardSegConst& K) {
+  if ((X >> 32) == 0 && K.d_magic) return div_magic32((uint32_t)X, K.d_magic);
+  return X / (unsigned long long)K.d;
+}
+
+/* Number of table entries of every queue: windows 0..b_last of its requests, plus the end marker. */
+__global__ void __launch_bounds__(256)
+k_win_count(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
+            const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
+            const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+            uint32_t* __restrict__ win_cnt) {
+  const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= n_seg) return;
+  uint32_t w = 0;
+  const uint32_t b0 = seg_off[s], b1 = seg_off[s + 1];
+  if (b1 > b0 && !hdr->wide) {
+    const PardSegConst K = ktab[s];
+    if (K.narrow & 2u) {
+      set_status(hdr, PARD_EDATA);               /* requests queued at a stage the pipeline lacks */
+    } else {
+      const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
+      const uint32_t dbits = hdr->dbits;
+      const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+      const long long X = (long long)((src[b1 - 1] >> ibits) & dmask) - K.A_rel;   /* latest deadline of the queue */
+      unsigned long long nb = X < 0 ? 0 : win_of((unsigned long long)X, K) + 1;
+      if (nb >= kWinMaxPerSeg) { nb = 0; hdr->use_scan = 1; }
+      w = (uint32_t)nb + 1;
+    }
+  }
+  win_cnt[s] = w;
+}
+
+/* Exclusive scan of the entry counts by one block; falls back to the scan kernels when the table is too small. */
+__global__ void __launch_bounds__(1024)
+k_win_scan(PlanHeader* hdr, uint32_t* __restrict__ win_off /* in: counts, out: offsets, [n_seg+1] */,
+           uint32_t n_seg, uint32_t capacity, uint32_t force_scan) {
+  __shared__ uint32_t s_warp[32];
+  __shared__ uint32_t s_carry;
+  if (threadIdx.x == 0) s_carry = 0;
+  __syncthreads();
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (uint32_t base = 0; base < n_seg + 1; base += 1024) {
+    const uint32_t i = base + threadIdx.x;
+    const uint32_t v = i < n_seg ? win_off[i] : 0;
+    uint32_t x = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= (uint32_t)o) x += y;
+    }
+    if (lane == 31) s_warp[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t w = s_warp[lane];
+      uint32_t t = w;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, t, o);
+        if (lane >= (uint32_t)o) t += y;
+      }
+      s_warp[lane] = t - w;
+    }
+    __syncthreads();
+    const uint32_t excl = s_carry + s_warp[warp] + x - v;
+    if (i <= n_seg) win_off[i] = excl;
+    __syncthreads();
+    if (threadIdx.x == 1023) s_carry = excl + v;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0 && (s_carry > capacity || force_scan)) hdr->use_scan = 1;
+}
+
+/* P of every table entry: one warp per entry searches the queue's sorted elements, 32 probes per step. */
+__global__ void __launch_bounds__(256)
+k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+             const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
+             const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+             const uint32_t* __restrict__ win_off, WinEntry* __restrict__ wtab) {
+  if (hdr->use_scan || hdr->wide) return;
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t total = win_off[n_seg], step = (gridDim.x * blockDim.x) >> 5;
+  for (uint32_t e = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; e < total; e += step) {   /* whole warps stay together */
+  uint32_t slo = 0, shi = n_seg;                 /* last queue whose first entry is <= e */
+  while (shi - slo > 1) {
+    const uint32_t mid = slo + (shi - slo) / 2;
+    if (win_off[mid] <= e) slo = mid; else shi = mid;
+  }
+  const uint32_t s = slo, b = e - win_off[s];
+  const PardSegConst K = ktab[s];
+  const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
+  const uint32_t dbits = hdr->dbits;
+  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  const long long thr = K.A_rel + (long long)b * K.d;     /* window >= b  <=>  deadline offset >= thr */
+  uint32_t lo = seg_off[s], hi = seg_off[s + 1];
+  const uint32_t first = lo;
+  while (lo < hi) {
+    const uint32_t span = hi - lo;
+    const uint32_t p = lo + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);
+    const bool less = (long long)((__ldg(src + p) >> ibits) & dmask) < thr;
+    const uint32_t k = __popc(__ballot_sync(0xffffffffu, less));
+    const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
+    const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
+    if (k > 0) lo = p_below + 1;
+    if (k < 32) hi = p_at;
+  }
+  if (lane == 0) wtab[e].P = lo - first;
+  }
+}
+
+/* E and Kp of every table entry: one warp per queue runs over its windows, 32 at a time. */
+__global__ void __launch_bounds__(256)
+k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
+             const uint32_t* __restrict__ win_off, WinEntry* __restrict__ wtab) {
+  if (hdr->use_scan || hdr->wide) return;
+  const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t lane = threadIdx.x & 31;
+  if (s >= n_seg) return;
+  const uint32_t w0 = win_off[s], cnt = win_off[s + 1] - w0;
+  if (cnt == 0) return;
+  const uint32_t cap = ktab[s].cap;
+  WinEntry* tab = wtab + w0;
+  const uint32_t P0 = tab[0].P;
+  int32_t e_carry = P0 > 0 ? -(int32_t)(P0 - 1) : kWinInf;     /* the expired run: u = 0 */
+  uint32_t k_carry = 0;
+  if (lane == 0) { tab[0].E = e_carry; tab[0].Kp = 0; }
+  for (uint32_t b0 = 0; b0 + 1 < cnt; b0 += 32) {              /* windows b0..b0+31 -> entries b0+1.. */
+    const uint32_t b = b0 + lane;
+    int32_t val = kWinInf;
+    uint32_t kept = 0;
+    if (b + 1 < cnt) {
+      const uint32_t p = tab[b].P, q = tab[b + 1].P;
+      if (q > p) {
+        const uint32_t u = win_u(b, cap);
+        val = (int32_t)u - (int32_t)(q - 1);
+        const uint32_t top = u < q ? u : q;
+        kept = top > p ? top - p : 0;
+      }
+    }
+    for (int o = 1; o < 32; o <<= 1) {
+      const int32_t v2 = __shfl_up_sync(0xffffffffu, val, o);
+      const uint32_t k2 = __shfl_up_sync(0xffffffffu, kept, o);
+      if (lane >= (uint32_t)o) { val = min(val, v2); kept += k2; }
+    }
+    const int32_t e_inc = min(e_carry, val);
+    const uint32_t k_inc = k_carry + kept;
+    if (b + 1 < cnt) { tab[b + 1].E = e_inc; tab[b + 1].Kp = k_inc; }
+    e_carry = __shfl_sync(0xffffffffu, e_inc, 31);
+    k_carry = __shfl_sync(0xffffffffu, k_inc, 31);
+  }
+}
+
+/* Decision pass from the window tables: every request on its own. */
+template <bool RAW>
+__global__ void __launch_bounds__(kDecThreads, 3)
+k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+             const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
+             const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+             const uint32_t* __restrict__ win_off, const WinEntry* __restrict__ wtab,
+             uint8_t* __restrict__ out_keep, long long* __restrict__ out_est,
+             uint32_t* __restrict__ out_perm, uint32_t* __restrict__ kept_tmp,
+             uint32_t* __restrict__ seg_kept) {
+  if (hdr->use_scan || hdr->wide) return;
+  const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
+  const uint64_t base = ((uint64_t)blockIdx.x * kDecThreads + threadIdx.x) * kDecItems;
+  if (base >= n) return;
+  const bool full = base + kDecItems <= n;
+  unsigned long long e[kDecItems];
+  if (full) {
+    load4(T.src + base, e);
+    load4(T.src + base + 4, e + 4);
+  } else {
+#pragma unroll
+    for (int i = 0; i < kDecItems; ++i) e[i] = base + i < n ? T.src[base + i] : 0;
+  }
+  uint32_t cur_seg = (uint32_t)(e[0] >> T.kshift);
+  PardSegConst K = ktab[cur_seg];
+  uint32_t sstart = seg_off[cur_seg], send = seg_off[cur_seg + 1], woff = win_off[cur_seg];
+  const bool narrow = T.narrow && K.narrow == 1 && full && cur_seg == (uint32_t)(e[kDecItems - 1] >> T.kshift);
+
+  uint32_t keepbits = 0, idx[kDecItems];
+  long long est[kDecItems];
+#pragma unroll
+  for (int i = 0; i < kDecItems; ++i) {
+    const uint64_t j = base + i;
+    const bool valid = j < n;
+    uint32_t c = 0, ahead = 0, kept = 0;
+    idx[i] = (uint32_t)e[i] & T.imask;
+    if (valid) {
+      long long X;
+      if (narrow) {
+        X = (int32_t)(__funnelshift_r((uint32_t)e[i], (uint32_t)(e[i] >> 32), T.ibits) & (uint32_t)T.dmask) - K.a_rel32;
+      } else {
+        const uint32_t sg = (uint32_t)(e[i] >> T.kshift);
+        if (sg != cur_seg) {
+          cur_seg = sg;
+          K = ktab[sg];
+          sstart = seg_off[sg];
+          send = seg_off[sg + 1];
+          woff = win_off[sg];
+        }
+        X = (long long)((e[i] >> T.ibits) & T.dmask) - K.A_rel;
+      }
+      const uint32_t r = (uint32_t)j - sstart;
+      uint32_t u = 0;
+      if (X >= 0) {                                   /* window b of the request and its table entry */
+        const uint32_t b = (uint32_t)win_of((unsigned long long)X, K);
+        u = win_u(b, K.cap);
+        const WinEntry w = wtab[woff + b];
+        if (RAW) {
+          const uint32_t top = r < u ? r : u;
+          ahead = w.Kp + (top > w.P ? top - w.P : 0);
+          c = r;
+        } else {
+          /* min over t < r of (u_t - t); values above 1 cannot lower the position */
+          int32_t m = w.E;
+          if (r > w.P) m = min(m, (int32_t)u - (int32_t)(r - 1));
+          c = r == 0 ? 0u : r - 1 + (uint32_t)min(m, 1);
+          ahead = c;
+        }
+      } else {                                        /* deadline before even position 0 completes */
+        c = RAW ? r : 0u;
+      }
+      kept = c < u ? 1u : 0u;
+      const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;
+      est[i] = K.A + (long long)((unsigned long long)round * (unsigned long long)K.d);
+      if (kept && kept_tmp) kept_tmp[sstart + ahead] = idx[i];
+      if ((uint32_t)j + 1 == send) seg_kept[cur_seg] = ahead + kept;   /* the last request knows the queue's count */
+    }
+    keepbits |= kept << i;
+  }
+  if (full) {
+    if (out_keep) {
       const uint32_t klo = ((keepbits & 15u) * 0x00204081u) & 0x01010101u;
       const uint32_t khi = (((keepbits >> 4) & 15u) * 0x00204081u) & 0x01010101u;
       *reinterpret_cast<uint2*>(out_keep + base) = make_uint2(klo, khi);
@@ -1077,7 +1379,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   /* ---- host-side checks, nothing launched before they pass ---- */
   if (!pipelines || n_pipelines < 1 || !out) return PARD_EINVAL;
   if (n_pipelines > kMaxPipelinesPerCall) return PARD_ERANGE;
-  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT)) return PARD_EINVAL;
+  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN)) return PARD_EINVAL;
   int rc = check_state(state, n_ctx);
   if (rc != PARD_OK) return rc;
   if (n >= PARD_MAX_REQUESTS) return PARD_ERANGE;
@@ -1120,6 +1422,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   uint32_t* kept_base = (uint32_t*)(ws + L.kept_base);
   uint32_t* chunk_base = (uint32_t*)(ws + L.chunk_base);
   uint32_t* kept_tmp = (uint32_t*)(ws + L.kept_tmp);
+  uint32_t* win_off = (uint32_t*)(ws + L.win_off);
+  WinEntry* wtab = (WinEntry*)(ws + L.wtab);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -1170,18 +1474,34 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
                                                              out->d_seg_offsets);
   if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
-    if (mode & PARD_MODE_RAW) {
-      k_tile_agg<true><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
-      k_tile_scan<true><<<1, 1024, 0, stream>>>(tile_agg, L.dec_tiles, tile_carry);
-      k_decide<true><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
-                                                              out->d_keep, (long long*)out->d_est_us, out->d_perm,
-                                                              tmp, seg_kept);
+    long long* est = (long long*)out->d_est_us;
+    const bool raw = mode & PARD_MODE_RAW;
+    /* window tables, and the decision from them */
+    k_win_count<<<(L.n_seg + 255) / 256, 256, 0, stream>>>(hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off);
+    k_win_scan<<<1, 1024, 0, stream>>>(hdr, win_off, L.n_seg, L.win_capacity, (mode & PARD_MODE_SCAN) ? 1u : 0u);
+    k_win_bounds<<<std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream>>>(
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, wtab);
+    k_win_prefix<<<(L.n_seg + 7) / 8, 256, 0, stream>>>(hdr, L.n_seg, ktab, win_off, wtab);
+    const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
+    if (raw)
+      k_decide_win<true><<<win_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
+                                                               wtab, out->d_keep, est, out->d_perm, tmp, seg_kept);
+    else
+      k_decide_win<false><<<win_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
+                                                                wtab, out->d_keep, est, out->d_perm, tmp, seg_kept);
+    /* fallback when a queue has too many batch windows: the same decision by scanning
+     * (these three return at once otherwise) */
+    const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 6);
+    if (raw) {
+      k_tile_agg<true><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
+      k_tile_scan<true><<<1, 1024, 0, stream>>>(hdr, tile_agg, L.dec_tiles, tile_carry);
+      k_decide<true><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+                                                            out->d_keep, est, out->d_perm, tmp, seg_kept);
     } else {
-      k_tile_agg<false><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
-      k_tile_scan<false><<<1, 1024, 0, stream>>>(tile_agg, L.dec_tiles, tile_carry);
-      k_decide<false><<<L.dec_tiles, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
-                                                               out->d_keep, (long long*)out->d_est_us, out->d_perm,
-                                                               tmp, seg_kept);
+      k_tile_agg<false><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
+      k_tile_scan<false><<<1, 1024, 0, stream>>>(hdr, tile_agg, L.dec_tiles, tile_carry);
+      k_decide<false><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+                                                             out->d_keep, est, out->d_perm, tmp, seg_kept);
     }
   }
   k_kept_scan<<<1, 1024, 0, stream>>>(seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
@@ -1212,8 +1532,9 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
   /* key_width, seg_const, seg_bounds, kept_scan always; prepass, ctx_span, pack, passes, decide and
-   * tile_agg, tile_scan and kept_move (when the compacted indices are requested) when n > 0 */
-  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 4 : 4;
+   * the four window-table kernels, decide_win, tile_agg, tile_scan and kept_move (when the
+   * compacted indices are requested) when n > 0 */
+  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 9 : 4;
   return PARD_OK;
 }
 

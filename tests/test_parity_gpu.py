@@ -13,10 +13,15 @@ pytestmark = pytest.mark.gpu
 
 
 def both(wl, mode=0):
-    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, mode)
+    """Oracle vs library, with the decision taken from the batch-window tables
+    (default) and by the scan kernels (PARD_MODE_SCAN)."""
+    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, mode & 1)
     rc, got = run_library(wl, mode)
     assert rc == 0
     assert_identical(got, want)
+    rc, got2 = run_library(wl, mode | pb.PARD_MODE_SCAN)
+    assert rc == 0
+    assert_identical(got2, want)
     return got
 
 
@@ -231,3 +236,14 @@ def test_sharded_plans_concatenate_to_the_whole_job():
 @pytest.mark.parametrize("name", ["C2", "C3", "C3b", "C4", "C5"])
 def test_configs_full_size(name):
     both(inputs.make(name))
+
+
+def test_window_count_limits():
+    """4,094 batch windows in one queue still use the window tables, 4,097 do not;
+    both sides of the limit give the oracle's plan."""
+    rng = np.random.default_rng(11)
+    for span_windows in (4094, 4097):
+        d = 10
+        dl = rng.integers(0, span_windows * d, size=50_000)
+        dl[0] = span_windows * d - 1                      # the last window is occupied
+        both(_one_stage(len(dl), dl, d=d, B=3))

@@ -26,13 +26,14 @@ constexpr uint32_t kMaxPipelinesPerCall = 65536;
 constexpr uint32_t kSpinLimit = 1u << 22;          /* polls before giving up    */
 
 constexpr int kSortThreads = 512;
-constexpr int kSortItems = 16;
-constexpr int kSortTile = kSortThreads * kSortItems;
+constexpr int kLoWarps = 8;                        /* warps 0..7 also do the look-back (one thread per digit) */
+constexpr int kItemsLo = 10, kItemsHi = 22;        /* rounds of 32 elements per warp: look-back warps / others (measured best) */
+constexpr int kSortTile = 32 * (kLoWarps * kItemsLo + (kSortThreads / 32 - kLoWarps) * kItemsHi);
 constexpr int kDecThreads = 256;
 constexpr int kDecItems = 8;
 constexpr int kDecTile = kDecThreads * kDecItems;
 constexpr int kCompactChunk = 4096;                /* indices moved by one block of k_kept_move */
-constexpr int kLookBatch = 16;                     /* earlier tiles inspected per round trip in the sort */
+constexpr int kLookBatch = 8;                      /* earlier tiles inspected per round trip in the sort */
 
 /* look-back word of the sort: [31:30] state, [29:0] count */
 constexpr uint32_t kLbAgg = 1u << 30;
@@ -353,9 +354,10 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
 /* ------------------------------------------------------------------------ */
 /* one LSD radix pass (8 bits), stable, tile prefixes by decoupled look-back */
 /* ------------------------------------------------------------------------ */
-/* Tile = kSortTile elements, warp w owns the consecutive elements
- * [w*32*kSortItems, (w+1)*32*kSortItems) and visits them 32 at a time, so the
- * tile order is (warp, round, lane).
+/* Tile = kSortTile elements; every warp owns a run of consecutive elements
+ * (kItemsLo rounds of 32 for the warps that also do the look-back, kItemsHi
+ * rounds for the others) and visits it 32 at a time, so the tile order is
+ * (warp, round, lane).
  *   1. every warp counts its digits (shared atomics, order irrelevant);
  *   2. thread d turns the counts of digit d into the first tile-local slot of
  *      every (warp, digit) and publishes the tile's count for the look-back;
@@ -389,13 +391,50 @@ struct SortSmem {
   uint32_t abort;
 };
 
+/* one warp's share of step 1: ITEMS rounds of 32 consecutive elements */
+template <int ITEMS>
+__device__ __forceinline__ void sort_load_count(unsigned long long (&key)[kItemsHi], const unsigned long long* src,
+                                                uint64_t first, uint32_t n, uint32_t shift, uint32_t* slot_row,
+                                                uint32_t lane) {
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const uint64_t j = first + i * 32 + lane;
+    key[i] = j < n ? src[j] : ~0ull;
+  }
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) atomicAdd(&slot_row[(uint32_t)(key[i] >> shift) & 255u], 1u);
+}
+
+/* one warp's share of step 4 */
+template <int ITEMS>
+__device__ __forceinline__ void sort_rank_drop(const unsigned long long (&key)[kItemsHi], uint32_t shift,
+                                               uint32_t* slot_row, uint32_t* match_row, unsigned long long* keys,
+                                               uint32_t lanebit) {
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
+    atomicOr(&match_row[d], lanebit);
+    __syncwarp();
+    const uint32_t grp = match_row[d];
+    const uint32_t below = grp & (lanebit - 1);
+    const uint32_t first = slot_row[d];                /* same word for the whole group */
+    __syncwarp();
+    if (below == 0) {                                  /* lowest lane of the group */
+      slot_row[d] = first + __popc(grp);
+      match_row[d] = 0;
+    }
+    keys[first + __popc(below)] = key[i];
+    __syncwarp();
+  }
+}
+
 __global__ void __launch_bounds__(kSortThreads, 2)
 k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf_a,
             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ hist,
             uint32_t* __restrict__ lookback, uint32_t* __restrict__ lookback_next, uint32_t n,
             uint32_t ibits) {
   constexpr int WARPS = kSortThreads / 32;
-  static_assert(kSortThreads >= kBins && kSortThreads % 32 == 0, "one thread per digit in the lower part");
+  static_assert(kLoWarps * 32 == kBins, "one look-back thread per digit");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SortSmem& S = *reinterpret_cast<SortSmem*>(smem_raw);
 
@@ -419,15 +458,15 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   const uint64_t base = (uint64_t)tile * kSortTile;
   const uint32_t shift = ibits + 8 * pass;
 
-  /* 1. load and count */
-  unsigned long long key[kSortItems];
-#pragma unroll
-  for (int i = 0; i < kSortItems; ++i) {
-    const uint64_t j = base + warp * (32 * kSortItems) + i * 32 + lane;
-    key[i] = j < n ? src[j] : ~0ull;
-  }
-#pragma unroll
-  for (int i = 0; i < kSortItems; ++i) atomicAdd(&S.slot[warp][(uint32_t)(key[i] >> shift) & 255u], 1u);
+  /* 1. load and count.  The warps that will do the look-back own fewer
+   * elements than the others, so that both groups finish at about the same
+   * time and the look-back has registers for a wide batch. */
+  unsigned long long key[kItemsHi];
+  const bool lo_warp = warp < kLoWarps;
+  const uint32_t wfirst = lo_warp ? warp * (32 * kItemsLo)
+                                  : kLoWarps * 32 * kItemsLo + (warp - kLoWarps) * (32 * kItemsHi);
+  if (lo_warp) sort_load_count<kItemsLo>(key, src, base + wfirst, n, shift, S.slot[warp], lane);
+  else sort_load_count<kItemsHi>(key, src, base + wfirst, n, shift, S.slot[warp], lane);
   __syncthreads();
 
   /* 2. thread d owns digit d */
@@ -497,22 +536,8 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   }
 
   /* 4. rank and drop into the tile buffer */
-#pragma unroll
-  for (int i = 0; i < kSortItems; ++i) {
-    const uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
-    atomicOr(&S.match[warp][d], lanebit);
-    __syncwarp();
-    const uint32_t grp = S.match[warp][d];
-    const uint32_t below = grp & (lanebit - 1);
-    const uint32_t first = S.slot[warp][d];            /* same word for the whole group */
-    __syncwarp();
-    if (below == 0) {                                  /* lowest lane of the group */
-      S.slot[warp][d] = first + __popc(grp);
-      S.match[warp][d] = 0;
-    }
-    S.keys[first + __popc(below)] = key[i];
-    __syncwarp();
-  }
+  if (lo_warp) sort_rank_drop<kItemsLo>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
+  else sort_rank_drop<kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
   __syncthreads();
   if (S.abort) {
     if (tid == 0) set_status(hdr, PARD_ETIMEOUT);

@@ -261,10 +261,10 @@ int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets,
  * elapsed milliseconds per phase into ms_sum[PARD_N_PHASES] and returns the
  * number of sampled calls.  Process-wide state: do not call begin/end while
  * another thread is inside pard_plan.  The paper has no counterpart. */
-#define PARD_N_PHASES 13
+#define PARD_N_PHASES 15
 int pard_profile_begin(uint32_t every, uint32_t max_samples);
 int pard_profile_end(float* ms_sum, uint32_t* n_samples);
-/* "clear", "prepass", "segments", "pack", "sort0".."sort7", "decide" */
+/* "clear", "prepass", "segments", "pack", "sort0".."sort7", "tables", "decide", "compact" */
 const char* pard_profile_phase_name(uint32_t phase);
 
 #ifdef __cplusplus

@@ -23,7 +23,7 @@ PARD_EWORKSPACE, PARD_ETIMEOUT, PARD_ECUDA, PARD_EDATA, PARD_ESTATIC = -5, -6, -
 PARD_STATIC_SCRATCH_BYTES = 8 << 20
 PARD_LOAD_HOST_ONLY = 1
 PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT, PARD_MODE_SCAN = 0, 1, 2, 4
-PARD_N_PHASES = 13
+PARD_N_PHASES = 15
 
 EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pipeline_n_stages",
            "pard_pipeline_n_slots", "pard_pipeline_paths", "pard_plan_workspace_bytes", "pard_plan",

@@ -49,14 +49,16 @@ struct PlanHeader {
   uint32_t ticket[kMaxPasses + 1];
   uint32_t wide;              /* 1: segment, deadline and index bits exceed 64; nothing is sorted */
   uint32_t use_scan;          /* 1: too many batch windows for the window tables: decide by scanning */
-  uint32_t pad[64 - 8 - (kMaxPasses + 1)];
+  uint32_t win_total;         /* window-table entries handed out */
+  uint32_t pad[64 - 9 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
   uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, hist, lookback, zero_end,
-      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, wtab, kept_tmp, buf_a, buf_b, total;
+      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, wtab, kept_tmp,
+      buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
 };
 
@@ -98,6 +100,8 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.tile_carry = o; o = al(o + 4ull * L.dec_tiles);
   L.win_capacity = (uint32_t)(n / 32 + 4ull * L.n_seg + 1024);
   L.win_off = o;   o = al(o + 4ull * (L.n_seg + 1));
+  L.win_cnt = o;   o = al(o + 4ull * (L.n_seg + 1));
+  L.win_own = o;   o = al(o + 4ull * L.win_capacity);
   L.wtab = o;      o = al(o + 16ull * L.win_capacity);
   L.kept_tmp = o;  o = al(o + 4ull * n);
   L.buf_a = o;     o = al(o + 8ull * n);
@@ -203,38 +207,6 @@ __global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
     hdr->npass = 0;
     hdr->wide = 1;
     set_status(hdr, PARD_ERANGE);
-  }
-}
-
-/* First position of every segment in the sorted elements: one warp per
- * segment searches for the segment id in the elements' upper bits, probing 32
- * positions per step. */
-__global__ void __launch_bounds__(256)
-k_seg_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
-             const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t n_seg,
-             uint32_t* __restrict__ seg_off, uint32_t* __restrict__ out_seg_off) {
-  const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const uint32_t lane = threadIdx.x & 31;
-  if (s > n_seg) return;                         /* whole warps leave together */
-  uint32_t lo = 0;
-  if (!hdr->wide && n > 0) {
-    const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
-    const uint32_t kshift = ibits + hdr->dbits;
-    uint32_t hi = n;                             /* answer: first element whose segment id is >= s */
-    while (lo < hi) {
-      const uint32_t span = hi - lo;
-      const uint32_t p = lo + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);   /* lo <= p < hi, non-decreasing in lane */
-      const bool less = (uint32_t)(__ldg(src + p) >> kshift) < s;
-      const uint32_t k = __popc(__ballot_sync(0xffffffffu, less));   /* lanes 0..k-1 saw a smaller id */
-      const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
-      const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
-      if (k > 0) lo = p_below + 1;
-      if (k < 32) hi = p_at;
-    }
-  }
-  if (lane == 0) {
-    seg_off[s] = lo;
-    if (out_seg_off) out_seg_off[s] = lo;
   }
 }
 
@@ -1029,69 +1001,72 @@ __device__ __forceinline__ unsigned long long win_of(unsigned long long X, const
   return X / (unsigned long long)K.d;
 }
 
-/* Number of table entries of every queue: windows 0..b_last of its requests, plus the end marker. */
+/* One warp per queue: its first and last sorted position (a 32-ary search for
+ * the segment id in the elements' upper bits), the number of its batch windows
+ * (from its latest deadline), and a range of table entries for them, taken
+ * from a shared counter; every entry is labelled with its queue.  If the
+ * table cannot hold the windows the call falls back to the scan kernels. */
 __global__ void __launch_bounds__(256)
-k_win_count(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
-            const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
-            const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-            uint32_t* __restrict__ win_cnt) {
-  const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
-  if (s >= n_seg) return;
-  uint32_t w = 0;
-  const uint32_t b0 = seg_off[s], b1 = seg_off[s + 1];
-  if (b1 > b0 && !hdr->wide) {
+k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
+          const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t n_seg,
+          const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
+          uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
+          uint32_t* __restrict__ win_own, uint32_t capacity, uint32_t force_scan) {
+  const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t lane = threadIdx.x & 31;
+  if (s > n_seg) return;                         /* whole warps leave together */
+  if (s == 0 && lane == 0 && force_scan) hdr->use_scan = 1;
+  uint32_t lo[2] = {0, 0};
+  const bool wide = hdr->wide != 0;
+  const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
+  const uint32_t dbits = hdr->dbits;
+  if (!wide && n > 0) {
+    const uint32_t kshift = ibits + dbits;
+    uint32_t hi[2] = {n, n};                     /* answers: first element whose segment id is >= s, >= s+1 */
+    while (lo[0] < hi[0] || lo[1] < hi[1]) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        if (lo[q] < hi[q]) {                     /* uniform across the warp */
+          const uint32_t span = hi[q] - lo[q];
+          const uint32_t p = lo[q] + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);   /* lo <= p < hi */
+          const bool less = (uint32_t)(__ldg(src + p) >> kshift) < s + q;
+          const uint32_t k = __popc(__ballot_sync(0xffffffffu, less));   /* lanes 0..k-1 saw a smaller id */
+          const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
+          const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
+          if (k > 0) lo[q] = p_below + 1;
+          if (k < 32) hi[q] = p_at;
+        }
+      }
+    }
+  }
+  if (lane == 0) {
+    seg_off[s] = lo[0];
+    if (out_seg_off) out_seg_off[s] = lo[0];
+  }
+  if (s == n_seg) return;
+  /* batch windows of the queue: 0..b_last of its requests, plus the end marker */
+  uint32_t w = 0, first = 0;
+  if (lane == 0 && lo[1] > lo[0] && !wide) {
     const PardSegConst K = ktab[s];
     if (K.narrow & 2u) {
       set_status(hdr, PARD_EDATA);               /* requests queued at a stage the pipeline lacks */
     } else {
-      const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
-      const uint32_t dbits = hdr->dbits;
       const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
-      const long long X = (long long)((src[b1 - 1] >> ibits) & dmask) - K.A_rel;   /* latest deadline of the queue */
-      unsigned long long nb = X < 0 ? 0 : win_of((unsigned long long)X, K) + 1;
-      if (nb >= kWinMaxPerSeg) { nb = 0; hdr->use_scan = 1; }
-      w = (uint32_t)nb + 1;
-    }
-  }
-  win_cnt[s] = w;
-}
-
-/* Exclusive scan of the entry counts by one block; falls back to the scan kernels when the table is too small. */
-__global__ void __launch_bounds__(1024)
-k_win_scan(PlanHeader* hdr, uint32_t* __restrict__ win_off /* in: counts, out: offsets, [n_seg+1] */,
-           uint32_t n_seg, uint32_t capacity, uint32_t force_scan) {
-  __shared__ uint32_t s_warp[32];
-  __shared__ uint32_t s_carry;
-  if (threadIdx.x == 0) s_carry = 0;
-  __syncthreads();
-  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t base = 0; base < n_seg + 1; base += 1024) {
-    const uint32_t i = base + threadIdx.x;
-    const uint32_t v = i < n_seg ? win_off[i] : 0;
-    uint32_t x = v;
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
-      if (lane >= (uint32_t)o) x += y;
-    }
-    if (lane == 31) s_warp[warp] = x;
-    __syncthreads();
-    if (warp == 0) {
-      const uint32_t w = s_warp[lane];
-      uint32_t t = w;
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xffffffffu, t, o);
-        if (lane >= (uint32_t)o) t += y;
+      const long long X = (long long)((src[lo[1] - 1] >> ibits) & dmask) - K.A_rel;   /* latest deadline of the queue */
+      const unsigned long long nb = X < 0 ? 0 : win_of((unsigned long long)X, K) + 1;
+      if (nb >= kWinMaxPerSeg) {
+        hdr->use_scan = 1;
+      } else {
+        w = (uint32_t)nb + 1;
+        first = atomicAdd(&hdr->win_total, w);
+        if (first + w > capacity) { hdr->use_scan = 1; w = 0; }
       }
-      s_warp[lane] = t - w;
     }
-    __syncthreads();
-    const uint32_t excl = s_carry + s_warp[warp] + x - v;
-    if (i <= n_seg) win_off[i] = excl;
-    __syncthreads();
-    if (threadIdx.x == 1023) s_carry = excl + v;
-    __syncthreads();
   }
-  if (threadIdx.x == 0 && (s_carry > capacity || force_scan)) hdr->use_scan = 1;
+  w = __shfl_sync(0xffffffffu, w, 0);
+  first = __shfl_sync(0xffffffffu, first, 0);
+  if (lane == 0) { win_off[s] = first; win_cnt[s] = w; }
+  for (uint32_t e = lane; e < w; e += 32) win_own[first + e] = s;
 }
 
 /* P of every table entry: one warp per entry searches the queue's sorted elements, 32 probes per step. */
@@ -1099,17 +1074,13 @@ __global__ void __launch_bounds__(256)
 k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
              const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-             const uint32_t* __restrict__ win_off, WinEntry* __restrict__ wtab) {
+             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_own,
+             WinEntry* __restrict__ wtab) {
   if (hdr->use_scan || hdr->wide) return;
   const uint32_t lane = threadIdx.x & 31;
-  const uint32_t total = win_off[n_seg], step = (gridDim.x * blockDim.x) >> 5;
+  const uint32_t total = hdr->win_total, step = (gridDim.x * blockDim.x) >> 5;
   for (uint32_t e = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; e < total; e += step) {   /* whole warps stay together */
-  uint32_t slo = 0, shi = n_seg;                 /* last queue whose first entry is <= e */
-  while (shi - slo > 1) {
-    const uint32_t mid = slo + (shi - slo) / 2;
-    if (win_off[mid] <= e) slo = mid; else shi = mid;
-  }
-  const uint32_t s = slo, b = e - win_off[s];
+  const uint32_t s = win_own[e], b = e - win_off[s];
   const PardSegConst K = ktab[s];
   const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
   const uint32_t dbits = hdr->dbits;
@@ -1134,12 +1105,13 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
 /* E and Kp of every table entry: one warp per queue runs over its windows, 32 at a time. */
 __global__ void __launch_bounds__(256)
 k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
-             const uint32_t* __restrict__ win_off, WinEntry* __restrict__ wtab) {
+             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
+             WinEntry* __restrict__ wtab) {
   if (hdr->use_scan || hdr->wide) return;
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
   if (s >= n_seg) return;
-  const uint32_t w0 = win_off[s], cnt = win_off[s + 1] - w0;
+  const uint32_t w0 = win_off[s], cnt = win_cnt[s];
   if (cnt == 0) return;
   const uint32_t cap = ktab[s].cap;
   WinEntry* tab = wtab + w0;
@@ -1341,7 +1313,7 @@ k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ 
 
 /* ---- optional phase timing (process-wide) ---- */
 constexpr int kEventsPerSample = PARD_N_PHASES + 1;
-static_assert(PARD_N_PHASES == 4 + kMaxPasses + 1, "phase list");
+static_assert(PARD_N_PHASES == 4 + kMaxPasses + 3, "phase list");
 struct Profiler {
   std::mutex mu;
   bool on = false;
@@ -1449,6 +1421,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   uint32_t* kept_tmp = (uint32_t*)(ws + L.kept_tmp);
   uint32_t* win_off = (uint32_t*)(ws + L.win_off);
   WinEntry* wtab = (WinEntry*)(ws + L.wtab);
+  uint32_t* win_cnt = (uint32_t*)(ws + L.win_cnt);
+  uint32_t* win_own = (uint32_t*)(ws + L.win_own);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -1495,18 +1469,18 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
           n32, ibits);
   }
   mark();
-  k_seg_bounds<<<(L.n_seg + 1 + 7) / 8, 256, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, L.n_seg, seg_off,
-                                                             out->d_seg_offsets);
+  k_seg_win<<<(L.n_seg + 1 + 7) / 8, 256, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
+                                                        out->d_seg_offsets, win_off, win_cnt, win_own, L.win_capacity,
+                                                        (mode & PARD_MODE_SCAN) ? 1u : 0u);
   if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
     long long* est = (long long*)out->d_est_us;
     const bool raw = mode & PARD_MODE_RAW;
     /* window tables, and the decision from them */
-    k_win_count<<<(L.n_seg + 255) / 256, 256, 0, stream>>>(hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off);
-    k_win_scan<<<1, 1024, 0, stream>>>(hdr, win_off, L.n_seg, L.win_capacity, (mode & PARD_MODE_SCAN) ? 1u : 0u);
     k_win_bounds<<<std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream>>>(
-        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, wtab);
-    k_win_prefix<<<(L.n_seg + 7) / 8, 256, 0, stream>>>(hdr, L.n_seg, ktab, win_off, wtab);
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_own, wtab);
+    k_win_prefix<<<(L.n_seg + 7) / 8, 256, 0, stream>>>(hdr, L.n_seg, ktab, win_off, win_cnt, wtab);
+    mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     if (raw)
       k_decide_win<true><<<win_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
@@ -1516,7 +1490,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
                                                                 wtab, out->d_keep, est, out->d_perm, tmp, seg_kept);
     /* fallback when a queue has too many batch windows: the same decision by scanning
      * (these three return at once otherwise) */
-    const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 6);
+    const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3);
     if (raw) {
       k_tile_agg<true><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
       k_tile_scan<true><<<1, 1024, 0, stream>>>(hdr, tile_agg, L.dec_tiles, tile_carry);
@@ -1529,6 +1503,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
                                                              out->d_keep, est, out->d_perm, tmp, seg_kept);
     }
   }
+  if (n == 0) mark();
+  mark();
   k_kept_scan<<<1, 1024, 0, stream>>>(seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
                                       (unsigned long long*)out->d_n_kept);
   if (n > 0 && out->d_kept_idx)
@@ -1556,10 +1532,10 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* key_width, seg_const, seg_bounds, kept_scan always; prepass, ctx_span, pack, passes, decide and
-   * the four window-table kernels, decide_win, tile_agg, tile_scan and kept_move (when the
+  /* key_width, seg_const, seg_win, kept_scan always; prepass, ctx_span, pack, passes, decide and
+   * win_bounds, win_prefix, decide_win, tile_agg, tile_scan and kept_move (when the
    * compacted indices are requested) when n > 0 */
-  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 9 : 4;
+  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 7 : 4;
   return PARD_OK;
 }
 
@@ -1606,6 +1582,6 @@ extern "C" int pard_profile_end(float* ms_sum, uint32_t* n_samples) {
 extern "C" const char* pard_profile_phase_name(uint32_t phase) {
   static const char* names[PARD_N_PHASES] = {"clear", "prepass", "segments", "pack", "sort0", "sort1",
                                               "sort2", "sort3", "sort4", "sort5", "sort6", "sort7",
-                                              "decide"};
+                                              "tables", "decide", "compact"};
   return phase < PARD_N_PHASES ? names[phase] : "";
 }

@@ -13,6 +13,7 @@ __device__ __forceinline__ uint32_t ctx_start(const uint32_t* __restrict__ seg_o
 
 __global__ void k_goodput_init(const uint32_t* __restrict__ seg_off, uint32_t n_ctx, uint32_t S,
                                long long* __restrict__ out_total, long long* __restrict__ out_kept) {
+  pdl_wait();
   uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= n_ctx) return;
   out_total[c] = (long long)seg_off[(size_t)(c + 1) * S] - (long long)seg_off[(size_t)c * S];
@@ -40,6 +41,7 @@ constexpr uint32_t kChunk = kThreads * kVecs * 16;             /* flags per bloc
 __global__ void __launch_bounds__(kThreads)
 k_goodput_count(const uint8_t* __restrict__ keep, const uint32_t* __restrict__ seg_off, uint32_t n,
                 uint32_t n_ctx, uint32_t S, unsigned long long* __restrict__ out_kept) {
+  pdl_wait();
   constexpr int WARPS = kThreads / 32;
   __shared__ uint32_t s_sum[WARPS];
   __shared__ uint32_t s_ctx0, s_end0;
@@ -120,11 +122,11 @@ extern "C" int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets
       (uint64_t)n_ctx * (uint64_t)stage_stride > PARD_MAX_SEGMENTS)
     return PARD_ERANGE;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  k_goodput_init<<<(n_ctx + 255) / 256, 256, 0, stream>>>(d_seg_offsets, n_ctx, (uint32_t)stage_stride,
+  launch_pdl(k_goodput_init, (n_ctx + 255) / 256, 256, 0, stream, d_seg_offsets, n_ctx, (uint32_t)stage_stride,
                                                           (long long*)d_out_total, (long long*)d_out_kept);
   if (n > 0) {
     uint32_t blocks = (uint32_t)((n + kChunk - 1) / kChunk);
-    k_goodput_count<<<blocks, kThreads, 0, stream>>>(d_keep, d_seg_offsets, (uint32_t)n, n_ctx,
+    launch_pdl(k_goodput_count, blocks, kThreads, 0, stream, d_keep, d_seg_offsets, (uint32_t)n, n_ctx,
                                                      (uint32_t)stage_stride,
                                                      (unsigned long long*)d_out_kept);
   }

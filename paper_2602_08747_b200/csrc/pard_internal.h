@@ -52,6 +52,31 @@ struct __align__(16) PardSegConst {
 };
 static_assert(sizeof(PardSegConst) == 64, "one 64-byte line per segment");
 
+#ifdef __CUDACC__
+/* Programmatic dependent launch: every kernel of the library is launched with
+ * the stream-serialization attribute, so that its blocks may be scheduled while
+ * the previous kernel of the stream drains, and starts with pdl_wait(), which
+ * returns once that previous kernel has completed and its writes are visible.
+ * No kernel touches memory or exits before the wait. */
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 #define PARD_CUDA_OK(expr)                    \
   do {                                        \
     cudaError_t e__ = (expr);                 \

@@ -126,6 +126,7 @@ __global__ void __launch_bounds__(256)
 k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
           unsigned long long* __restrict__ ctx_dmin_inv, unsigned long long* __restrict__ ctx_dmax,
           PlanHeader* hdr) {
+  pdl_wait();
   constexpr uint32_t kNone = 0xffffffffu;
   const uint32_t lane = threadIdx.x & 31;
   uint32_t run_ctx = kNone;
@@ -187,6 +188,7 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
 __global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin_inv,
                            const unsigned long long* __restrict__ ctx_dmax, uint32_t n_ctx,
                            PlanHeader* hdr) {
+  pdl_wait();
   uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
   unsigned long long span = 0;
   if (c < n_ctx && ~ctx_dmin_inv[c] <= ctx_dmax[c]) span = ctx_dmax[c] - ~ctx_dmin_inv[c];
@@ -199,6 +201,7 @@ __global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin_inv,
 
 /* Width of the sort key, once the widest deadline span is known. */
 __global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
+  pdl_wait();
   const uint32_t dbits = bit_width64(hdr->span_max);
   hdr->dbits = dbits;
   hdr->keybits = sbits + dbits;
@@ -225,6 +228,7 @@ k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
             pard_queue_state_t st, uint32_t n_ctx,
             const unsigned long long* __restrict__ ctx_dmin_inv, PardSegConst* __restrict__ ktab,
             PlanHeader* hdr) {
+  pdl_wait();
   const uint32_t S = (uint32_t)st.stage_stride;
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t seg = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -296,6 +300,7 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
        const unsigned long long* __restrict__ ctx_dmin_inv, uint32_t ibits,
        const PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
        uint32_t* __restrict__ hist) {
+  pdl_wait();
   __shared__ uint32_t s_hist[kMaxPasses * kBins];
   if (hdr->wide) return;
   const uint32_t npass = hdr->npass, dbits = hdr->dbits;
@@ -405,6 +410,7 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ hist,
             uint32_t* __restrict__ lookback, uint32_t* __restrict__ lookback_next, uint32_t n,
             uint32_t ibits) {
+  pdl_wait();
   constexpr int WARPS = kSortThreads / 32;
   static_assert(kLoWarps * 32 == kBins, "one look-back thread per digit");
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -721,6 +727,7 @@ k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restr
            const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
            const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
            unsigned long long* __restrict__ tile_agg) {
+  pdl_wait();
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
@@ -760,6 +767,7 @@ template <bool RAW>
 __global__ void __launch_bounds__(1024)
 k_tile_scan(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ tile_agg,
             uint32_t n_tiles, int32_t* __restrict__ carry) {
+  pdl_wait();
   constexpr int PER = 8;
   if (hdr->wide || !hdr->use_scan) return;
   __shared__ int32_t s_wm[32];
@@ -828,6 +836,7 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
          const int32_t* __restrict__ carry, uint8_t* __restrict__ out_keep,
          long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
          uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept) {
+  pdl_wait();
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
@@ -1012,6 +1021,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
           const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
           uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
           uint32_t* __restrict__ win_own, uint32_t capacity, uint32_t force_scan) {
+  pdl_wait();
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
   if (s > n_seg) return;                         /* whole warps leave together */
@@ -1076,6 +1086,7 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
              const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_own,
              WinEntry* __restrict__ wtab) {
+  pdl_wait();
   if (hdr->use_scan || hdr->wide) return;
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t total = hdr->win_total, step = (gridDim.x * blockDim.x) >> 5;
@@ -1107,6 +1118,7 @@ __global__ void __launch_bounds__(256)
 k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
              const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
              WinEntry* __restrict__ wtab) {
+  pdl_wait();
   if (hdr->use_scan || hdr->wide) return;
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1155,6 +1167,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
              uint8_t* __restrict__ out_keep, long long* __restrict__ out_est,
              uint32_t* __restrict__ out_perm, uint32_t* __restrict__ kept_tmp,
              uint32_t* __restrict__ seg_kept) {
+  pdl_wait();
   if (hdr->use_scan || hdr->wide) return;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint64_t base = ((uint64_t)blockIdx.x * kDecThreads + threadIdx.x) * kDecItems;
@@ -1255,6 +1268,7 @@ __global__ void __launch_bounds__(1024)
 k_kept_scan(const uint32_t* __restrict__ seg_kept, uint32_t n_seg, uint32_t* __restrict__ kept_base,
             uint32_t* __restrict__ chunk_base, uint32_t* __restrict__ out_seg_kept,
             unsigned long long* __restrict__ out_n_kept) {
+  pdl_wait();
   __shared__ uint32_t s_a[32], s_b[32];
   __shared__ uint32_t s_ca, s_cb;
   if (threadIdx.x == 0) { s_ca = 0; s_cb = 0; }
@@ -1296,6 +1310,7 @@ __global__ void __launch_bounds__(256)
 k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ seg_off,
             const uint32_t* __restrict__ seg_kept, const uint32_t* __restrict__ kept_base,
             const uint32_t* __restrict__ chunk_base, uint32_t n_seg, uint32_t* __restrict__ out_kept_idx) {
+  pdl_wait();
   const uint32_t job = blockIdx.x;
   if (job >= chunk_base[n_seg]) return;
   uint32_t lo = 0, hi = n_seg;                 /* last queue whose first job is <= job */
@@ -1450,26 +1465,26 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 2047) / 2048, (uint64_t)sms * 8);
-    k_prepass<<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, hdr);
+    launch_pdl(k_prepass, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, hdr);
   }
   mark();
-  if (n > 0) k_ctx_span<<<(n_ctx + 255) / 256, 256, 0, stream>>>(ctx_dmin, ctx_dmax, n_ctx, hdr);
-  k_key_width<<<1, 1, 0, stream>>>(sbits, ibits, hdr);
-  k_seg_const<<<(L.n_seg + 3) / 4, 128, 0, stream>>>(d_pipes, n_pipelines, *state, n_ctx, ctx_dmin, ktab, hdr);
+  if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
+  launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr);
+  launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, d_pipes, n_pipelines, *state, n_ctx, ctx_dmin, ktab, hdr);
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
-    k_pack<<<grid, 256, 0, stream>>>(req4, n32, n_ctx, S, ctx_dmin, ibits, hdr, buf_a, hist);
+    launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ibits, hdr, buf_a, hist);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
     if (n > 0 && p < L.max_passes)
-      k_sort_pass<<<L.sort_tiles, kSortThreads, sizeof(SortSmem), stream>>>(
+      launch_pdl(k_sort_pass, L.sort_tiles, kSortThreads, sizeof(SortSmem), stream, 
           p, hdr, buf_a, buf_b, hist, lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words,
           n32, ibits);
   }
   mark();
-  k_seg_win<<<(L.n_seg + 1 + 7) / 8, 256, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
+  launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
                                                         out->d_seg_offsets, win_off, win_cnt, win_own, L.win_capacity,
                                                         (mode & PARD_MODE_SCAN) ? 1u : 0u);
   if (n > 0) {
@@ -1477,38 +1492,38 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     long long* est = (long long*)out->d_est_us;
     const bool raw = mode & PARD_MODE_RAW;
     /* window tables, and the decision from them */
-    k_win_bounds<<<std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream>>>(
+    launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream, 
         hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_own, wtab);
-    k_win_prefix<<<(L.n_seg + 7) / 8, 256, 0, stream>>>(hdr, L.n_seg, ktab, win_off, win_cnt, wtab);
+    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, win_off, win_cnt, wtab);
     mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     if (raw)
-      k_decide_win<true><<<win_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
+      launch_pdl(k_decide_win<true>, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
                                                                wtab, out->d_keep, est, out->d_perm, tmp, seg_kept);
     else
-      k_decide_win<false><<<win_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
+      launch_pdl(k_decide_win<false>, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
                                                                 wtab, out->d_keep, est, out->d_perm, tmp, seg_kept);
     /* fallback when a queue has too many batch windows: the same decision by scanning
      * (these three return at once otherwise) */
     const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3);
     if (raw) {
-      k_tile_agg<true><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
-      k_tile_scan<true><<<1, 1024, 0, stream>>>(hdr, tile_agg, L.dec_tiles, tile_carry);
-      k_decide<true><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+      launch_pdl(k_tile_agg<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
+      launch_pdl(k_tile_scan<true>, 1, 1024, 0, stream, hdr, tile_agg, L.dec_tiles, tile_carry);
+      launch_pdl(k_decide<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
                                                             out->d_keep, est, out->d_perm, tmp, seg_kept);
     } else {
-      k_tile_agg<false><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
-      k_tile_scan<false><<<1, 1024, 0, stream>>>(hdr, tile_agg, L.dec_tiles, tile_carry);
-      k_decide<false><<<scan_grid, kDecThreads, 0, stream>>>(hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+      launch_pdl(k_tile_agg<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
+      launch_pdl(k_tile_scan<false>, 1, 1024, 0, stream, hdr, tile_agg, L.dec_tiles, tile_carry);
+      launch_pdl(k_decide<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
                                                              out->d_keep, est, out->d_perm, tmp, seg_kept);
     }
   }
   if (n == 0) mark();
   mark();
-  k_kept_scan<<<1, 1024, 0, stream>>>(seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+  launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
                                       (unsigned long long*)out->d_n_kept);
   if (n > 0 && out->d_kept_idx)
-    k_kept_move<<<(uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg, 256, 0, stream>>>(
+    launch_pdl(k_kept_move, (uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg, 256, 0, stream, 
         kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
   mark();
   PARD_CUDA_OK(cudaGetLastError());

@@ -157,6 +157,12 @@ typedef struct pard_plan_out {
                                    batch-window tables would do (same results; the scan
                                    is otherwise the fallback for queues with thousands
                                    of batch windows)                                  */
+#define PARD_MODE_TEST_STALL 8u /* testing aid for the bounded device-side waits: the
+                                   first tile of the first sort pass withholds the word
+                                   later tiles wait for, so their waits run out (after
+                                   about a third of a second) and the call returns
+                                   PARD_ETIMEOUT with unspecified outputs; the CUDA
+                                   context stays usable                               */
 
 /* Device scratch pard_plan needs for n requests in n_ctx contexts. */
 int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,

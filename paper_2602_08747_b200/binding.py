@@ -22,7 +22,7 @@ PARD_EINVAL, PARD_ECYCLE, PARD_ERANGE, PARD_ENOMEM = -1, -2, -3, -4
 PARD_EWORKSPACE, PARD_ETIMEOUT, PARD_ECUDA, PARD_EDATA, PARD_ESTATIC = -5, -6, -7, -8, -9
 PARD_STATIC_SCRATCH_BYTES = 8 << 20
 PARD_LOAD_HOST_ONLY = 1
-PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT, PARD_MODE_SCAN = 0, 1, 2, 4
+PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT, PARD_MODE_SCAN, PARD_MODE_TEST_STALL = 0, 1, 2, 4, 8
 PARD_N_PHASES = 15
 
 EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pipeline_n_stages",

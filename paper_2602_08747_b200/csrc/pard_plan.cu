@@ -23,7 +23,7 @@ constexpr int kMaxPasses = 8;
 constexpr int kBins = 256;
 constexpr uint32_t kUClamp = (1u << 30) - 1;       /* >= any request count      */
 constexpr uint32_t kMaxPipelinesPerCall = 65536;
-constexpr uint32_t kSpinLimit = 1u << 22;          /* polls before giving up    */
+constexpr uint32_t kSpinLimit = 1u << 18;          /* polling rounds (about a microsecond each) before giving up */
 
 constexpr int kSortThreads = 512;
 constexpr int kLoWarps = 8;                        /* warps 0..7 also do the look-back (one thread per digit) */
@@ -50,7 +50,8 @@ struct PlanHeader {
   uint32_t wide;              /* 1: segment, deadline and index bits exceed 64; nothing is sorted */
   uint32_t use_scan;          /* 1: too many batch windows for the window tables: decide by scanning */
   uint32_t win_total;         /* window-table entries handed out */
-  uint32_t pad[64 - 9 - (kMaxPasses + 1)];
+  uint32_t aborted;           /* 1: a bounded wait ran out; the sort is incomplete and every later kernel returns */
+  uint32_t pad[64 - 10 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
@@ -112,6 +113,14 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
 
 __device__ __forceinline__ void set_status(PlanHeader* hdr, int status) {
   atomicCAS(&hdr->status, 0u, (uint32_t)(-status));
+}
+
+/* A bounded wait ran out: the elements are only partly sorted from here on, so nothing after
+ * this may use them as indices. */
+__device__ __forceinline__ void set_aborted(PlanHeader* hdr) {
+  hdr->aborted = 1;
+  __threadfence();
+  atomicExch(&hdr->status, (uint32_t)(-PARD_ETIMEOUT));
 }
 
 /* ------------------------------------------------------------------------ */
@@ -409,14 +418,14 @@ __global__ void __launch_bounds__(kSortThreads, 2)
 k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf_a,
             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ hist,
             uint32_t* __restrict__ lookback, uint32_t* __restrict__ lookback_next, uint32_t n,
-            uint32_t ibits) {
+            uint32_t ibits, uint32_t stall) {
   pdl_wait();
   constexpr int WARPS = kSortThreads / 32;
   static_assert(kLoWarps * 32 == kBins, "one look-back thread per digit");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SortSmem& S = *reinterpret_cast<SortSmem*>(smem_raw);
 
-  if (pass >= hdr->npass) return;
+  if (pass >= hdr->npass || hdr->aborted) return;
   const unsigned long long* src = (pass & 1) ? buf_b : buf_a;
   unsigned long long* dst = (pass & 1) ? buf_a : buf_b;
   hist += pass * kBins;
@@ -465,7 +474,7 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
     }
     if (lane == 31) { S.scan[0][warp] = x; S.scan[1][warp] = g; }
     /* the tile's count is all that later tiles need from this one for now */
-    st_relaxed(lookback + (size_t)tile * kBins + tid, cnt | kLbAgg);
+    if (!(stall && tile == 0)) st_relaxed(lookback + (size_t)tile * kBins + tid, cnt | kLbAgg);
     lookback_next[(size_t)tile * kBins + tid] = 0;     /* the array of the pass after this one */
   }
   __syncthreads();
@@ -509,7 +518,7 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
         __nanosleep(40);
       }
     }
-    st_relaxed(lookback + (size_t)tile * kBins + tid, ((excl + cnt) & kLbMask) | kLbIncl);
+    if (!(stall && tile == 0)) st_relaxed(lookback + (size_t)tile * kBins + tid, ((excl + cnt) & kLbMask) | kLbIncl);
     S.gofs[tid] = gstart + excl - dstart;
   }
 
@@ -518,7 +527,7 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   else sort_rank_drop<kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
   __syncthreads();
   if (S.abort) {
-    if (tid == 0) set_status(hdr, PARD_ETIMEOUT);
+    if (tid == 0) set_aborted(hdr);
     return;
   }
 
@@ -731,7 +740,7 @@ k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restr
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide || !hdr->use_scan) return;
+  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
@@ -769,7 +778,7 @@ k_tile_scan(const PlanHeader* __restrict__ hdr, const unsigned long long* __rest
             uint32_t n_tiles, int32_t* __restrict__ carry) {
   pdl_wait();
   constexpr int PER = 8;
-  if (hdr->wide || !hdr->use_scan) return;
+  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
   __shared__ int32_t s_wm[32];
   __shared__ uint32_t s_wh[32];
   __shared__ int32_t s_cm;
@@ -840,7 +849,7 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide || !hdr->use_scan) return;
+  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
@@ -1027,7 +1036,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
   if (s > n_seg) return;                         /* whole warps leave together */
   if (s == 0 && lane == 0 && force_scan) hdr->use_scan = 1;
   uint32_t lo[2] = {0, 0};
-  const bool wide = hdr->wide != 0;
+  const bool wide = hdr->wide != 0 || hdr->aborted != 0;   /* nothing usable was sorted */
   const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
   const uint32_t dbits = hdr->dbits;
   if (!wide && n > 0) {
@@ -1087,7 +1096,7 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
              const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_own,
              WinEntry* __restrict__ wtab) {
   pdl_wait();
-  if (hdr->use_scan || hdr->wide) return;
+  if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t total = hdr->win_total, step = (gridDim.x * blockDim.x) >> 5;
   for (uint32_t e = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; e < total; e += step) {   /* whole warps stay together */
@@ -1119,7 +1128,7 @@ k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegCo
              const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
              WinEntry* __restrict__ wtab) {
   pdl_wait();
-  if (hdr->use_scan || hdr->wide) return;
+  if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
   if (s >= n_seg) return;
@@ -1168,7 +1177,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
              uint32_t* __restrict__ out_perm, uint32_t* __restrict__ kept_tmp,
              uint32_t* __restrict__ seg_kept) {
   pdl_wait();
-  if (hdr->use_scan || hdr->wide) return;
+  if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint64_t base = ((uint64_t)blockIdx.x * kDecThreads + threadIdx.x) * kDecItems;
   if (base >= n) return;
@@ -1391,7 +1400,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   /* ---- host-side checks, nothing launched before they pass ---- */
   if (!pipelines || n_pipelines < 1 || !out) return PARD_EINVAL;
   if (n_pipelines > kMaxPipelinesPerCall) return PARD_ERANGE;
-  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN)) return PARD_EINVAL;
+  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN | PARD_MODE_TEST_STALL)) return PARD_EINVAL;
   int rc = check_state(state, n_ctx);
   if (rc != PARD_OK) return rc;
   if (n >= PARD_MAX_REQUESTS) return PARD_ERANGE;
@@ -1481,7 +1490,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     if (n > 0 && p < L.max_passes)
       launch_pdl(k_sort_pass, L.sort_tiles, kSortThreads, sizeof(SortSmem), stream, 
           p, hdr, buf_a, buf_b, hist, lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words,
-          n32, ibits);
+          n32, ibits, (p == 0 && (mode & PARD_MODE_TEST_STALL)) ? 1u : 0u);
   }
   mark();
   launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,

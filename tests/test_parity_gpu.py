@@ -162,6 +162,16 @@ def test_device_detected_errors():
     both(inputs.Workload("ok", [p], good, st, 1))
 
 
+def test_bounded_wait_runs_out_and_is_reported():
+    """Failure detection without a fault: with the stall aid the tiles of the first
+    sort pass wait for a word that never comes; each wait is bounded, the call
+    returns PARD_ETIMEOUT, nothing hangs and the next call is correct."""
+    wl = inputs.make("C3", n=300_000)
+    rc, _ = run_library(wl, mode=pb.PARD_MODE_TEST_STALL, check=False)
+    assert rc == pb.PARD_ETIMEOUT
+    both(wl)
+
+
 def test_key_wider_than_64_bits_is_reported():
     # 2^59 span * 2^14 requests * 64 segments does not fit one 64-bit sort element
     p = util.pipeline(inputs.chain_edges(2), 2, [5, 6])

@@ -36,6 +36,26 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
+def ncu_traffic(kernel):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary, or None
+    when the kernel source has changed since the counters were taken."""
+    import hashlib
+    try:
+        src = os.path.join(ROOT, "paper_2602_08747_b200", "csrc", "pard_plan.cu")
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+        vals = {}
+        for line in open(os.path.join(ROOT, "profiles", "dram_traffic_C3.txt")):
+            if line.startswith("#") or not line.strip():
+                continue
+            k, v = line.split()
+            vals[k] = v
+        if vals.get("source_sha256") != sha:
+            return None
+        return int(vals[kernel]) if kernel in vals else None
+    except Exception:
+        return None
+
+
 class ClockSampler(threading.Thread):
     """Polls SM clock and throttle reasons through NVML while the timed region runs."""
 
@@ -336,7 +356,7 @@ def run_ours(args):
         kernels = kernel_table(prof, wl.n, keep_frac, peak)
         timed = {k: v for k, v in kernels.items() if k not in ("other", "k_decide_win")}
         top = max(timed, key=lambda k: timed[k]["ms_per_step"])
-        traffic = None
+        traffic = ncu_traffic(top)
         roofline = {"bound": "hbm", "kernel": top, "achieved": timed[top]["achieved_gbs"], "peak": peak,
                     "unit": "GB/s", "frac": timed[top]["frac"], "traffic": traffic,
                     "peak_kind": "of " + peak_kind,

@@ -1168,7 +1168,7 @@ k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegCo
 
 /* Decision pass from the window tables: every request on its own. */
 template <bool RAW>
-__global__ void __launch_bounds__(kDecThreads, 3)
+__global__ void __launch_bounds__(kDecThreads, 4)
 k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
              const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,

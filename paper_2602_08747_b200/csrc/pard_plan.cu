@@ -32,7 +32,7 @@ constexpr int kSortTile = 32 * (kLoWarps * kItemsLo + (kSortThreads / 32 - kLoWa
 constexpr int kDecThreads = 256;
 constexpr int kDecItems = 8;
 constexpr int kDecTile = kDecThreads * kDecItems;
-constexpr int kCompactChunk = 4096;                /* indices moved by one block of k_kept_move */
+constexpr int kCompactChunk = 1024;                /* indices moved by one warp of k_kept_move */
 constexpr int kLookBatch = 8;                      /* earlier tiles inspected per round trip in the sort */
 
 /* look-back word of the sort: [31:30] state, [29:0] count */
@@ -51,14 +51,15 @@ struct PlanHeader {
   uint32_t use_scan;          /* 1: too many batch windows for the window tables: decide by scanning */
   uint32_t win_total;         /* window-table entries handed out */
   uint32_t aborted;           /* 1: a bounded wait ran out; the sort is incomplete and every later kernel returns */
-  uint32_t pad[64 - 10 - (kMaxPasses + 1)];
+  uint32_t big_total;         /* window-table entries that belong to long queues */
+  uint32_t pad[64 - 11 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
   uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, hist, lookback, zero_end,
-      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, wtab, kept_tmp,
+      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
 };
@@ -103,6 +104,7 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.win_off = o;   o = al(o + 4ull * (L.n_seg + 1));
   L.win_cnt = o;   o = al(o + 4ull * (L.n_seg + 1));
   L.win_own = o;   o = al(o + 4ull * L.win_capacity);
+  L.win_big = o;   o = al(o + 4ull * L.win_capacity);
   L.wtab = o;      o = al(o + 16ull * L.win_capacity);
   L.kept_tmp = o;  o = al(o + 4ull * n);
   L.buf_a = o;     o = al(o + 8ull * n);
@@ -147,6 +149,24 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
       atomicMax(&ctx_dmax[run_ctx], lmax);
     }
   };
+  /* whole warp (converged): one atomic pair if all lanes follow the same ctx, else one per lane */
+  auto warp_flush = [&]() {
+    const uint32_t c0 = __shfl_sync(0xffffffffu, run_ctx, 0);
+    if (__all_sync(0xffffffffu, run_ctx == c0)) {
+      for (int o = 16; o; o >>= 1) {
+        const unsigned long long a = __shfl_xor_sync(0xffffffffu, lmin, o);
+        const unsigned long long b = __shfl_xor_sync(0xffffffffu, lmax, o);
+        lmin = a < lmin ? a : lmin;
+        lmax = b > lmax ? b : lmax;
+      }
+      if (lane == 0) flush();
+    } else {
+      flush();
+    }
+    run_ctx = kNone;
+    lmin = ~0ull;
+    lmax = 0;
+  };
   const uint64_t chunk = (uint64_t)blockDim.x * 8;
   for (uint64_t base = (uint64_t)blockIdx.x * chunk; base < n; base += (uint64_t)gridDim.x * chunk) {
     uint4 r[8];
@@ -159,6 +179,8 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
         have |= 1u << i;
       }
     }
+    /* a new chunk usually lies in another ctx than the last one: hand the old one over together */
+    if (__any_sync(0xffffffffu, (have & 1u) && run_ctx != kNone && r[0].z != run_ctx)) warp_flush();
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       if (!((have >> i) & 1u)) continue;
@@ -178,19 +200,7 @@ k_prepass(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
       lmax = D > lmax ? D : lmax;
     }
   }
-  /* one atomic pair per warp when the whole warp ended in the same ctx */
-  const uint32_t c0 = __shfl_sync(0xffffffffu, run_ctx, 0);
-  if (__all_sync(0xffffffffu, run_ctx == c0)) {
-    for (int o = 16; o; o >>= 1) {
-      const unsigned long long a = __shfl_xor_sync(0xffffffffu, lmin, o);
-      const unsigned long long b = __shfl_xor_sync(0xffffffffu, lmax, o);
-      lmin = a < lmin ? a : lmin;
-      lmax = b > lmax ? b : lmax;
-    }
-    if (lane == 0) flush();
-  } else {
-    flush();
-  }
+  warp_flush();
   if (bad_seen) set_status(hdr, PARD_EDATA);
 }
 
@@ -1005,6 +1015,7 @@ struct __align__(16) WinEntry {
 };
 constexpr int32_t kWinInf = 0x7fffffff;
 constexpr uint32_t kWinMaxPerSeg = 4096;
+constexpr uint32_t kWinLongQueue = 8192;   /* above this a window boundary is searched by a whole warp, else by one lane */
 
 
 /* u of window b (the saturation of threshold_u) */
@@ -1029,7 +1040,8 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
           const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t n_seg,
           const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
           uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
-          uint32_t* __restrict__ win_own, uint32_t capacity, uint32_t force_scan) {
+          uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
+          uint32_t force_scan) {
   pdl_wait();
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1086,6 +1098,12 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
   first = __shfl_sync(0xffffffffu, first, 0);
   if (lane == 0) { win_off[s] = first; win_cnt[s] = w; }
   for (uint32_t e = lane; e < w; e += 32) win_own[first + e] = s;
+  if (w && lo[1] - lo[0] > kWinLongQueue) {      /* long queue: list its entries for the warp-wide search */
+    uint32_t at = 0;
+    if (lane == 0) at = atomicAdd(&hdr->big_total, w);
+    at = __shfl_sync(0xffffffffu, at, 0);
+    for (uint32_t e = lane; e < w; e += 32) win_big[at + e] = first + e;
+  }
 }
 
 /* P of every table entry: one warp per entry searches the queue's sorted elements, 32 probes per step. */
@@ -1094,12 +1112,33 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
              const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
              const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_own,
-             WinEntry* __restrict__ wtab) {
+             const uint32_t* __restrict__ win_big, WinEntry* __restrict__ wtab) {
   pdl_wait();
   if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t lane = threadIdx.x & 31;
-  const uint32_t total = hdr->win_total, step = (gridDim.x * blockDim.x) >> 5;
-  for (uint32_t e = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; e < total; e += step) {   /* whole warps stay together */
+  /* entries of short queues: one lane each, plain binary search */
+  {
+    const uint32_t total = hdr->win_total, step = gridDim.x * blockDim.x;
+    const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
+    const uint32_t dbits = hdr->dbits;
+    const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+    for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += step) {
+      const uint32_t s = win_own[e];
+      uint32_t lo = seg_off[s], hi = seg_off[s + 1];
+      if (hi - lo > kWinLongQueue) continue;
+      const uint32_t first = lo;
+      const long long thr = ktab[s].A_rel + (long long)(e - win_off[s]) * ktab[s].d;
+      while (lo < hi) {
+        const uint32_t mid = lo + (hi - lo) / 2;
+        if ((long long)((__ldg(src + mid) >> ibits) & dmask) < thr) lo = mid + 1; else hi = mid;
+      }
+      wtab[e].P = lo - first;
+    }
+  }
+  /* entries of long queues: one warp each, 32 probes per step */
+  const uint32_t total = hdr->big_total, step = (gridDim.x * blockDim.x) >> 5;
+  for (uint32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < total; i += step) {   /* whole warps stay together */
+  const uint32_t e = win_big[i];
   const uint32_t s = win_own[e], b = e - win_off[s];
   const PardSegConst K = ktab[s];
   const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
@@ -1272,67 +1311,84 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
 }
 
 /* Kept requests per queue -> first output slot of every queue, the number of
- * kCompactChunk-sized copy jobs before every queue, and the total.  One block. */
+ * kCompactChunk-sized copy jobs before every queue, and the total.  One block,
+ * eight queues per thread and round. */
 __global__ void __launch_bounds__(1024)
 k_kept_scan(const uint32_t* __restrict__ seg_kept, uint32_t n_seg, uint32_t* __restrict__ kept_base,
             uint32_t* __restrict__ chunk_base, uint32_t* __restrict__ out_seg_kept,
             unsigned long long* __restrict__ out_n_kept) {
   pdl_wait();
+  constexpr int PER = 8;
   __shared__ uint32_t s_a[32], s_b[32];
   __shared__ uint32_t s_ca, s_cb;
   if (threadIdx.x == 0) { s_ca = 0; s_cb = 0; }
   __syncthreads();
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t base = 0; base < n_seg + 1; base += 1024) {
-    const uint32_t i = base + threadIdx.x;
-    const uint32_t v = i < n_seg ? seg_kept[i] : 0;
-    const uint32_t c = (v + kCompactChunk - 1) / kCompactChunk;
-    if (out_seg_kept && i < n_seg) out_seg_kept[i] = v;
-    uint32_t x = v, y = c;
+  for (uint32_t base = 0; base < n_seg + 1; base += 1024 * PER) {
+    const uint32_t i0 = base + threadIdx.x * PER;
+    uint32_t v[PER], c[PER], x = 0, y = 0;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      v[k] = i0 + k < n_seg ? seg_kept[i0 + k] : 0;
+      c[k] = (v[k] + kCompactChunk - 1) / kCompactChunk;
+      if (out_seg_kept && i0 + k < n_seg) out_seg_kept[i0 + k] = v[k];
+      x += v[k];
+      y += c[k];
+    }
+    const uint32_t tx = x, ty = y;
     for (int o = 1; o < 32; o <<= 1) {
-      uint32_t p = __shfl_up_sync(0xffffffffu, x, o), q = __shfl_up_sync(0xffffffffu, y, o);
+      const uint32_t p = __shfl_up_sync(0xffffffffu, x, o), q = __shfl_up_sync(0xffffffffu, y, o);
       if (lane >= (uint32_t)o) { x += p; y += q; }
     }
     if (lane == 31) { s_a[warp] = x; s_b[warp] = y; }
     __syncthreads();
     if (warp == 0) {
-      uint32_t a = s_a[lane], b = s_b[lane], ta = a, tb = b;
+      const uint32_t a = s_a[lane], b = s_b[lane];
+      uint32_t ta = a, tb = b;
       for (int o = 1; o < 32; o <<= 1) {
-        uint32_t p = __shfl_up_sync(0xffffffffu, ta, o), q = __shfl_up_sync(0xffffffffu, tb, o);
+        const uint32_t p = __shfl_up_sync(0xffffffffu, ta, o), q = __shfl_up_sync(0xffffffffu, tb, o);
         if (lane >= (uint32_t)o) { ta += p; tb += q; }
       }
       s_a[lane] = ta - a;
       s_b[lane] = tb - b;
     }
     __syncthreads();
-    const uint32_t ea = s_ca + s_a[warp] + x - v, eb = s_cb + s_b[warp] + y - c;
-    if (i <= n_seg) { kept_base[i] = ea; chunk_base[i] = eb; }
+    uint32_t ea = s_ca + s_a[warp] + x - tx, eb = s_cb + s_b[warp] + y - ty;   /* exclusive, before this thread's queues */
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      if (i0 + k <= n_seg) { kept_base[i0 + k] = ea; chunk_base[i0 + k] = eb; }
+      ea += v[k];
+      eb += c[k];
+    }
     __syncthreads();
-    if (threadIdx.x == 1023) { s_ca = ea + v; s_cb = eb + c; }
+    if (threadIdx.x == 1023) { s_ca = ea; s_cb = eb; }
     __syncthreads();
   }
   if (threadIdx.x == 0 && out_n_kept) *out_n_kept = s_ca;
 }
 
-/* Packs the queues' survivors: copy job b moves up to kCompactChunk indices of one queue. */
+/* Packs the queues' survivors: copy job j moves up to kCompactChunk indices of one queue; a
+ * warp per job. */
 __global__ void __launch_bounds__(256)
 k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ seg_off,
             const uint32_t* __restrict__ seg_kept, const uint32_t* __restrict__ kept_base,
             const uint32_t* __restrict__ chunk_base, uint32_t n_seg, uint32_t* __restrict__ out_kept_idx) {
   pdl_wait();
-  const uint32_t job = blockIdx.x;
-  if (job >= chunk_base[n_seg]) return;
-  uint32_t lo = 0, hi = n_seg;                 /* last queue whose first job is <= job */
-  while (hi - lo > 1) {
-    const uint32_t mid = lo + (hi - lo) / 2;
-    if (chunk_base[mid] <= job) lo = mid; else hi = mid;
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t jobs = chunk_base[n_seg], step = (gridDim.x * blockDim.x) >> 5;
+  for (uint32_t job = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; job < jobs; job += step) {
+    uint32_t lo = 0, hi = n_seg;                 /* last queue whose first job is <= job */
+    while (hi - lo > 1) {
+      const uint32_t mid = lo + (hi - lo) / 2;
+      if (chunk_base[mid] <= job) lo = mid; else hi = mid;
+    }
+    const uint32_t s = lo;
+    const uint32_t first = (job - chunk_base[s]) * kCompactChunk;
+    const uint32_t count = min((uint32_t)kCompactChunk, seg_kept[s] - first);
+    const uint32_t* src = kept_tmp + seg_off[s] + first;
+    uint32_t* dst = out_kept_idx + kept_base[s] + first;
+    for (uint32_t i = lane; i < count; i += 32) dst[i] = src[i];
   }
-  const uint32_t s = lo;
-  const uint32_t first = (job - chunk_base[s]) * kCompactChunk;
-  const uint32_t count = min((uint32_t)kCompactChunk, seg_kept[s] - first);
-  const uint32_t* src = kept_tmp + seg_off[s] + first;
-  uint32_t* dst = out_kept_idx + kept_base[s] + first;
-  for (uint32_t i = threadIdx.x; i < count; i += blockDim.x) dst[i] = src[i];
 }
 
 /* ---- optional phase timing (process-wide) ---- */
@@ -1447,6 +1503,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   WinEntry* wtab = (WinEntry*)(ws + L.wtab);
   uint32_t* win_cnt = (uint32_t*)(ws + L.win_cnt);
   uint32_t* win_own = (uint32_t*)(ws + L.win_own);
+  uint32_t* win_big = (uint32_t*)(ws + L.win_big);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -1494,7 +1551,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   }
   mark();
   launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
-                                                        out->d_seg_offsets, win_off, win_cnt, win_own, L.win_capacity,
+                                                        out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
                                                         (mode & PARD_MODE_SCAN) ? 1u : 0u);
   if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
@@ -1502,7 +1559,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     const bool raw = mode & PARD_MODE_RAW;
     /* window tables, and the decision from them */
     launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream, 
-        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_own, wtab);
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_own, win_big, wtab);
     launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, win_off, win_cnt, wtab);
     mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
@@ -1532,7 +1589,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
                                       (unsigned long long*)out->d_n_kept);
   if (n > 0 && out->d_kept_idx)
-    launch_pdl(k_kept_move, (uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg, 256, 0, stream, 
+    launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
+                                               (uint32_t)sms * 8), 256, 0, stream, 
         kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
   mark();
   PARD_CUDA_OK(cudaGetLastError());

@@ -57,6 +57,9 @@ def lib():
         _lib.oracle_plan.restype = C.c_int
         _lib.oracle_plan.argtypes = ([C.c_void_p, C.c_int32, C.c_void_p, C.c_uint64,
                                       C.c_void_p, C.c_uint32, C.c_uint32] + [C.c_void_p] * 9)
+        _lib.oracle_estimate_w.restype = C.c_int
+        _lib.oracle_estimate_w.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint32, C.c_int32, C.c_int32,
+                                           C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_void_p]
     return _lib
 
 
@@ -106,6 +109,24 @@ def lsub(p, stage: int, batch_row, q_row, w_row=None) -> int:
     cp = _c_pipeline(p, k)
     return int(lib().oracle_lsub(C.addressof(cp), stage, k.add(batch_row, np.int32),
                                  k.add(q_row, np.int64), k.add(w_row, np.int64)))
+
+
+def estimate_w(pipelines, pipeline_of_ctx, n_ctx: int, stage_stride: int, slot_stride: int, wait_samples,
+               lambda_num: int = 1, lambda_den: int = 10, seed: int = 0) -> np.ndarray:
+    """w[n_ctx, slot_stride] (int64): the batch-wait estimate of every (stage, downstream path) slot.
+    wait_samples: int32 [n_ctx, stage_stride, M]."""
+    k = _Keep()
+    cps = (_Pipeline * len(pipelines))(*[_c_pipeline(p, k) for p in pipelines])
+    ws = np.ascontiguousarray(wait_samples, dtype=np.int32)
+    assert ws.shape[0] == n_ctx and ws.shape[1] == stage_stride
+    M = int(ws.shape[2])
+    w = np.zeros((n_ctx, slot_stride), dtype=np.int64)
+    rc = lib().oracle_estimate_w(C.addressof(cps), len(pipelines), k.add(pipeline_of_ctx, np.int32), n_ctx,
+                                 stage_stride, slot_stride, ws.ctypes.data, M, lambda_num, lambda_den,
+                                 seed & (2**64 - 1), w.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle_estimate_w: bad input")
+    return w
 
 
 def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:

@@ -14,6 +14,7 @@
  *   Order:  low budget first = smallest remaining budget first  (Sec. 4.3)
  *   Rule:   drop when the estimate exceeds the latency objective (Sec. 5.3)
  *   Counts: goodput / drop rate                                 (Sec. 5.1)
+ *   w_k:    quantile lambda of the sampled aggregated batch wait  (Sec. 4.2)
  *
  * Readings where the paper is silent (each also listed in the design notes):
  *   - Snapshot: the Request Broker loop is run over the whole queue at the
@@ -107,6 +108,67 @@ extern "C" int64_t oracle_lsub(const oracle_pipeline_t* p, int32_t stage,
     first = false;
   }
   return best;
+}
+
+namespace {
+
+/* splitmix64 (Steele, Lea, Flood: "Fast splittable pseudorandom number generators") */
+uint64_t splitmix64(uint64_t x) {
+  uint64_t z = x + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+/* every downstream path of `stage` continuing through `cur`, in lexicographic order */
+void collect_paths(const oracle_pipeline_t* p, int32_t cur, std::vector<int32_t>* prefix,
+                   std::vector<std::vector<int32_t>>* out) {
+  prefix->push_back(cur);
+  std::vector<int32_t> s = successors_ascending(p, cur);
+  if (s.empty()) out->push_back(*prefix);
+  for (int32_t j : s) collect_paths(p, j, prefix, out);
+  prefix->pop_back();
+}
+
+}  // namespace
+
+extern "C" int oracle_estimate_w(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                                 const int32_t* pipeline_of_ctx, uint32_t n_ctx,
+                                 int32_t stage_stride, int32_t slot_stride,
+                                 const int32_t* wait_samples, uint32_t M,
+                                 uint32_t lambda_num, uint32_t lambda_den, uint64_t seed,
+                                 int64_t* w_us) {
+  if (M == 0 || lambda_den == 0 || lambda_num > lambda_den) return -1;
+  uint64_t rank = (uint64_t)lambda_num * M / lambda_den;        /* lambda = 0: smallest, lambda = 1: largest */
+  if (rank > M - 1) rank = M - 1;
+  for (uint32_t c = 0; c < n_ctx; ++c) {
+    int32_t pi = pipeline_of_ctx ? pipeline_of_ctx[c] : 0;
+    if (pi < 0 || pi >= n_pipelines) return -1;
+    const oracle_pipeline_t* p = &pipelines[pi];
+    int64_t slot = 0;
+    for (int32_t k = 0; k < p->n_stages; ++k) {
+      std::vector<std::vector<int32_t>> paths;
+      std::vector<int32_t> prefix;
+      for (int32_t j : successors_ascending(p, k)) collect_paths(p, j, &prefix, &paths);
+      for (const std::vector<int32_t>& path : paths) {        /* one slot per (stage, downstream path) */
+        if (slot >= slot_stride) return -1;
+        std::vector<int64_t> sums(M);
+        for (uint32_t m = 0; m < M; ++m) {
+          int64_t sum = 0;                                    /* aggregated batch wait of one sampled request */
+          for (size_t j = 0; j < path.size(); ++j) {
+            uint64_t counter = seed + ((((uint64_t)c * (uint64_t)slot_stride + (uint64_t)slot) * M + m) * 64 + j);
+            uint64_t idx = ((splitmix64(counter) >> 32) * (uint64_t)M) >> 32;
+            sum += wait_samples[((size_t)c * stage_stride + path[j]) * M + idx];
+          }
+          sums[m] = sum;
+        }
+        std::sort(sums.begin(), sums.end());
+        w_us[(size_t)c * slot_stride + slot] = sums[rank];    /* F^{-1}(lambda) */
+        ++slot;
+      }
+    }
+  }
+  return 0;
 }
 
 extern "C" int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelines,

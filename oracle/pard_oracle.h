@@ -79,6 +79,24 @@ int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
                 uint32_t* seg_offsets, uint32_t* seg_kept,
                 int64_t* ctx_total, int64_t* ctx_kept);
 
+/* Batch-wait estimate w = F^{-1}(lambda) of the State Planner (Sec. 4.2, Batch
+ * wait estimation): for every (ctx, stage k, downstream path P) slot, draw M
+ * samples of the aggregated batch wait -- one recorded batch wait of every
+ * stage on P, picked at random -- and return the sample of rank
+ * floor(lambda_num * M / lambda_den) (clamped to M - 1) in ascending order.
+ * wait_samples[(ctx * stage_stride + stage) * M + j], j < M, are the stage's
+ * recorded batch waits in microseconds.  The random pick for sample m and the
+ * j-th stage of the path is  idx = (hi32(splitmix64(counter)) * M) >> 32  with
+ * counter = seed + (((ctx * slot_stride + slot) * M + m) * 64 + j)  (splitmix64
+ * as published by Steele, Lea and Flood).  w_us[ctx * slot_stride + slot] is
+ * written for the slots of the ctx's pipeline.  Returns 0, or -1 on bad input. */
+int oracle_estimate_w(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                      const int32_t* pipeline_of_ctx, uint32_t n_ctx,
+                      int32_t stage_stride, int32_t slot_stride,
+                      const int32_t* wait_samples, uint32_t M,
+                      uint32_t lambda_num, uint32_t lambda_den, uint64_t seed,
+                      int64_t* w_us);
+
 #ifdef __cplusplus
 }
 #endif

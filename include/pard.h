@@ -34,6 +34,8 @@ extern "C" {
 #define PARD_MAX_PATH_LEN_SUM (1 << 20)/* sum of the lengths of all those paths     */
 #define PARD_MAX_REQUESTS    (1ull << 30) /* requests per pard_plan call            */
 #define PARD_MAX_SEGMENTS    (1u << 24)   /* n_ctx * stage_stride                   */
+#define PARD_MAX_WAIT_SAMPLES (1u << 15)   /* samples per slot in pard_estimate_w      */
+#define PARD_WAIT_LIMIT_US   (1 << 24)    /* recorded batch waits lie in [0, 2^24)  */
 #define PARD_TIME_LIMIT_US   (1ll << 60)  /* every time input lies in [0, 2^60)     */
 #define PARD_LAT_LIMIT_US    (1ll << 40)  /* every profile entry lies in [1, 2^40)  */
 
@@ -258,6 +260,42 @@ int pard_plan_host(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines
 int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets,
                  uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                  int64_t* d_out_total, int64_t* d_out_kept, void* cuda_stream);
+
+/* Batch-wait estimate of the State Planner (Sec. 4.2, Batch wait estimation,
+ * and Sec. 5.3 Overheads: M = 10,000 samples, refreshed off the critical path).
+ * For every ctx and every (stage k, downstream path P) slot of its pipeline,
+ *   w[ctx][slot] = F^{-1}(lambda),   lambda = lambda_num / lambda_den in [0, 1],
+ * where F is the empirical distribution of n_samples draws of the batch wait
+ * aggregated over the stages of P: draw m adds, for the j-th stage i of P, one
+ * recorded wait  d_wait_samples[(ctx * stage_stride + i) * n_samples + idx],
+ *   idx = (hi32(splitmix64(seed + (((ctx*slot_stride + slot) * n_samples + m) * 64 + j)))
+ *          * n_samples) >> 32,
+ * (splitmix64 of Steele, Lea and Flood; 64-bit wrap-around arithmetic), and
+ * F^{-1}(lambda) is the draw of rank min(n_samples - 1, floor(lambda * n_samples))
+ * in ascending order: lambda = 0 gives the smallest draw, lambda = 1 the largest.
+ * The result feeds pard_queue_state_t.d_w_us.
+ *   d_wait_samples  DEVICE, int32 [n_ctx][stage_stride][n_samples]: for every
+ *                   stage its n_samples most recent recorded batch waits in
+ *                   microseconds, each in [0, PARD_WAIT_LIMIT_US); rows of
+ *                   stages the pipeline lacks are not read
+ *   d_w_us          DEVICE, int64 [n_ctx][slot_stride]; entries at slots the
+ *                   ctx's pipeline lacks are left untouched
+ *   d_workspace     DEVICE, 256-byte aligned, pard_estimate_w_workspace_bytes()
+ *   mode            0 or PARD_MODE_NOWAIT (then pard_plan_status on this
+ *                   workspace fetches the status later)
+ * 1 <= n_samples <= PARD_MAX_WAIT_SAMPLES.  Host-detectable errors come back
+ * before anything is launched; a drawn sample outside its range, a pipeline id
+ * outside [0, n_pipelines) or a pipeline with more stages or slots than the
+ * strides gives PARD_EDATA with unspecified outputs.  One kernel is enqueued
+ * on cuda_stream; no device memory is allocated.  The caller owns all buffers. */
+int pard_estimate_w_workspace_bytes(uint32_t n_pipelines, uint64_t* bytes);
+int pard_estimate_w(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+                    const int32_t* d_pipeline_of_ctx, uint32_t n_ctx,
+                    int32_t stage_stride, int32_t slot_stride,
+                    const int32_t* d_wait_samples, uint32_t n_samples,
+                    uint32_t lambda_num, uint32_t lambda_den, uint64_t seed, uint32_t mode,
+                    int64_t* d_w_us, void* d_workspace, uint64_t workspace_bytes,
+                    void* cuda_stream);
 
 /* ---- optional device timing of the planner's phases ----------------------
  * For benchmarks.  Between pard_profile_begin and pard_profile_end every

@@ -24,12 +24,15 @@ PARD_STATIC_SCRATCH_BYTES = 8 << 20
 PARD_LOAD_HOST_ONLY = 1
 PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT, PARD_MODE_SCAN, PARD_MODE_TEST_STALL = 0, 1, 2, 4, 8
 PARD_N_PHASES = 15
+PARD_MAX_WAIT_SAMPLES = 1 << 15
+PARD_WAIT_LIMIT_US = 1 << 24
 
 EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pipeline_n_stages",
            "pard_pipeline_n_slots", "pard_pipeline_paths", "pard_plan_workspace_bytes", "pard_plan",
            "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput", "pard_plan_status",
            "pard_plan_kernel_launches", "pard_profile_begin", "pard_profile_end",
-           "pard_profile_phase_name", "pard_plan_static"]
+           "pard_profile_phase_name", "pard_plan_static", "pard_estimate_w_workspace_bytes",
+           "pard_estimate_w"]
 
 
 class PardError(RuntimeError):
@@ -88,6 +91,10 @@ def library() -> C.CDLL:
         lib.pard_plan_static.argtypes = plan_args[:8] + [C.c_void_p]
         lib.pard_plan_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.pard_plan_kernel_launches.argtypes = [C.c_uint64, C.c_uint32, C.c_int32, C.c_void_p]
+        lib.pard_estimate_w_workspace_bytes.argtypes = [C.c_uint32, C.c_void_p]
+        lib.pard_estimate_w.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_int32, C.c_int32,
+                                        C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint32,
+                                        C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
         lib.pard_profile_begin.argtypes = [C.c_uint32, C.c_uint32]
         lib.pard_profile_end.argtypes = [C.c_void_p, C.c_void_p]
         lib.pard_profile_phase_name.restype = C.c_char_p
@@ -124,7 +131,10 @@ class Pipeline:
         self._h = C.c_void_p(handle)
 
     def __del__(self):
-        self.free()
+        try:
+            self.free()
+        except Exception:          # interpreter shutdown: the module globals are already gone
+            pass
 
     def free(self):
         if getattr(self, "_h", None) is not None and self._h.value:
@@ -300,6 +310,27 @@ def pard_goodput(d_keep, d_seg_offsets, n: int, n_ctx: int, stage_stride: int, d
                                 _ptr(d_out_total), _ptr(d_out_kept), stream or None)
     if check:
         _check(rc, "pard_goodput")
+    return rc
+
+
+def pard_estimate_w_workspace_bytes(n_pipelines: int) -> int:
+    b = C.c_uint64()
+    _check(library().pard_estimate_w_workspace_bytes(n_pipelines, C.byref(b)), "pard_estimate_w_workspace_bytes")
+    return b.value
+
+
+def pard_estimate_w(pipelines: Sequence[Pipeline], d_pipeline_of_ctx, n_ctx: int, stage_stride: int,
+                    slot_stride: int, d_wait_samples, n_samples: int, lambda_num: int, lambda_den: int,
+                    seed: int, mode: int, d_w_us, d_workspace, workspace_bytes: Optional[int] = None,
+                    stream: int = 0, check: bool = True) -> int:
+    hs = _handles(pipelines)
+    wb = workspace_bytes if workspace_bytes is not None else d_workspace.numel() * d_workspace.element_size()
+    rc = library().pard_estimate_w(hs, len(pipelines), _ptr(d_pipeline_of_ctx), n_ctx, stage_stride,
+                                   slot_stride, _ptr(d_wait_samples), n_samples, lambda_num, lambda_den,
+                                   seed & (2**64 - 1), mode, _ptr(d_w_us), _ptr(d_workspace),
+                                   wb, stream or None)
+    if check:
+        _check(rc, "pard_estimate_w")
     return rc
 
 

@@ -209,6 +209,25 @@ def draw_state(rng, pipelines, pipeline_of_ctx, now_us, stage_stride=None,
                       None, poc)
 
 
+def draw_wait_samples(rng, wl: "Workload", n_samples: int = 10_000) -> np.ndarray:
+    """Recorded batch waits, int32 [n_ctx, stage_stride, n_samples] in microseconds.
+    A request that reaches stage i while a batch of duration d_i(B_i) runs waits
+    for the rest of it: a fraction of d_i(B_i) (Sec. 3.2).  The fraction is
+    Beta(a, b) distributed with a, b drawn per (ctx, stage) from [0.6, 2.5], so
+    that stages differ in how early or late in a batch their requests arrive;
+    Beta(1, 1) is the uniform arrival of the paper's worked example."""
+    st = wl.state
+    S = st.stage_stride
+    out = np.zeros((wl.n_ctx, S, n_samples), dtype=np.int32)
+    for c in range(wl.n_ctx):
+        p = wl.pipelines[int(st.pipeline_of_ctx[c]) if st.pipeline_of_ctx is not None else 0]
+        for k in range(p.n_stages):
+            d = min(p.latency(k, int(st.batch[c, k])), (1 << 24) - 1)
+            a, b = rng.uniform(0.6, 2.5, size=2)
+            out[c, k] = np.minimum((rng.beta(a, b, size=n_samples) * d).astype(np.int64), d - 1 if d > 1 else 0)
+    return out
+
+
 def balance_workers(wl: Workload, slo_us) -> None:
     """Balanced variant: m_s = ceil(n_s * d_s(B_s) / (B_s * SLO/2)) workers per
     queue, so that a queue drains in about half an SLO and a sizeable share of

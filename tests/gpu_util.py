@@ -50,3 +50,26 @@ def assert_identical(got, want):
                 bad = np.flatnonzero(g != w)
                 raise AssertionError("%s differs at %d positions, first %d: got %s want %s"
                                      % (k, bad.size, bad[0], g[bad[0]], w[bad[0]]))
+
+
+def run_estimate_w(wl, samples, lambda_num, lambda_den, seed, slot_stride=None, check=True, fill=-7):
+    """pard_estimate_w on cuda:0; returns (status, w [n_ctx, slot_stride] as numpy).
+    The output buffer is pre-filled with `fill` so that untouched entries show."""
+    import torch
+    pbuild.build()
+    dev = "cuda:0"
+    pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
+    st = wl.state
+    R = slot_stride or st.slot_stride
+    d_samples = torch.from_numpy(np.ascontiguousarray(samples, dtype=np.int32)).to(dev)
+    d_poc = None if st.pipeline_of_ctx is None else torch.from_numpy(st.pipeline_of_ctx.astype(np.int32)).to(dev)
+    d_w = torch.full((wl.n_ctx, R), fill, dtype=torch.int64, device=dev)
+    ws = pb.alloc_workspace(pb.pard_estimate_w_workspace_bytes(len(pipes)), dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    rc = pb.pard_estimate_w(pipes, d_poc, wl.n_ctx, st.stage_stride, R, d_samples, int(samples.shape[2]),
+                            lambda_num, lambda_den, seed, 0, d_w, ws, stream=stream, check=check)
+    torch.cuda.synchronize()
+    w = d_w.cpu().numpy()
+    for p in pipes:
+        p.free()
+    return rc, w

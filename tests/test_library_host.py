@@ -157,3 +157,33 @@ def test_plan_argument_checks_happen_before_any_launch():
     assert lib.pard_plan(hs, 1, None, 0, C.byref(bad), 1, 0, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
     assert lib.pard_plan(hs, 1, None, 5, C.byref(cst), 1, 0, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
     assert lib.pard_goodput(None, None, 0, 1, 2, None, None, None) == pb.PARD_EINVAL
+
+
+def test_estimate_w_argument_checks_happen_before_any_launch():
+    p = inputs.make_pipeline(inputs.chain_edges(2), 2, [1, 1], [[5], [5]])
+    h = pb.pard_load_pipeline(p, host_only=True)
+    lib = pb.library()
+    v = C.c_uint64()
+    assert lib.pard_estimate_w_workspace_bytes(0, C.byref(v)) == pb.PARD_EINVAL
+    assert lib.pard_estimate_w_workspace_bytes(1, None) == pb.PARD_EINVAL
+    assert lib.pard_estimate_w_workspace_bytes(3, C.byref(v)) == pb.PARD_OK and v.value >= 256 + 24
+    hs = (C.c_void_p * 1)(h.handle)
+    buf = np.zeros(64, np.int64)
+    a = buf.ctypes.data
+
+    def call(pipes=hs, n_pipes=1, poc=None, n_ctx=1, S=2, R=1, samples=a, M=8, num=1, den=10, mode=0, w=a):
+        return lib.pard_estimate_w(pipes, n_pipes, poc, n_ctx, S, R, samples, M, num, den, 0, mode, w, None, 0, None)
+
+    assert call(pipes=None) == pb.PARD_EINVAL
+    assert call(samples=None) == pb.PARD_EINVAL
+    assert call(w=None) == pb.PARD_EINVAL
+    assert call(n_ctx=0) == pb.PARD_EINVAL
+    assert call(num=11) == pb.PARD_EINVAL                  # lambda > 1
+    assert call(den=0) == pb.PARD_EINVAL
+    assert call(mode=pb.PARD_MODE_RAW) == pb.PARD_EINVAL
+    assert call(n_pipes=2) == pb.PARD_EINVAL               # several pipelines need the ctx map
+    assert call(S=0) == pb.PARD_EINVAL
+    assert call(M=0) == pb.PARD_ERANGE
+    assert call(M=pb.PARD_MAX_WAIT_SAMPLES + 1) == pb.PARD_ERANGE
+    assert call(S=65) == pb.PARD_ERANGE
+    assert call(n_ctx=1 << 20, R=1 << 12) == pb.PARD_ERANGE

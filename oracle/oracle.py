@@ -41,7 +41,8 @@ class _State(C.Structure):
     _fields_ = [("stage_stride", C.c_int32), ("slot_stride", C.c_int32),
                 ("pipeline_of_ctx", C.c_void_p), ("now_us", C.c_void_p),
                 ("batch", C.c_void_p), ("free_at_us", C.c_void_p),
-                ("q_us", C.c_void_p), ("w_us", C.c_void_p), ("workers", C.c_void_p)]
+                ("q_us", C.c_void_p), ("w_us", C.c_void_p), ("workers", C.c_void_p),
+                ("priority", C.c_void_p)]
 
 
 def lib():
@@ -60,6 +61,10 @@ def lib():
         _lib.oracle_estimate_w.restype = C.c_int
         _lib.oracle_estimate_w.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint32, C.c_int32, C.c_int32,
                                            C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_void_p]
+        _lib.oracle_update_priority.restype = C.c_int
+        _lib.oracle_update_priority.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint32, C.c_int32,
+                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32,
+                                                C.c_uint32, C.c_void_p]
     return _lib
 
 
@@ -129,6 +134,24 @@ def estimate_w(pipelines, pipeline_of_ctx, n_ctx: int, stage_stride: int, slot_s
     return w
 
 
+def update_priority(pipelines, pipeline_of_ctx, n_ctx: int, stage_stride: int, batch, workers, arrivals,
+                    window: int, interval_us: int, priority) -> np.ndarray:
+    """New decision order of every (ctx, stage) queue (uint8 [n_ctx, stage_stride]; 0 = low budget
+    first, 1 = high budget first) from the previous one and the arrival history
+    (uint32 [n_ctx, stage_stride, n_hist])."""
+    k = _Keep()
+    cps = (_Pipeline * len(pipelines))(*[_c_pipeline(p, k) for p in pipelines])
+    x = np.ascontiguousarray(arrivals, dtype=np.uint32)
+    assert x.shape[0] == n_ctx and x.shape[1] == stage_stride
+    out = np.array(priority, dtype=np.uint8).reshape(n_ctx, stage_stride).copy()
+    rc = lib().oracle_update_priority(C.addressof(cps), len(pipelines), k.add(pipeline_of_ctx, np.int32), n_ctx,
+                                      stage_stride, k.add(batch, np.int32), k.add(workers, np.int32),
+                                      x.ctypes.data, int(x.shape[2]), window, interval_us, out.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle_update_priority: bad input")
+    return out
+
+
 def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:
     """Runs the oracle planner; returns a dict of numpy outputs."""
     k = _Keep()
@@ -141,7 +164,8 @@ def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:
                  k.add(state.pipeline_of_ctx, np.int32), k.add(state.now_us, np.int64),
                  k.add(state.batch, np.int32), k.add(state.free_at_us, np.int64),
                  k.add(state.q_us, np.int64), k.add(state.w_us, np.int64),
-                 k.add(state.workers, np.int32))
+                 k.add(state.workers, np.int32),
+                 k.add(getattr(state, "priority", None), np.uint8))
     out = {
         "keep": np.zeros(n, np.uint8), "est_us": np.zeros(n, np.int64),
         "perm": np.zeros(n, np.uint32), "kept_idx": np.zeros(n, np.uint32),

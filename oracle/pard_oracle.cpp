@@ -11,7 +11,9 @@
  *   Eq. 3   L = (t_e - t_s + d_k) + (sum q_i + sum d_i + w_k)  (Sec. 4.2)
  *   DAG:    the estimate is taken along every subsequent path and the
  *           maximum is used                                     (Sec. 4.2, 5.1)
- *   Order:  low budget first = smallest remaining budget first  (Sec. 4.3)
+ *   Order:  low budget first = smallest remaining budget first, or high
+ *           budget first = largest first, per queue                (Sec. 4.3)
+ *   mu/eps: load factor, fluctuation bound, delayed transition     (Sec. 4.3)
  *   Rule:   drop when the estimate exceeds the latency objective (Sec. 5.3)
  *   Counts: goodput / drop rate                                 (Sec. 5.1)
  *   w_k:    quantile lambda of the sampled aggregated batch wait  (Sec. 4.2)
@@ -23,7 +25,8 @@
  *   - A dropped request never enters a batch, so the position that decides the
  *     batch index counts kept requests only (mode 0).  Mode 1 counts all.
  *   - d_k is the profile at the stage's current batch size for every batch.
- *   - est == deadline is kept; equal deadlines are served in index order.
+ *   - est == deadline is kept; equal deadlines are served in index order
+ *     (under either priority).
  *   - w covers the stages after k; one value per (stage, downstream path).
  *   - m identical workers drain one queue: a batch round starts B*m requests.
  */
@@ -219,10 +222,19 @@ extern "C" int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelin
       int64_t base = std::max(st->now_us[c], free_row[k]);   /* t_e of the next batch */
       int64_t lsub = oracle_lsub(p, k, batch_row, q_row, w_row);
 
-      /* low budget first: smallest deadline first, ties in index order */
-      std::stable_sort(qk.begin(), qk.end(), [&](uint32_t a, uint32_t b) {
-        return requests[a].deadline_us < requests[b].deadline_us;
-      });
+      /* the remaining budget of a request is its deadline minus the same `now`
+       * for the whole queue, so budget order is deadline order.
+       * low budget first: smallest deadline first; high budget first: largest
+       * deadline first; ties in index order either way */
+      bool high_first = st->priority && st->priority[(size_t)c * S + k] != 0;
+      if (high_first)
+        std::stable_sort(qk.begin(), qk.end(), [&](uint32_t a, uint32_t b) {
+          return requests[a].deadline_us > requests[b].deadline_us;
+        });
+      else
+        std::stable_sort(qk.begin(), qk.end(), [&](uint32_t a, uint32_t b) {
+          return requests[a].deadline_us < requests[b].deadline_us;
+        });
 
       int64_t kept = 0, raw = 0;
       for (uint32_t i : qk) {                    /* the Request Broker, one request at a time */
@@ -250,5 +262,58 @@ extern "C" int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelin
   }
   if (seg_offsets) seg_offsets[(size_t)n_ctx * S] = (uint32_t)pos;
   if (n_kept) *n_kept = kept_all;
+  return 0;
+}
+
+extern "C" int oracle_update_priority(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                                      const int32_t* pipeline_of_ctx, uint32_t n_ctx,
+                                      int32_t stage_stride, const int32_t* batch,
+                                      const int32_t* workers, const uint32_t* arrivals,
+                                      uint32_t n_hist, uint32_t window, uint32_t interval_us,
+                                      uint8_t* priority) {
+  typedef unsigned __int128 u128;
+  if (window < 1 || window > n_hist || interval_us < 1) return -1;
+  for (uint32_t c = 0; c < n_ctx; ++c) {
+    int32_t pi = pipeline_of_ctx ? pipeline_of_ctx[c] : 0;
+    if (pi < 0 || pi >= n_pipelines) return -1;
+    const oracle_pipeline_t* p = &pipelines[pi];
+    for (int32_t k = 0; k < p->n_stages; ++k) {
+      size_t seg = (size_t)c * stage_stride + k;
+      int32_t B = batch[seg];
+      if (B < 1 || B > p->bmax[k]) return -1;
+      int64_t m = workers ? workers[seg] : 1;
+      if (m < 1) return -1;
+      int64_t d = profile_at(p, k, B);
+      int64_t cap = (int64_t)B * m;                       /* T_m = cap / d requests per microsecond */
+      const uint32_t* x = arrivals + seg * n_hist;        /* T_in, one sample per interval */
+
+      /* eps = sum |T_in - T_s| / sum T_in with T_s[j] = (x[j-W+1] + ... + x[j]) / W.
+       * Scaled by W to stay in integers:  eps = dev / (W * sum_x). */
+      uint64_t W = window, sum_x = 0, dev = 0;
+      for (uint32_t j = window - 1; j < n_hist; ++j) {
+        uint64_t win = 0;
+        for (uint32_t i = j + 1 - window; i <= j; ++i) win += x[i];
+        uint64_t wx = W * x[j];
+        dev += wx > win ? wx - win : win - wx;            /* W * |T_in[j] - T_s[j]| */
+        sum_x += x[j];
+      }
+      if (sum_x == 0) {                                   /* nothing arrived: within capacity */
+        priority[seg] = 0;
+        continue;
+      }
+      /* mu = (x_now / interval) / (cap / d) = x_now * d / (cap * interval);
+       * mu > 1 + eps  <=>  x_now * d * (W * sum_x) > cap * interval * (W * sum_x + dev)
+       * mu < 1 - eps  <=>  x_now * d * (W * sum_x) < cap * interval * (W * sum_x - dev) */
+      uint64_t x_now = x[n_hist - 1];
+      u128 lhs = (u128)x_now * (u128)(uint64_t)d * (u128)(W * sum_x);
+      u128 scale = (u128)(uint64_t)cap * (u128)interval_us;
+      u128 upper = scale * (u128)(W * sum_x + dev);
+      if (lhs > upper) {
+        priority[seg] = 1;                                /* under-provisioned: high budget first */
+      } else if (W * sum_x > dev && lhs < scale * (u128)(W * sum_x - dev)) {
+        priority[seg] = 0;                                /* within capacity: low budget first */
+      }                                                   /* else: inside [1 - eps, 1 + eps], unchanged */
+    }
+  }
   return 0;
 }

@@ -38,7 +38,8 @@ typedef struct oracle_request {
 } oracle_request_t;
 
 /* Runtime state, row-major per ctx; rows have stage_stride / slot_stride
- * entries.  pipeline_of_ctx, w_us and workers may be NULL (=> 0, 0, 1). */
+ * entries.  pipeline_of_ctx, w_us, workers and priority may be NULL
+ * (=> 0, 0, 1, 0). */
 typedef struct oracle_state {
   int32_t        stage_stride;
   int32_t        slot_stride;
@@ -49,6 +50,8 @@ typedef struct oracle_state {
   const int64_t* q_us;
   const int64_t* w_us;
   const int32_t* workers;
+  const uint8_t* priority;      /* [n_ctx][stage_stride] decision order of each queue (Sec. 4.3):
+                                   0 = low budget first, 1 = high budget first; NULL => 0 */
 } oracle_state_t;
 
 /* Number of downstream paths of `stage` (0 for a sink). */
@@ -96,6 +99,31 @@ int oracle_estimate_w(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
                       const int32_t* wait_samples, uint32_t M,
                       uint32_t lambda_num, uint32_t lambda_den, uint64_t seed,
                       int64_t* w_us);
+
+/* Adaptive request priority with delayed transition (Sec. 4.3).  For every
+ * (ctx, stage) queue:
+ *   T_in   the input workload: arrivals[(ctx * stage_stride + stage) * n_hist + j],
+ *          j < n_hist, is the number of requests that arrived in the j-th
+ *          sampling interval of interval_us microseconds, oldest first
+ *   T_s    T_in filtered by a sliding-window average over `window` samples;
+ *          defined for j >= window - 1 (the first window - 1 samples only fill
+ *          the window)
+ *   eps  = sum |T_in - T_s| / sum T_in          both sums over j >= window - 1
+ *   T_m  = B_k * m_k / d_k(B_k)                 module throughput (requests per us)
+ *   mu   = T_in / T_m, with T_in the latest sample as a rate (per us)
+ * The new priority is 1 (high budget first) if mu > 1 + eps, 0 (low budget
+ * first) if mu < 1 - eps, and the previous one otherwise; a queue with no
+ * arrival in the summed intervals gets 0.  All comparisons are exact (integer
+ * cross-multiplication).  priority[n_ctx * stage_stride] holds the previous
+ * priorities on entry and the new ones on return; entries of stages the ctx's
+ * pipeline lacks are left untouched.  workers may be NULL (=> 1).
+ * Returns 0, or -1 on bad input. */
+int oracle_update_priority(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                           const int32_t* pipeline_of_ctx, uint32_t n_ctx,
+                           int32_t stage_stride, const int32_t* batch,
+                           const int32_t* workers, const uint32_t* arrivals,
+                           uint32_t n_hist, uint32_t window, uint32_t interval_us,
+                           uint8_t* priority);
 
 #ifdef __cplusplus
 }

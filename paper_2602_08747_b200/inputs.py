@@ -53,6 +53,7 @@ class QueueState:
     w_us: Optional[np.ndarray] = None         # int64 [n_ctx, slot_stride]
     workers: Optional[np.ndarray] = None      # int32 [n_ctx, stage_stride]
     pipeline_of_ctx: Optional[np.ndarray] = None   # int32 [n_ctx]
+    priority: Optional[np.ndarray] = None     # uint8 [n_ctx, stage_stride]; 0 low / 1 high budget first
 
 
 @dataclass

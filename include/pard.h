@@ -35,6 +35,8 @@ extern "C" {
 #define PARD_MAX_REQUESTS    (1ull << 30) /* requests per pard_plan call            */
 #define PARD_MAX_SEGMENTS    (1u << 24)   /* n_ctx * stage_stride                   */
 #define PARD_MAX_WAIT_SAMPLES (1u << 15)   /* samples per slot in pard_estimate_w      */
+#define PARD_MAX_HISTORY     4096         /* workload samples per queue in pard_update_priority */
+#define PARD_RATE_LIMIT      (1u << 24)   /* arrivals per sampling interval lie in [0, 2^24) */
 #define PARD_WAIT_LIMIT_US   (1 << 24)    /* recorded batch waits lie in [0, 2^24)  */
 #define PARD_TIME_LIMIT_US   (1ll << 60)  /* every time input lies in [0, 2^60)     */
 #define PARD_LAT_LIMIT_US    (1ll << 40)  /* every profile entry lies in [1, 2^40)  */
@@ -134,11 +136,17 @@ typedef struct pard_queue_state {
                                       (stage, downstream path) slot; NULL => 0       */
   const int32_t* d_workers;        /* [n_ctx][stage_stride] identical workers m_k >= 1
                                       draining the queue; NULL => 1                  */
+  const uint8_t* d_priority;       /* [n_ctx][stage_stride] decision order of the queue
+                                      (Sec. 4.3): 0 = low budget first, any other value =
+                                      high budget first; NULL => 0.  pard_update_priority
+                                      maintains such an array                        */
 } pard_queue_state_t;
 
 /* Outputs of pard_plan, all DEVICE memory owned by the caller.  Per-request
  * outputs are in service order: segments ascending, inside a segment by
- * (deadline, original index) ascending.  A NULL member is not produced. */
+ * (deadline, original index) ascending -- for a queue served high budget first
+ * by deadline descending, equal deadlines still in ascending index order.  A
+ * NULL member is not produced. */
 typedef struct pard_plan_out {
   uint8_t*  d_keep;        /* [n]  1 = kept, 0 = dropped                             */
   int64_t*  d_est_us;      /* [n]  estimated completion time t_s + L of Eq. 3        */
@@ -170,8 +178,10 @@ typedef struct pard_plan_out {
 int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                               uint64_t* bytes);
 
-/* The planner (Sec. 4.2 Eq. 1-3, Sec. 4.3 low-budget-first order).
- * For every segment, in ascending (deadline, index) order, with
+/* The planner (Sec. 4.2 Eq. 1-3; decision order of Sec. 4.3: the remaining
+ * budget of a request is its deadline minus the snapshot's `now`, so low
+ * budget first is deadline ascending and high budget first is deadline
+ * descending).  For every segment, in its decision order, with
  *   d    = d_k(B_k)                         profile at the current batch size
  *   cap  = B_k * m_k                        requests started per batch round
  *   base = max(now, free_at_k)              start of the next batch to form
@@ -296,6 +306,43 @@ int pard_estimate_w(const pard_pipeline_t* const* pipelines, uint32_t n_pipeline
                     uint32_t lambda_num, uint32_t lambda_den, uint64_t seed, uint32_t mode,
                     int64_t* d_w_us, void* d_workspace, uint64_t workspace_bytes,
                     void* cuda_stream);
+
+/* Adaptive request priority with delayed transition (Sec. 4.3): chooses, for
+ * every (ctx, stage) queue, the decision order that pard_plan reads from
+ * pard_queue_state_t.d_priority.  With
+ *   T_in   the queue's input workload: d_arrivals[(ctx * stage_stride + stage)
+ *          * n_hist + j], j < n_hist, requests that arrived in the j-th sampling
+ *          interval of interval_us microseconds, oldest first, each in
+ *          [0, PARD_RATE_LIMIT)
+ *   T_s    T_in smoothed by a sliding-window average over `window` samples,
+ *          defined from sample window - 1 on (earlier samples only fill the
+ *          window)
+ *   eps  = sum |T_in - T_s| / sum T_in           (both sums from sample window - 1 on)
+ *   T_m  = B_k * m_k / d_k(B_k)                  module throughput from batch size and
+ *                                                execution duration
+ *   mu   = T_in / T_m                            T_in: the latest sample as a rate
+ * the queue's priority becomes 1 (high budget first) when mu > 1 + eps, 0 (low
+ * budget first) when mu < 1 - eps, and is left as it is in between; a queue
+ * without any arrival in the summed samples gets 0.  Comparisons are exact
+ * (integers, cross-multiplied).
+ *   d_batch, d_workers  DEVICE, as in pard_queue_state_t (d_workers NULL => 1);
+ *                       B_k * m_k must stay below 2^31
+ *   d_priority          DEVICE, uint8 [n_ctx][stage_stride], read (previous
+ *                       priority) and written; entries of stages the ctx's
+ *                       pipeline lacks are left untouched
+ *   d_workspace         DEVICE, 256-byte aligned, pard_update_priority_workspace_bytes()
+ *   mode                0 or PARD_MODE_NOWAIT (pard_plan_status fetches the status)
+ * 1 <= window <= n_hist <= PARD_MAX_HISTORY, 1 <= interval_us < 2^31.
+ * Host-detectable errors come back before anything is launched; a batch size,
+ * worker count or sample out of range gives PARD_EDATA with unspecified
+ * outputs.  One kernel is enqueued on cuda_stream; nothing is allocated. */
+int pard_update_priority_workspace_bytes(uint32_t n_pipelines, uint64_t* bytes);
+int pard_update_priority(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+                         const int32_t* d_pipeline_of_ctx, uint32_t n_ctx, int32_t stage_stride,
+                         const int32_t* d_batch, const int32_t* d_workers,
+                         const uint32_t* d_arrivals, uint32_t n_hist, uint32_t window,
+                         uint32_t interval_us, uint32_t mode, uint8_t* d_priority,
+                         void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
 
 /* ---- optional device timing of the planner's phases ----------------------
  * For benchmarks.  Between pard_profile_begin and pard_profile_end every

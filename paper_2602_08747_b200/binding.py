@@ -26,13 +26,15 @@ PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT, PARD_MODE_SCAN, PARD_MODE_T
 PARD_N_PHASES = 15
 PARD_MAX_WAIT_SAMPLES = 1 << 15
 PARD_WAIT_LIMIT_US = 1 << 24
+PARD_MAX_HISTORY = 4096
+PARD_RATE_LIMIT = 1 << 24
 
 EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pipeline_n_stages",
            "pard_pipeline_n_slots", "pard_pipeline_paths", "pard_plan_workspace_bytes", "pard_plan",
            "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput", "pard_plan_status",
            "pard_plan_kernel_launches", "pard_profile_begin", "pard_profile_end",
            "pard_profile_phase_name", "pard_plan_static", "pard_estimate_w_workspace_bytes",
-           "pard_estimate_w"]
+           "pard_estimate_w", "pard_update_priority_workspace_bytes", "pard_update_priority"]
 
 
 class PardError(RuntimeError):
@@ -53,7 +55,7 @@ class _State(C.Structure):
     _fields_ = [("stage_stride", C.c_int32), ("slot_stride", C.c_int32),
                 ("d_pipeline_of_ctx", C.c_void_p), ("d_now_us", C.c_void_p),
                 ("d_batch", C.c_void_p), ("d_free_at_us", C.c_void_p), ("d_q_us", C.c_void_p),
-                ("d_w_us", C.c_void_p), ("d_workers", C.c_void_p)]
+                ("d_w_us", C.c_void_p), ("d_workers", C.c_void_p), ("d_priority", C.c_void_p)]
 
 
 class _Out(C.Structure):
@@ -95,6 +97,11 @@ def library() -> C.CDLL:
         lib.pard_estimate_w.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_int32, C.c_int32,
                                         C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint32,
                                         C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
+        lib.pard_update_priority_workspace_bytes.argtypes = [C.c_uint32, C.c_void_p]
+        lib.pard_update_priority.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_int32,
+                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32,
+                                             C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64,
+                                             C.c_void_p]
         lib.pard_profile_begin.argtypes = [C.c_uint32, C.c_uint32]
         lib.pard_profile_end.argtypes = [C.c_void_p, C.c_void_p]
         lib.pard_profile_phase_name.restype = C.c_char_p
@@ -195,11 +202,12 @@ class QueueStateArrays:
     w_us: object = None
     workers: object = None
     pipeline_of_ctx: object = None
+    priority: object = None
 
     def c_struct(self) -> _State:
         return _State(self.stage_stride, self.slot_stride, _ptr(self.pipeline_of_ctx),
                       _ptr(self.now_us), _ptr(self.batch), _ptr(self.free_at_us), _ptr(self.q_us),
-                      _ptr(self.w_us), _ptr(self.workers))
+                      _ptr(self.w_us), _ptr(self.workers), _ptr(self.priority))
 
 
 @dataclass
@@ -334,6 +342,28 @@ def pard_estimate_w(pipelines: Sequence[Pipeline], d_pipeline_of_ctx, n_ctx: int
     return rc
 
 
+def pard_update_priority_workspace_bytes(n_pipelines: int) -> int:
+    b = C.c_uint64()
+    _check(library().pard_update_priority_workspace_bytes(n_pipelines, C.byref(b)),
+           "pard_update_priority_workspace_bytes")
+    return b.value
+
+
+def pard_update_priority(pipelines: Sequence[Pipeline], d_pipeline_of_ctx, n_ctx: int, stage_stride: int,
+                         d_batch, d_workers, d_arrivals, n_hist: int, window: int, interval_us: int,
+                         mode: int, d_priority, d_workspace, workspace_bytes: Optional[int] = None,
+                         stream: int = 0, check: bool = True) -> int:
+    hs = _handles(pipelines)
+    wb = workspace_bytes if workspace_bytes is not None else d_workspace.numel() * d_workspace.element_size()
+    rc = library().pard_update_priority(hs, len(pipelines), _ptr(d_pipeline_of_ctx), n_ctx, stage_stride,
+                                        _ptr(d_batch), _ptr(d_workers), _ptr(d_arrivals), n_hist, window,
+                                        interval_us, mode, _ptr(d_priority), _ptr(d_workspace), wb,
+                                        stream or None)
+    if check:
+        _check(rc, "pard_update_priority")
+    return rc
+
+
 # --------------------------------------------------------------------------
 # conveniences: move a workload to the device and allocate outputs (memory only)
 # --------------------------------------------------------------------------
@@ -353,7 +383,8 @@ def device_state(state, device="cuda") -> QueueStateArrays:
                             mv(state.now_us, np.int64), mv(state.batch, np.int32),
                             mv(state.free_at_us, np.int64), mv(state.q_us, np.int64),
                             mv(state.w_us, np.int64), mv(state.workers, np.int32),
-                            mv(state.pipeline_of_ctx, np.int32))
+                            mv(state.pipeline_of_ctx, np.int32),
+                            mv(getattr(state, "priority", None), np.uint8))
 
 
 def alloc_out(n: int, n_seg: int, device="cuda") -> PlanOut:

@@ -7,7 +7,7 @@
 namespace {
 
 struct HostLayout {
-  uint64_t plan, req, pipeline_of_ctx, now, batch, free_at, q, w, workers;
+  uint64_t plan, req, pipeline_of_ctx, now, batch, free_at, q, w, workers, priority;
   uint64_t keep, est, perm, kept_idx, n_kept, seg_off, seg_kept, total;
   uint64_t plan_bytes;
 };
@@ -30,6 +30,7 @@ int make_host_layout(uint64_t n, uint32_t n_ctx, int32_t S, int32_t R, HostLayou
   L->q = o;               o = al(o + 8 * segs);
   L->w = o;               o = al(o + 8ull * n_ctx * (uint64_t)R);
   L->workers = o;         o = al(o + 4 * segs);
+  L->priority = o;        o = al(o + segs);
   L->keep = o;            o = al(o + n);
   L->est = o;             o = al(o + 8 * n);
   L->perm = o;            o = al(o + 4 * n);
@@ -96,6 +97,8 @@ extern "C" int pard_plan_host(const pard_pipeline_t* const* pipelines, uint32_t 
   d.d_w_us = (const int64_t*)p;
   p = up(L.workers, st->d_workers, 4 * segs);            fail |= p == (const void*)-1;
   d.d_workers = (const int32_t*)p;
+  p = up(L.priority, st->d_priority, segs);              fail |= p == (const void*)-1;
+  d.d_priority = (const uint8_t*)p;
   if (fail) return PARD_ECUDA;
 
   pard_plan_out_t dout;

@@ -23,6 +23,9 @@ constexpr int kMaxPasses = 8;
 constexpr int kBins = 256;
 constexpr uint32_t kUClamp = (1u << 30) - 1;       /* >= any request count      */
 constexpr uint32_t kMaxPipelinesPerCall = 65536;
+constexpr uint32_t kSegNarrow = 1u;                /* bits of PardSegConst::narrow */
+constexpr uint32_t kSegNoStage = 2u;
+constexpr uint32_t kSegHighFirst = 4u;
 constexpr uint32_t kSpinLimit = 1u << 18;          /* polling rounds (about a microsecond each) before giving up */
 
 constexpr int kSortThreads = 512;
@@ -245,7 +248,8 @@ __device__ __forceinline__ unsigned long long magic64(unsigned long long d) {
 __global__ void __launch_bounds__(128)
 k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
             pard_queue_state_t st, uint32_t n_ctx,
-            const unsigned long long* __restrict__ ctx_dmin_inv, PardSegConst* __restrict__ ktab,
+            const unsigned long long* __restrict__ ctx_dmin_inv,
+            const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
             PlanHeader* hdr) {
   pdl_wait();
   const uint32_t S = (uint32_t)st.stage_stride;
@@ -299,11 +303,15 @@ k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
         out.d = d;
         out.cap = (uint32_t)(cap > (int64_t)(1u << 30) ? (int64_t)(1u << 30) : cap);
         out.A = base + d + lsub;
-        out.A_rel = out.A - (int64_t)(~ctx_dmin_inv[c]);
+        /* A against the origin of the queue's deadline offsets: offsets count up from the ctx's
+         * smallest deadline, or, for a queue served high budget first, down from its largest */
+        const bool high_first = st.d_priority && st.d_priority[(size_t)c * S + k] != 0;
+        out.A_rel = high_first ? (int64_t)ctx_dmax[c] - out.A : out.A - (int64_t)(~ctx_dmin_inv[c]);
         out.d_magic = (d >= 2 && d < ((int64_t)1 << 32)) ? magic64((uint64_t)d) : 0;
         out.cap_magic = out.cap >= 2 ? magic64(out.cap) : 0;
         const int64_t lim = (int64_t)1 << 29;
         out.narrow = (out.d_magic != 0 && d < ((int64_t)1 << 31) && out.A_rel > -lim && out.A_rel < lim) ? 1u : 0u;
+        if (high_first) out.narrow |= kSegHighFirst;
         out.a_rel32 = (int32_t)out.A_rel;
         out.d32 = (uint32_t)d;
       }
@@ -316,7 +324,8 @@ k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
 /* request -> sort element; digit histograms of every pass */
 __global__ void __launch_bounds__(256)
 k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
-       const unsigned long long* __restrict__ ctx_dmin_inv, uint32_t ibits,
+       const unsigned long long* __restrict__ ctx_dmin_inv, const unsigned long long* __restrict__ ctx_dmax,
+       const uint8_t* __restrict__ priority, uint32_t ibits,
        const PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
        uint32_t* __restrict__ hist) {
   pdl_wait();
@@ -333,8 +342,12 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
     uint32_t ctx = r.z, stage = r.w & 0xffffu;
     unsigned long long e;
     if (ctx < n_ctx && stage < S) {
-      unsigned long long off = (D - ~ctx_dmin_inv[ctx]) & dmask;
-      e = ((((unsigned long long)(ctx * S + stage) << dbits) | off) << ibits) | j;
+      /* ascending offsets give the queue's decision order: deadlines counted up from the ctx's
+       * smallest, or down from its largest when the queue is served high budget first */
+      const uint32_t seg = ctx * S + stage;
+      const bool high_first = priority && __ldg(&priority[seg]) != 0;
+      unsigned long long off = (high_first ? ctx_dmax[ctx] - D : D - ~ctx_dmin_inv[ctx]) & dmask;
+      e = ((((unsigned long long)seg << dbits) | off) << ibits) | j;
     } else {
       e = j;                                  /* flagged by the prepass; keep indices in range */
     }
@@ -609,6 +622,12 @@ __device__ __forceinline__ uint32_t threshold_u(int64_t X, const PardSegConst& K
   return u > kUClamp ? kUClamp : (uint32_t)u;
 }
 
+/* X = deadline - A of a request from its deadline offset: offsets of a queue served high
+ * budget first count down from the ctx's largest deadline, and A_rel is that deadline - A */
+__device__ __forceinline__ long long slack_of(unsigned long long off, const PardSegConst& K) {
+  return (K.narrow & kSegHighFirst) ? K.A_rel - (long long)off : (long long)off - K.A_rel;
+}
+
 /* 32 bytes with one access; p is 32-byte aligned */
 __device__ __forceinline__ void load4(const unsigned long long* p, unsigned long long* v) {
   asm volatile("ld.global.nc.v4.u64 {%0, %1, %2, %3}, [%4];"
@@ -656,16 +675,17 @@ __device__ __forceinline__ void tile_first_half(const TileCtx& T, uint64_t base,
   uint32_t cur_seg = seg_first;
   lheadbits = 0;
   run = seg_identity<RAW>();
-  if ((K.narrow & 2u) && base < T.n) set_status(T.hdr, PARD_EDATA);   /* queue of a stage the pipeline lacks */
-  if (one_seg && T.narrow && K.narrow == 1) {
+  if ((K.narrow & kSegNoStage) && base < T.n) set_status(T.hdr, PARD_EDATA);   /* queue of a stage the pipeline lacks */
+  if (one_seg && T.narrow && (K.narrow & (kSegNarrow | kSegNoStage)) == kSegNarrow) {
     /* one queue, and every quantity fits 32 bits: the common case */
     const uint32_t r0 = (uint32_t)base - sstart;
+    const bool high_first = K.narrow & kSegHighFirst;
 #pragma unroll
     for (int i = 0; i < kDecItems; ++i) {
       const uint32_t lo = (uint32_t)e[i], hi = (uint32_t)(e[i] >> 32);
       idx[i] = lo & T.imask;
       const uint32_t off = __funnelshift_r(lo, hi, T.ibits) & (uint32_t)T.dmask;
-      const int32_t X = (int32_t)off - K.a_rel32;
+      const int32_t X = high_first ? K.a_rel32 - (int32_t)off : (int32_t)off - K.a_rel32;
       const unsigned long long uu = (unsigned long long)(div_magic32((uint32_t)X, K.d_magic) + 1u) * K.cap;
       u[i] = X < 0 ? 0u : (uu > kUClamp ? kUClamp : (uint32_t)uu);
       r[i] = r0 + i;
@@ -689,11 +709,11 @@ __device__ __forceinline__ void tile_first_half(const TileCtx& T, uint64_t base,
           cur_seg = sg;
           K = T.ktab[sg];
           sstart = T.seg_off[sg];
-          if (K.narrow & 2u) set_status(T.hdr, PARD_EDATA);
+          if (K.narrow & kSegNoStage) set_status(T.hdr, PARD_EDATA);
         }
       }
       r[i] = (uint32_t)j - sstart;
-      u[i] = threshold_u((int64_t)off - K.A_rel, K);
+      u[i] = threshold_u(slack_of(off, K), K);
     } else {
       idx[i] = 0; r[i] = 0; u[i] = kUClamp;                    /* acts as a head, never read */
     }
@@ -852,8 +872,8 @@ __global__ void __launch_bounds__(kDecThreads, 3)
 k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
          const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
          const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-         const int32_t* __restrict__ carry, uint8_t* __restrict__ out_keep,
-         long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
+         const uint32_t* __restrict__ win_off, const int32_t* __restrict__ carry,
+         uint8_t* __restrict__ out_keep, long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
          uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept) {
   pdl_wait();
   constexpr int WARPS = kDecThreads / 32;
@@ -901,8 +921,13 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
     K = ktab[seg_first];
     sstart = seg_off[seg_first];
   }
-  const bool fast = one_seg && T.narrow && K.narrow == 1;
+  /* A queue served high budget first keeps a prefix (thresholds fall along the queue while
+   * positions rise); win_off holds the length of that prefix, and the admitted position is
+   * the raw one capped by it. */
+  uint32_t hb_kept = (K.narrow & kSegHighFirst) ? win_off[seg_first] : 0u;
+  const bool fast = one_seg && T.narrow && (K.narrow & (kSegNarrow | kSegNoStage)) == kSegNarrow;
   if (fast) {
+    const bool high_first = K.narrow & kSegHighFirst;
 #pragma unroll
     for (int i = 0; i < kDecItems; ++i) {
       const bool local = (lheadbits >> i) & 1u;
@@ -913,6 +938,7 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
         ahead = r[i] == 0 ? 0u : (uint32_t)pre;
       } else {
         c = r[i] == 0 ? 0u : (uint32_t)min((int32_t)r[i] - 1 + pre, (int32_t)r[i]);   /* both below 2^31 */
+        if (high_first) c = min(r[i], hb_kept);
         ahead = c;
       }
       const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;
@@ -933,6 +959,7 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
         K = ktab[sg];
         sstart = seg_off[sg];
         send = seg_off[sg + 1];
+        hb_kept = (K.narrow & kSegHighFirst) ? win_off[sg] : 0u;
       }
     }
     /* reduction over the earlier requests of the same queue */
@@ -949,6 +976,7 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
         const int64_t cc = (int64_t)r[i] - 1 + pre;               /* r-1 + min over t < r of (u_t - t) */
         c = cc < (int64_t)r[i] ? (uint32_t)cc : r[i];
       }
+      if (K.narrow & kSegHighFirst) c = min(r[i], hb_kept);
       ahead = c;
     }
     const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;     /* floor(c / cap) */
@@ -1075,11 +1103,32 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
     if (out_seg_off) out_seg_off[s] = lo[0];
   }
   if (s == n_seg) return;
+  /* A queue served high budget first needs no window table: its thresholds fall along the
+   * queue while the positions rise, so the kept requests are a prefix of it.  The prefix
+   * length (first position r with r >= u_r) is found by a 32-ary search and handed to the
+   * decision kernels in win_off. */
+  if (lo[1] > lo[0] && !wide && (ktab[s].narrow & (kSegHighFirst | kSegNoStage)) == kSegHighFirst) {
+    const PardSegConst K = ktab[s];
+    const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+    uint32_t a = lo[0], b = lo[1];
+    while (a < b) {                                /* uniform across the warp */
+      const uint32_t span = b - a;
+      const uint32_t p = a + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);   /* a <= p < b */
+      const bool kept = p - lo[0] < threshold_u(slack_of((__ldg(src + p) >> ibits) & dmask, K), K);
+      const uint32_t k = __popc(__ballot_sync(0xffffffffu, kept));   /* lanes 0..k-1 probe kept requests */
+      const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
+      const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
+      if (k > 0) a = p_below + 1;
+      if (k < 32) b = p_at;
+    }
+    if (lane == 0) { win_off[s] = a - lo[0]; win_cnt[s] = 0; }
+    return;
+  }
   /* batch windows of the queue: 0..b_last of its requests, plus the end marker */
   uint32_t w = 0, first = 0;
   if (lane == 0 && lo[1] > lo[0] && !wide) {
     const PardSegConst K = ktab[s];
-    if (K.narrow & 2u) {
+    if (K.narrow & kSegNoStage) {
       set_status(hdr, PARD_EDATA);               /* requests queued at a stage the pipeline lacks */
     } else {
       const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
@@ -1232,7 +1281,8 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
   uint32_t cur_seg = (uint32_t)(e[0] >> T.kshift);
   PardSegConst K = ktab[cur_seg];
   uint32_t sstart = seg_off[cur_seg], send = seg_off[cur_seg + 1], woff = win_off[cur_seg];
-  const bool narrow = T.narrow && K.narrow == 1 && full && cur_seg == (uint32_t)(e[kDecItems - 1] >> T.kshift);
+  const bool narrow = T.narrow && (K.narrow & (kSegNarrow | kSegNoStage)) == kSegNarrow && full &&
+                      cur_seg == (uint32_t)(e[kDecItems - 1] >> T.kshift);
 
   uint32_t keepbits = 0, idx[kDecItems];
   long long est[kDecItems];
@@ -1245,7 +1295,8 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
     if (valid) {
       long long X;
       if (narrow) {
-        X = (int32_t)(__funnelshift_r((uint32_t)e[i], (uint32_t)(e[i] >> 32), T.ibits) & (uint32_t)T.dmask) - K.a_rel32;
+        const int32_t off = (int32_t)(__funnelshift_r((uint32_t)e[i], (uint32_t)(e[i] >> 32), T.ibits) & (uint32_t)T.dmask);
+        X = (K.narrow & kSegHighFirst) ? K.a_rel32 - off : off - K.a_rel32;
       } else {
         const uint32_t sg = (uint32_t)(e[i] >> T.kshift);
         if (sg != cur_seg) {
@@ -1255,11 +1306,15 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
           send = seg_off[sg + 1];
           woff = win_off[sg];
         }
-        X = (long long)((e[i] >> T.ibits) & T.dmask) - K.A_rel;
+        X = slack_of((e[i] >> T.ibits) & T.dmask, K);
       }
       const uint32_t r = (uint32_t)j - sstart;
       uint32_t u = 0;
-      if (X >= 0) {                                   /* window b of the request and its table entry */
+      if (K.narrow & kSegHighFirst) {                 /* the kept requests are the first woff of the queue */
+        u = threshold_u(X, K);
+        ahead = min(r, woff);
+        c = RAW ? r : ahead;
+      } else if (X >= 0) {                            /* window b of the request and its table entry */
         const uint32_t b = (uint32_t)win_of((unsigned long long)X, K);
         u = win_u(b, K.cap);
         const WinEntry w = wtab[woff + b];
@@ -1536,11 +1591,11 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   mark();
   if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
   launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr);
-  launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, d_pipes, n_pipelines, *state, n_ctx, ctx_dmin, ktab, hdr);
+  launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, d_pipes, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab, hdr);
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
-    launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ibits, hdr, buf_a, hist);
+    launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, ibits, hdr, buf_a, hist);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
@@ -1575,12 +1630,12 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     if (raw) {
       launch_pdl(k_tile_agg<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
       launch_pdl(k_tile_scan<true>, 1, 1024, 0, stream, hdr, tile_agg, L.dec_tiles, tile_carry);
-      launch_pdl(k_decide<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+      launch_pdl(k_decide<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, tile_carry,
                                                             out->d_keep, est, out->d_perm, tmp, seg_kept);
     } else {
       launch_pdl(k_tile_agg<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
       launch_pdl(k_tile_scan<false>, 1, 1024, 0, stream, hdr, tile_agg, L.dec_tiles, tile_carry);
-      launch_pdl(k_decide<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_carry,
+      launch_pdl(k_decide<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, tile_carry,
                                                              out->d_keep, est, out->d_perm, tmp, seg_kept);
     }
   }

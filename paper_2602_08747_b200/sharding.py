@@ -34,7 +34,7 @@ def shard_workload(wl: inputs.Workload, world: int, rank: int) -> inputs.Workloa
 
     state = inputs.QueueState(st.stage_stride, st.slot_stride, rows(st.now_us), rows(st.batch),
                               rows(st.free_at_us), rows(st.q_us), rows(st.w_us), rows(st.workers),
-                              rows(st.pipeline_of_ctx))
+                              rows(st.pipeline_of_ctx), rows(st.priority))
     return inputs.Workload("%s[%d/%d]" % (wl.name, rank, world), wl.pipelines, req, state, hi - lo,
                            dict(wl.notes))
 

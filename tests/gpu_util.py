@@ -73,3 +73,28 @@ def run_estimate_w(wl, samples, lambda_num, lambda_den, seed, slot_stride=None, 
     for p in pipes:
         p.free()
     return rc, w
+
+
+def run_update_priority(pipelines, pipeline_of_ctx, n_ctx, S, batch, workers, arrivals, window, interval_us,
+                        priority, check=True):
+    """pard_update_priority on cuda:0; returns (status, new priorities [n_ctx, S] as numpy)."""
+    import torch
+    pbuild.build()
+    dev = "cuda:0"
+    pipes = [pb.pard_load_pipeline(p) for p in pipelines]
+
+    def mv(a, dt):
+        return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(dev)
+
+    x = np.ascontiguousarray(arrivals, dtype=np.uint32)
+    d_prio = mv(np.asarray(priority, dtype=np.uint8).reshape(n_ctx, S), np.uint8)
+    ws = pb.alloc_workspace(pb.pard_update_priority_workspace_bytes(len(pipes)), dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    rc = pb.pard_update_priority(pipes, mv(pipeline_of_ctx, np.int32), n_ctx, S, mv(batch, np.int32),
+                                 mv(workers, np.int32), mv(x.view(np.int32), np.int32), int(x.shape[2]), window,
+                                 interval_us, 0, d_prio, ws, stream=stream, check=check)
+    torch.cuda.synchronize()
+    out = d_prio.cpu().numpy()
+    for p in pipes:
+        p.free()
+    return rc, out

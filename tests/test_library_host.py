@@ -187,3 +187,39 @@ def test_estimate_w_argument_checks_happen_before_any_launch():
     assert call(M=pb.PARD_MAX_WAIT_SAMPLES + 1) == pb.PARD_ERANGE
     assert call(S=65) == pb.PARD_ERANGE
     assert call(n_ctx=1 << 20, R=1 << 12) == pb.PARD_ERANGE
+
+
+def test_update_priority_argument_checks_happen_before_any_launch():
+    p = inputs.make_pipeline(inputs.chain_edges(2), 2, [1, 1], [[5], [5]])
+    h = pb.pard_load_pipeline(p, host_only=True)
+    lib = pb.library()
+    v = C.c_uint64()
+    assert lib.pard_update_priority_workspace_bytes(0, C.byref(v)) == pb.PARD_EINVAL
+    assert lib.pard_update_priority_workspace_bytes(1, None) == pb.PARD_EINVAL
+    assert lib.pard_update_priority_workspace_bytes(3, C.byref(v)) == pb.PARD_OK and v.value >= 256 + 24
+    hs = (C.c_void_p * 1)(h.handle)
+    buf = np.zeros(64, np.int64)
+    a = buf.ctypes.data
+
+    def call(pipes=hs, n_pipes=1, poc=None, n_ctx=1, S=2, batch=a, workers=None, x=a, H=8, W=4, tau=1000,
+             mode=0, prio=a):
+        return lib.pard_update_priority(pipes, n_pipes, poc, n_ctx, S, batch, workers, x, H, W, tau, mode, prio,
+                                        None, 0, None)
+
+    assert call(pipes=None) == pb.PARD_EINVAL
+    assert call(batch=None) == pb.PARD_EINVAL
+    assert call(x=None) == pb.PARD_EINVAL
+    assert call(prio=None) == pb.PARD_EINVAL
+    assert call(n_ctx=0) == pb.PARD_EINVAL
+    assert call(S=0) == pb.PARD_EINVAL
+    assert call(W=0) == pb.PARD_EINVAL
+    assert call(W=9) == pb.PARD_EINVAL                     # window longer than the history
+    assert call(tau=0) == pb.PARD_EINVAL
+    assert call(mode=pb.PARD_MODE_RAW) == pb.PARD_EINVAL
+    assert call(n_pipes=2) == pb.PARD_EINVAL               # several pipelines need the ctx map
+    assert call(S=65) == pb.PARD_ERANGE
+    assert call(H=pb.PARD_MAX_HISTORY + 1, W=4) == pb.PARD_ERANGE
+    assert call(tau=1 << 31) == pb.PARD_ERANGE
+    # a host-only handle cannot be used on a device (without a device the CUDA call fails first)
+    assert call() in (pb.PARD_EINVAL, pb.PARD_ECUDA)
+    h.free()

@@ -353,6 +353,11 @@ int pard_update_priority(const pard_pipeline_t* const* pipelines, uint32_t n_pip
  * number of sampled calls.  Process-wide state: do not call begin/end while
  * another thread is inside pard_plan.  The paper has no counterpart. */
 #define PARD_N_PHASES 15
+/* Or-ed into `every`: no events inside the decision pass (an event between two
+ * kernels costs a few microseconds and keeps the second from being scheduled
+ * while the first drains); "tables" then holds the time of the whole pass --
+ * window tables, decision, compaction -- and "decide", "compact" are 0. */
+#define PARD_PROFILE_COARSE 0x80000000u
 int pard_profile_begin(uint32_t every, uint32_t max_samples);
 int pard_profile_end(float* ms_sum, uint32_t* n_samples);
 /* "clear", "prepass", "segments", "pack", "sort0".."sort7", "tables", "decide", "compact" */

@@ -55,13 +55,15 @@ struct PlanHeader {
   uint32_t win_total;         /* window-table entries handed out */
   uint32_t aborted;           /* 1: a bounded wait ran out; the sort is incomplete and every later kernel returns */
   uint32_t big_total;         /* window-table entries that belong to long queues */
-  uint32_t pad[64 - 11 - (kMaxPasses + 1)];
+  uint32_t agg_done;          /* blocks of k_tile_agg that have stored their aggregates */
+  uint32_t dec_done;          /* blocks of k_decide that have stored their queues' kept counts */
+  uint32_t pad[64 - 13 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
-  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, hist, lookback, zero_end,
+  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, lookback, zero_end,
       pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
@@ -94,6 +96,7 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.ctx_dmax = o;  o = al(o + 8ull * n_ctx);
   L.seg_off = o;   o = al(o + 4ull * (L.n_seg + 1));
   L.seg_kept = o;  o = al(o + 4ull * L.n_seg);
+  L.win_done = o;  o = al(o + 4ull * L.n_seg);
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
   L.lookback = o;  o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);   /* two arrays, used in turn */
   L.zero_end = o;
@@ -756,16 +759,85 @@ __device__ __forceinline__ SegVal warp_scan(SegVal v, uint32_t lane) {
   return v;
 }
 
+/* Exclusive segmented scan of the tile aggregates by one block, eight tiles
+ * per thread and round: carry[t] is the reduction over the elements that
+ * precede tile t in the queue that is open at the start of tile t. */
+template <bool RAW, int THREADS>
+__device__ void tile_scan_block(const unsigned long long* tile_agg, uint32_t n_tiles, int32_t* carry) {
+  constexpr int PER = 8, WARPS = THREADS / 32;
+  __shared__ int32_t s_wm[32];
+  __shared__ uint32_t s_wh[32];
+  __shared__ int32_t s_cm;
+  __shared__ uint32_t s_ch;
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) { s_cm = seg_identity<RAW>().m; s_ch = 0; }
+  __syncthreads();
+  for (uint32_t b = 0; b < n_tiles; b += THREADS * PER) {
+    const uint32_t t0 = b + threadIdx.x * PER;
+    SegVal v[PER];
+    SegVal run = seg_identity<RAW>();
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      v[k] = t0 + k < n_tiles ? unpack_val(__ldcg(&tile_agg[t0 + k])) : seg_identity<RAW>();
+      run = seg_combine<RAW>(run, v[k]);
+    }
+    const SegVal inc = warp_scan<RAW>(run, lane);
+    SegVal exc;
+    exc.m = __shfl_up_sync(0xffffffffu, inc.m, 1);
+    exc.head = __shfl_up_sync(0xffffffffu, inc.head, 1);
+    if (lane == 0) exc = seg_identity<RAW>();
+    if (lane == 31) { s_wm[warp] = inc.m; s_wh[warp] = inc.head; }
+    __syncthreads();
+    if (warp == 0) {                        /* scan of the warp aggregates, led by the carry */
+      SegVal a = seg_identity<RAW>();
+      if (lane < WARPS) { a.m = s_wm[lane]; a.head = s_wh[lane]; }
+      SegVal ai = warp_scan<RAW>(a, lane);
+      SegVal ae;
+      ae.m = __shfl_up_sync(0xffffffffu, ai.m, 1);
+      ae.head = __shfl_up_sync(0xffffffffu, ai.head, 1);
+      if (lane == 0) ae = seg_identity<RAW>();
+      SegVal c0; c0.m = s_cm; c0.head = s_ch;
+      ae = seg_combine<RAW>(c0, ae);
+      const SegVal all = seg_combine<RAW>(c0, ai);
+      __syncwarp();
+      s_wm[lane] = ae.m; s_wh[lane] = ae.head;
+      if (lane == 31) { s_cm = all.m; s_ch = all.head; }
+    }
+    __syncthreads();
+    SegVal pre; pre.m = s_wm[warp]; pre.head = s_wh[warp];
+    pre = seg_combine<RAW>(pre, exc);
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      if (t0 + k < n_tiles) carry[t0 + k] = pre.m;
+      pre = seg_combine<RAW>(pre, v[k]);
+    }
+    __syncthreads();
+  }
+}
+
+/* True in every thread of exactly one block: the one whose arrival at `counter` is the last of
+ * the grid.  Every thread's earlier global writes are visible to that block afterwards. */
+__device__ __forceinline__ bool last_block_done(uint32_t* counter) {
+  __shared__ uint32_t s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  const bool last = s_last != 0;
+  if (last) __threadfence();
+  return last;
+}
+
 /* Tile aggregates: the segmented reduction over each tile of kDecTile sorted
- * elements.  Tiles are independent; k_tile_scan turns the aggregates into the
- * value carried into every tile, so that the decision kernel never waits on
- * another block. */
+ * elements.  Tiles are independent; the block that finishes last scans the
+ * aggregates into the value carried into every tile, so that the decision
+ * kernel never waits on another block. */
 template <bool RAW>
 __global__ void __launch_bounds__(kDecThreads)
 k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
            const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
            const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-           unsigned long long* __restrict__ tile_agg) {
+           unsigned long long* __restrict__ tile_agg, int32_t* __restrict__ carry) {
   pdl_wait();
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
@@ -797,65 +869,63 @@ k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restr
   }
   __syncthreads();
   }
+  /* the block that finishes last turns the aggregates into the value carried into every tile */
+  if (last_block_done(&const_cast<PlanHeader*>(hdr)->agg_done)) tile_scan_block<RAW, kDecThreads>(tile_agg, n_tiles, carry);
 }
 
-/* Exclusive segmented scan of the tile aggregates by one block, eight tiles
- * per thread and round: carry[t] is the reduction over the elements that
- * precede tile t in the queue that is open at the start of tile t. */
-template <bool RAW>
-__global__ void __launch_bounds__(1024)
-k_tile_scan(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ tile_agg,
-            uint32_t n_tiles, int32_t* __restrict__ carry) {
-  pdl_wait();
-  constexpr int PER = 8;
-  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
-  __shared__ int32_t s_wm[32];
-  __shared__ uint32_t s_wh[32];
-  __shared__ int32_t s_cm;
-  __shared__ uint32_t s_ch;
-  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) { s_cm = seg_identity<RAW>().m; s_ch = 0; }
+/* Kept requests per queue -> first output slot of every queue, the number of
+ * kCompactChunk-sized copy jobs before every queue, and the total.  One block,
+ * eight queues per thread and round. */
+template <int THREADS>
+__device__ void kept_scan_block(const uint32_t* seg_kept, uint32_t n_seg, uint32_t* kept_base,
+                                uint32_t* chunk_base, uint32_t* out_seg_kept, unsigned long long* out_n_kept) {
+  constexpr int PER = 8, WARPS = THREADS / 32;
+  __shared__ uint32_t s_a[32], s_b[32];
+  __shared__ uint32_t s_ca, s_cb;
+  if (threadIdx.x == 0) { s_ca = 0; s_cb = 0; }
   __syncthreads();
-  for (uint32_t b = 0; b < n_tiles; b += 1024 * PER) {
-    const uint32_t t0 = b + threadIdx.x * PER;
-    SegVal v[PER];
-    SegVal run = seg_identity<RAW>();
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (uint32_t base = 0; base < n_seg + 1; base += THREADS * PER) {
+    const uint32_t i0 = base + threadIdx.x * PER;
+    uint32_t v[PER], c[PER], x = 0, y = 0;
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
-      v[k] = t0 + k < n_tiles ? unpack_val(tile_agg[t0 + k]) : seg_identity<RAW>();
-      run = seg_combine<RAW>(run, v[k]);
+      v[k] = i0 + k < n_seg ? __ldcg(&seg_kept[i0 + k]) : 0;
+      c[k] = (v[k] + kCompactChunk - 1) / kCompactChunk;
+      if (out_seg_kept && i0 + k < n_seg) out_seg_kept[i0 + k] = v[k];
+      x += v[k];
+      y += c[k];
     }
-    const SegVal inc = warp_scan<RAW>(run, lane);
-    SegVal exc;
-    exc.m = __shfl_up_sync(0xffffffffu, inc.m, 1);
-    exc.head = __shfl_up_sync(0xffffffffu, inc.head, 1);
-    if (lane == 0) exc = seg_identity<RAW>();
-    if (lane == 31) { s_wm[warp] = inc.m; s_wh[warp] = inc.head; }
+    const uint32_t tx = x, ty = y;
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t p = __shfl_up_sync(0xffffffffu, x, o), q = __shfl_up_sync(0xffffffffu, y, o);
+      if (lane >= (uint32_t)o) { x += p; y += q; }
+    }
+    if (lane == 31) { s_a[warp] = x; s_b[warp] = y; }
     __syncthreads();
-    if (warp == 0) {                        /* scan of the 32 warp aggregates, led by the carry */
-      SegVal a; a.m = s_wm[lane]; a.head = s_wh[lane];
-      SegVal ai = warp_scan<RAW>(a, lane);
-      SegVal ae;
-      ae.m = __shfl_up_sync(0xffffffffu, ai.m, 1);
-      ae.head = __shfl_up_sync(0xffffffffu, ai.head, 1);
-      if (lane == 0) ae = seg_identity<RAW>();
-      SegVal c0; c0.m = s_cm; c0.head = s_ch;
-      ae = seg_combine<RAW>(c0, ae);
-      const SegVal all = seg_combine<RAW>(c0, ai);
-      s_wm[lane] = ae.m; s_wh[lane] = ae.head;
-      __syncwarp();
-      if (lane == 31) { s_cm = all.m; s_ch = all.head; }
+    if (warp == 0) {
+      const uint32_t a = lane < WARPS ? s_a[lane] : 0u, b = lane < WARPS ? s_b[lane] : 0u;
+      uint32_t ta = a, tb = b;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t p = __shfl_up_sync(0xffffffffu, ta, o), q = __shfl_up_sync(0xffffffffu, tb, o);
+        if (lane >= (uint32_t)o) { ta += p; tb += q; }
+      }
+      s_a[lane] = ta - a;
+      s_b[lane] = tb - b;
     }
     __syncthreads();
-    SegVal pre; pre.m = s_wm[warp]; pre.head = s_wh[warp];
-    pre = seg_combine<RAW>(pre, exc);
+    uint32_t ea = s_ca + s_a[warp] + x - tx, eb = s_cb + s_b[warp] + y - ty;   /* exclusive, before this thread's queues */
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
-      if (t0 + k < n_tiles) carry[t0 + k] = pre.m;
-      pre = seg_combine<RAW>(pre, v[k]);
+      if (i0 + k <= n_seg) { kept_base[i0 + k] = ea; chunk_base[i0 + k] = eb; }
+      ea += v[k];
+      eb += c[k];
     }
+    __syncthreads();
+    if (threadIdx.x == THREADS - 1) { s_ca = ea; s_cb = eb; }
     __syncthreads();
   }
+  if (threadIdx.x == 0 && out_n_kept) *out_n_kept = s_ca;
 }
 
 /* Decision pass; one tile of kDecTile sorted elements per block, a thread owns
@@ -874,12 +944,19 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
          const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
          const uint32_t* __restrict__ win_off, const int32_t* __restrict__ carry,
          uint8_t* __restrict__ out_keep, long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
-         uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept) {
+         uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept, uint32_t n_seg,
+         uint32_t* __restrict__ kept_base, uint32_t* __restrict__ chunk_base,
+         uint32_t* __restrict__ out_seg_kept, unsigned long long* __restrict__ out_n_kept) {
   pdl_wait();
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
+  if (hdr->wide || hdr->aborted || !hdr->use_scan) {
+    /* the window-table kernel has decided (or nothing could be): only the scan of the queues'
+     * kept counts is left, and one block does it */
+    if (blockIdx.x == 0) kept_scan_block<kDecThreads>(seg_kept, n_seg, kept_base, chunk_base, out_seg_kept, out_n_kept);
+    return;
+  }
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
@@ -1014,6 +1091,8 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
   }
   __syncthreads();
   }
+  if (last_block_done(&const_cast<PlanHeader*>(hdr)->dec_done))
+    kept_scan_block<kDecThreads>(seg_kept, n_seg, kept_base, chunk_base, out_seg_kept, out_n_kept);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -1155,76 +1234,17 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
   }
 }
 
-/* P of every table entry: one warp per entry searches the queue's sorted elements, 32 probes per step. */
-__global__ void __launch_bounds__(256)
-k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
-             const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
-             const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_own,
-             const uint32_t* __restrict__ win_big, WinEntry* __restrict__ wtab) {
-  pdl_wait();
-  if (hdr->use_scan || hdr->wide || hdr->aborted) return;
-  const uint32_t lane = threadIdx.x & 31;
-  /* entries of short queues: one lane each, plain binary search */
-  {
-    const uint32_t total = hdr->win_total, step = gridDim.x * blockDim.x;
-    const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
-    const uint32_t dbits = hdr->dbits;
-    const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
-    for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += step) {
-      const uint32_t s = win_own[e];
-      uint32_t lo = seg_off[s], hi = seg_off[s + 1];
-      if (hi - lo > kWinLongQueue) continue;
-      const uint32_t first = lo;
-      const long long thr = ktab[s].A_rel + (long long)(e - win_off[s]) * ktab[s].d;
-      while (lo < hi) {
-        const uint32_t mid = lo + (hi - lo) / 2;
-        if ((long long)((__ldg(src + mid) >> ibits) & dmask) < thr) lo = mid + 1; else hi = mid;
-      }
-      wtab[e].P = lo - first;
-    }
-  }
-  /* entries of long queues: one warp each, 32 probes per step */
-  const uint32_t total = hdr->big_total, step = (gridDim.x * blockDim.x) >> 5;
-  for (uint32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < total; i += step) {   /* whole warps stay together */
-  const uint32_t e = win_big[i];
-  const uint32_t s = win_own[e], b = e - win_off[s];
-  const PardSegConst K = ktab[s];
-  const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
-  const uint32_t dbits = hdr->dbits;
-  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
-  const long long thr = K.A_rel + (long long)b * K.d;     /* window >= b  <=>  deadline offset >= thr */
-  uint32_t lo = seg_off[s], hi = seg_off[s + 1];
-  const uint32_t first = lo;
-  while (lo < hi) {
-    const uint32_t span = hi - lo;
-    const uint32_t p = lo + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);
-    const bool less = (long long)((__ldg(src + p) >> ibits) & dmask) < thr;
-    const uint32_t k = __popc(__ballot_sync(0xffffffffu, less));
-    const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
-    const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
-    if (k > 0) lo = p_below + 1;
-    if (k < 32) hi = p_at;
-  }
-  if (lane == 0) wtab[e].P = lo - first;
-  }
-}
-
-/* E and Kp of every table entry: one warp per queue runs over its windows, 32 at a time. */
-__global__ void __launch_bounds__(256)
-k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
-             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
-             WinEntry* __restrict__ wtab) {
-  pdl_wait();
-  if (hdr->use_scan || hdr->wide || hdr->aborted) return;
-  const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const uint32_t lane = threadIdx.x & 31;
-  if (s >= n_seg) return;
+/* E and Kp of the table entries of one queue, once all their P are known: the warp runs over
+ * the queue's windows, 32 at a time. */
+__device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* __restrict__ ktab,
+                                                const uint32_t* __restrict__ win_off,
+                                                const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab,
+                                                uint32_t lane) {
   const uint32_t w0 = win_off[s], cnt = win_cnt[s];
   if (cnt == 0) return;
   const uint32_t cap = ktab[s].cap;
   WinEntry* tab = wtab + w0;
-  const uint32_t P0 = tab[0].P;
+  const uint32_t P0 = __ldcg(&tab[0].P);
   int32_t e_carry = P0 > 0 ? -(int32_t)(P0 - 1) : kWinInf;     /* the expired run: u = 0 */
   uint32_t k_carry = 0;
   if (lane == 0) { tab[0].E = e_carry; tab[0].Kp = 0; }
@@ -1233,7 +1253,7 @@ k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegCo
     int32_t val = kWinInf;
     uint32_t kept = 0;
     if (b + 1 < cnt) {
-      const uint32_t p = tab[b].P, q = tab[b + 1].P;
+      const uint32_t p = __ldcg(&tab[b].P), q = __ldcg(&tab[b + 1].P);
       if (q > p) {
         const uint32_t u = win_u(b, cap);
         val = (int32_t)u - (int32_t)(q - 1);
@@ -1254,8 +1274,89 @@ k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegCo
   }
 }
 
-/* Decision pass from the window tables: every request on its own. */
-template <bool RAW>
+/* The window tables.  P of every entry: a search in the queue's sorted elements, by one lane
+ * (short queue) or by a whole warp with 32 probes per step (long queue).  Every finished entry
+ * is counted per queue; the warp that finishes a queue's last entry goes on to the queue's
+ * prefix pass (E, Kp), so the tables are complete when the kernel ends. */
+__global__ void __launch_bounds__(256)
+k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+             const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
+             const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
+             const uint32_t* __restrict__ win_own, const uint32_t* __restrict__ win_big,
+             uint32_t* __restrict__ win_done, WinEntry* __restrict__ wtab) {
+  pdl_wait();
+  if (hdr->use_scan || hdr->wide || hdr->aborted) return;
+  const uint32_t lane = threadIdx.x & 31;
+  const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
+  const uint32_t dbits = hdr->dbits;
+  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  /* entries of short queues: one lane each, plain binary search; the warp stays together */
+  {
+    const uint32_t total = hdr->win_total, step = gridDim.x * blockDim.x;
+    for (uint32_t e0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; e0 < total; e0 += step) {
+      const uint32_t e = e0 + lane;
+      uint32_t s = 0;
+      bool finished = false;
+      if (e < total) {
+        s = win_own[e];
+        uint32_t lo = seg_off[s], hi = seg_off[s + 1];
+        if (hi - lo <= kWinLongQueue) {
+          const uint32_t first = lo;
+          const long long thr = ktab[s].A_rel + (long long)(e - win_off[s]) * ktab[s].d;
+          while (lo < hi) {
+            const uint32_t mid = lo + (hi - lo) / 2;
+            if ((long long)((__ldg(src + mid) >> ibits) & dmask) < thr) lo = mid + 1; else hi = mid;
+          }
+          wtab[e].P = lo - first;
+          __threadfence();
+          finished = atomicAdd(&win_done[s], 1u) + 1 == win_cnt[s];
+        }
+      }
+      uint32_t fin = __ballot_sync(0xffffffffu, finished);
+      if (fin) __threadfence();
+      while (fin) {                                  /* queues completed by this warp, one after the other */
+        const uint32_t sq = __shfl_sync(0xffffffffu, s, __ffs(fin) - 1);
+        win_prefix_warp(sq, ktab, win_off, win_cnt, wtab, lane);
+        fin &= fin - 1;
+      }
+    }
+  }
+  /* entries of long queues: one warp each, 32 probes per step */
+  const uint32_t total = hdr->big_total, step = (gridDim.x * blockDim.x) >> 5;
+  for (uint32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < total; i += step) {   /* whole warps stay together */
+    const uint32_t e = win_big[i];
+    const uint32_t s = win_own[e], b = e - win_off[s];
+    const PardSegConst K = ktab[s];
+    const long long thr = K.A_rel + (long long)b * K.d;     /* window >= b  <=>  deadline offset >= thr */
+    uint32_t lo = seg_off[s], hi = seg_off[s + 1];
+    const uint32_t first = lo;
+    while (lo < hi) {
+      const uint32_t span = hi - lo;
+      const uint32_t p = lo + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);
+      const bool less = (long long)((__ldg(src + p) >> ibits) & dmask) < thr;
+      const uint32_t k = __popc(__ballot_sync(0xffffffffu, less));
+      const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
+      const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
+      if (k > 0) lo = p_below + 1;
+      if (k < 32) hi = p_at;
+    }
+    uint32_t finished = 0;
+    if (lane == 0) {
+      wtab[e].P = lo - first;
+      __threadfence();
+      finished = atomicAdd(&win_done[s], 1u) + 1 == win_cnt[s] ? 1u : 0u;
+    }
+    if (__shfl_sync(0xffffffffu, finished, 0)) {
+      __threadfence();
+      win_prefix_warp(s, ktab, win_off, win_cnt, wtab, lane);
+    }
+  }
+}
+
+/* Decision pass from the window tables: every request on its own.  HF: some
+ * queue may be served high budget first (the caller gave priorities). */
+template <bool RAW, bool HF>
 __global__ void __launch_bounds__(kDecThreads, 4)
 k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
              const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
@@ -1296,7 +1397,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
       long long X;
       if (narrow) {
         const int32_t off = (int32_t)(__funnelshift_r((uint32_t)e[i], (uint32_t)(e[i] >> 32), T.ibits) & (uint32_t)T.dmask);
-        X = (K.narrow & kSegHighFirst) ? K.a_rel32 - off : off - K.a_rel32;
+        X = (HF && (K.narrow & kSegHighFirst)) ? K.a_rel32 - off : off - K.a_rel32;
       } else {
         const uint32_t sg = (uint32_t)(e[i] >> T.kshift);
         if (sg != cur_seg) {
@@ -1306,11 +1407,11 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
           send = seg_off[sg + 1];
           woff = win_off[sg];
         }
-        X = slack_of((e[i] >> T.ibits) & T.dmask, K);
+        X = HF ? slack_of((e[i] >> T.ibits) & T.dmask, K) : (long long)((e[i] >> T.ibits) & T.dmask) - K.A_rel;
       }
       const uint32_t r = (uint32_t)j - sstart;
       uint32_t u = 0;
-      if (K.narrow & kSegHighFirst) {                 /* the kept requests are the first woff of the queue */
+      if (HF && (K.narrow & kSegHighFirst)) {                 /* the kept requests are the first woff of the queue */
         u = threshold_u(X, K);
         ahead = min(r, woff);
         c = RAW ? r : ahead;
@@ -1365,63 +1466,6 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
   }
 }
 
-/* Kept requests per queue -> first output slot of every queue, the number of
- * kCompactChunk-sized copy jobs before every queue, and the total.  One block,
- * eight queues per thread and round. */
-__global__ void __launch_bounds__(1024)
-k_kept_scan(const uint32_t* __restrict__ seg_kept, uint32_t n_seg, uint32_t* __restrict__ kept_base,
-            uint32_t* __restrict__ chunk_base, uint32_t* __restrict__ out_seg_kept,
-            unsigned long long* __restrict__ out_n_kept) {
-  pdl_wait();
-  constexpr int PER = 8;
-  __shared__ uint32_t s_a[32], s_b[32];
-  __shared__ uint32_t s_ca, s_cb;
-  if (threadIdx.x == 0) { s_ca = 0; s_cb = 0; }
-  __syncthreads();
-  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t base = 0; base < n_seg + 1; base += 1024 * PER) {
-    const uint32_t i0 = base + threadIdx.x * PER;
-    uint32_t v[PER], c[PER], x = 0, y = 0;
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-      v[k] = i0 + k < n_seg ? seg_kept[i0 + k] : 0;
-      c[k] = (v[k] + kCompactChunk - 1) / kCompactChunk;
-      if (out_seg_kept && i0 + k < n_seg) out_seg_kept[i0 + k] = v[k];
-      x += v[k];
-      y += c[k];
-    }
-    const uint32_t tx = x, ty = y;
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t p = __shfl_up_sync(0xffffffffu, x, o), q = __shfl_up_sync(0xffffffffu, y, o);
-      if (lane >= (uint32_t)o) { x += p; y += q; }
-    }
-    if (lane == 31) { s_a[warp] = x; s_b[warp] = y; }
-    __syncthreads();
-    if (warp == 0) {
-      const uint32_t a = s_a[lane], b = s_b[lane];
-      uint32_t ta = a, tb = b;
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t p = __shfl_up_sync(0xffffffffu, ta, o), q = __shfl_up_sync(0xffffffffu, tb, o);
-        if (lane >= (uint32_t)o) { ta += p; tb += q; }
-      }
-      s_a[lane] = ta - a;
-      s_b[lane] = tb - b;
-    }
-    __syncthreads();
-    uint32_t ea = s_ca + s_a[warp] + x - tx, eb = s_cb + s_b[warp] + y - ty;   /* exclusive, before this thread's queues */
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-      if (i0 + k <= n_seg) { kept_base[i0 + k] = ea; chunk_base[i0 + k] = eb; }
-      ea += v[k];
-      eb += c[k];
-    }
-    __syncthreads();
-    if (threadIdx.x == 1023) { s_ca = ea; s_cb = eb; }
-    __syncthreads();
-  }
-  if (threadIdx.x == 0 && out_n_kept) *out_n_kept = s_ca;
-}
-
 /* Packs the queues' survivors: copy job j moves up to kCompactChunk indices of one queue; a
  * warp per job. */
 __global__ void __launch_bounds__(256)
@@ -1451,16 +1495,19 @@ constexpr int kEventsPerSample = PARD_N_PHASES + 1;
 static_assert(PARD_N_PHASES == 4 + kMaxPasses + 3, "phase list");
 struct Profiler {
   std::mutex mu;
-  bool on = false;
+  bool on = false, coarse = false;
   uint32_t every = 1, max_samples = 0, calls = 0, n_samples = 0;
   std::vector<cudaEvent_t> ev;
 };
 Profiler g_prof;
 
+constexpr int kPhaseTables = 4 + kMaxPasses;       /* "tables", then "decide", "compact" */
+
 /* events of this call if it is a sampled one, else nullptr */
-cudaEvent_t* profile_acquire() {
+cudaEvent_t* profile_acquire(bool* coarse) {
   std::lock_guard<std::mutex> lock(g_prof.mu);
   if (!g_prof.on) return nullptr;
+  *coarse = g_prof.coarse;
   uint32_t call = g_prof.calls++;
   if (call % g_prof.every != 0 || g_prof.n_samples >= g_prof.max_samples) return nullptr;
   return g_prof.ev.data() + (size_t)(g_prof.n_samples++) * kEventsPerSample;
@@ -1559,6 +1606,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   uint32_t* win_cnt = (uint32_t*)(ws + L.win_cnt);
   uint32_t* win_own = (uint32_t*)(ws + L.win_own);
   uint32_t* win_big = (uint32_t*)(ws + L.win_big);
+  uint32_t* win_done = (uint32_t*)(ws + L.win_done);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -1566,10 +1614,12 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   const uint32_t ibits = std::max(1u, ceil_log2(n));
   const uint32_t sbits = ceil_log2(L.n_seg);
 
-  cudaEvent_t* evs = profile_acquire();
+  bool prof_coarse = false;
+  cudaEvent_t* evs = profile_acquire(&prof_coarse);
   int phase = 0;
   auto mark = [&]() {                      /* boundary between two phases */
-    if (evs) cudaEventRecord(evs[phase], stream);
+    const bool inner = phase == kPhaseTables + 1 || phase == kPhaseTables + 2;   /* inside the decision pass */
+    if (evs && !(prof_coarse && inner)) cudaEventRecord(evs[phase], stream);
     ++phase;
   };
   mark();
@@ -1614,35 +1664,34 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     const bool raw = mode & PARD_MODE_RAW;
     /* window tables, and the decision from them */
     launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream, 
-        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_own, win_big, wtab);
-    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, win_off, win_cnt, wtab);
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
     mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
-    if (raw)
-      launch_pdl(k_decide_win<true>, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
-                                                               wtab, out->d_keep, est, out->d_perm, tmp, seg_kept);
-    else
-      launch_pdl(k_decide_win<false>, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
-                                                                wtab, out->d_keep, est, out->d_perm, tmp, seg_kept);
-    /* fallback when a queue has too many batch windows: the same decision by scanning
-     * (these three return at once otherwise) */
+    auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
+                          : (state->d_priority ? k_decide_win<false, true> : k_decide_win<false, false>);
+    launch_pdl(decide_win, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, wtab,
+               out->d_keep, est, out->d_perm, tmp, seg_kept);
+    /* fallback when a queue has too many batch windows: the same decision by scanning (the
+     * aggregate kernel returns at once otherwise) */
     const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3);
-    if (raw) {
-      launch_pdl(k_tile_agg<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
-      launch_pdl(k_tile_scan<true>, 1, 1024, 0, stream, hdr, tile_agg, L.dec_tiles, tile_carry);
-      launch_pdl(k_decide<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, tile_carry,
-                                                            out->d_keep, est, out->d_perm, tmp, seg_kept);
-    } else {
-      launch_pdl(k_tile_agg<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg);
-      launch_pdl(k_tile_scan<false>, 1, 1024, 0, stream, hdr, tile_agg, L.dec_tiles, tile_carry);
-      launch_pdl(k_decide<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, tile_carry,
-                                                             out->d_keep, est, out->d_perm, tmp, seg_kept);
-    }
+    if (raw)
+      launch_pdl(k_tile_agg<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg,
+                 tile_carry);
+    else
+      launch_pdl(k_tile_agg<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg,
+                 tile_carry);
   }
-  if (n == 0) mark();
+  /* the scan path's decision kernel; whichever path decided, it ends with the scan of the queues'
+   * kept counts (first output slot of every queue, copy jobs, total) */
+  {
+    if (n == 0) mark();
+    const uint32_t scan_grid = std::max<uint32_t>(1u, std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3));
+    auto decide = (mode & PARD_MODE_RAW) ? k_decide<true> : k_decide<false>;
+    launch_pdl(decide, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, tile_carry,
+               out->d_keep, (long long*)out->d_est_us, out->d_perm, out->d_kept_idx ? kept_tmp : nullptr, seg_kept,
+               L.n_seg, kept_base, chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept);
+  }
   mark();
-  launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
-                                      (unsigned long long*)out->d_n_kept);
   if (n > 0 && out->d_kept_idx)
     launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
                                                (uint32_t)sms * 8), 256, 0, stream, 
@@ -1669,14 +1718,16 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* key_width, seg_const, seg_win, kept_scan always; prepass, ctx_span, pack, passes, decide and
-   * win_bounds, win_prefix, decide_win, tile_agg, tile_scan and kept_move (when the
-   * compacted indices are requested) when n > 0 */
-  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 7 : 4;
+  /* key_width, seg_const, seg_win and the scan path's decision kernel (which ends with the scan of
+   * the kept counts) always; prepass, ctx_span, pack, the passes, win_bounds, decide_win, tile_agg
+   * and kept_move (when the compacted indices are requested) when n > 0 */
+  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 4 : 4;
   return PARD_OK;
 }
 
 extern "C" int pard_profile_begin(uint32_t every, uint32_t max_samples) {
+  const bool coarse = (every & PARD_PROFILE_COARSE) != 0;
+  every &= ~PARD_PROFILE_COARSE;
   if (every < 1 || max_samples < 1 || max_samples > 65536) return PARD_EINVAL;
   std::lock_guard<std::mutex> lock(g_prof.mu);
   if (g_prof.on) return PARD_EINVAL;
@@ -1688,6 +1739,7 @@ extern "C" int pard_profile_begin(uint32_t every, uint32_t max_samples) {
       return PARD_ECUDA;
     }
   g_prof.every = every;
+  g_prof.coarse = coarse;
   g_prof.max_samples = max_samples;
   g_prof.calls = 0;
   g_prof.n_samples = 0;
@@ -1705,7 +1757,10 @@ extern "C" int pard_profile_end(float* ms_sum, uint32_t* n_samples) {
     if (cudaEventSynchronize(e[PARD_N_PHASES]) != cudaSuccess) { rc = PARD_ECUDA; break; }
     for (int i = 0; i < PARD_N_PHASES && ms_sum; ++i) {
       float ms = 0.f;
-      if (cudaEventElapsedTime(&ms, e[i], e[i + 1]) != cudaSuccess) rc = PARD_ECUDA;
+      int to = i + 1;
+      if (g_prof.coarse && i == kPhaseTables) to = PARD_N_PHASES;       /* the decision pass as one phase */
+      if (g_prof.coarse && i > kPhaseTables) continue;
+      if (cudaEventElapsedTime(&ms, e[i], e[to]) != cudaSuccess) rc = PARD_ECUDA;
       ms_sum[i] += ms;
     }
   }

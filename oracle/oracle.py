@@ -65,6 +65,9 @@ def lib():
         _lib.oracle_update_priority.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint32, C.c_int32,
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32,
                                                 C.c_uint32, C.c_void_p]
+        _lib.oracle_queue_delay.restype = C.c_int
+        _lib.oracle_queue_delay.argtypes = [C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_uint32, C.c_uint32, C.c_void_p]
     return _lib
 
 
@@ -150,6 +153,21 @@ def update_priority(pipelines, pipeline_of_ctx, n_ctx: int, stage_stride: int, b
     if rc != 0:
         raise ValueError("oracle_update_priority: bad input")
     return out
+
+
+def queue_delay(now_us, sample_time_us, sample_delay_us, window_us: int) -> np.ndarray:
+    """q[n_ctx, stage_stride] (int64): the linear weighted sliding-window average of the recorded
+    queueing delays.  sample_time_us int64 and sample_delay_us int32 are [n_ctx, stage_stride, M]."""
+    t = np.ascontiguousarray(sample_time_us, dtype=np.int64)
+    d = np.ascontiguousarray(sample_delay_us, dtype=np.int32)
+    now = np.ascontiguousarray(now_us, dtype=np.int64)
+    assert t.shape == d.shape and t.ndim == 3 and now.shape == (t.shape[0],)
+    q = np.zeros(t.shape[:2], dtype=np.int64)
+    rc = lib().oracle_queue_delay(t.shape[0], t.shape[1], now.ctypes.data, t.ctypes.data, d.ctypes.data,
+                                  t.shape[2], window_us, q.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle_queue_delay: bad input")
+    return q
 
 
 def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:

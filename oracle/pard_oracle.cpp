@@ -14,6 +14,7 @@
  *   Order:  low budget first = smallest remaining budget first, or high
  *           budget first = largest first, per queue                (Sec. 4.3)
  *   mu/eps: load factor, fluctuation bound, delayed transition     (Sec. 4.3)
+ *   q_k:    linear weighted sliding-window average queueing delay  (Sec. 4.2)
  *   Rule:   drop when the estimate exceeds the latency objective (Sec. 5.3)
  *   Counts: goodput / drop rate                                 (Sec. 5.1)
  *   w_k:    quantile lambda of the sampled aggregated batch wait  (Sec. 4.2)
@@ -313,6 +314,34 @@ extern "C" int oracle_update_priority(const oracle_pipeline_t* pipelines, int32_
       } else if (W * sum_x > dev && lhs < scale * (u128)(W * sum_x - dev)) {
         priority[seg] = 0;                                /* within capacity: low budget first */
       }                                                   /* else: inside [1 - eps, 1 + eps], unchanged */
+    }
+  }
+  return 0;
+}
+
+extern "C" int oracle_queue_delay(uint32_t n_ctx, int32_t stage_stride, const int64_t* now_us,
+                                  const int64_t* sample_time_us, const int32_t* sample_delay_us,
+                                  uint32_t n_samples, uint32_t window_us, int64_t* q_us) {
+  typedef unsigned __int128 u128;
+  if (window_us < 1 || stage_stride < 1) return -1;
+  for (uint32_t c = 0; c < n_ctx; ++c) {
+    for (int32_t k = 0; k < stage_stride; ++k) {
+      size_t seg = (size_t)c * stage_stride + k;
+      u128 weighted = 0;                                   /* sum weight_j * delay_j */
+      u128 weights = 0;                                    /* sum weight_j */
+      for (uint32_t j = 0; j < n_samples; ++j) {
+        int64_t t = sample_time_us[seg * n_samples + j];
+        if (t < 0) continue;                               /* empty slot */
+        int32_t delay = sample_delay_us[seg * n_samples + j];
+        if (delay < 0) return -1;
+        if (t > now_us[c]) continue;                       /* not yet happened at this snapshot */
+        int64_t age = now_us[c] - t;
+        if (age >= (int64_t)window_us) continue;           /* slid out of the window */
+        uint64_t weight = (uint64_t)window_us - (uint64_t)age;   /* newest: window, oldest: 1 */
+        weighted += (u128)weight * (u128)(uint64_t)delay;
+        weights += weight;
+      }
+      q_us[seg] = weights == 0 ? 0 : (int64_t)(weighted / weights);
     }
   }
   return 0;

@@ -125,6 +125,21 @@ int oracle_update_priority(const oracle_pipeline_t* pipelines, int32_t n_pipelin
                            uint32_t n_hist, uint32_t window, uint32_t interval_us,
                            uint8_t* priority);
 
+/* Recent average queueing delay q_k of the State Planner (Sec. 4.2: monitored
+ * with a sliding window, by default a 5 s linear weighted one).  For every
+ * (ctx, stage): over the recorded samples j < n_samples, taken at time
+ * sample_time_us[..][j] with measured queueing delay sample_delay_us[..][j],
+ *   weight_j = window_us - (now - t_j)   if 0 <= now - t_j < window_us, else 0
+ *   q        = floor( sum weight_j * delay_j / sum weight_j ),  0 when no sample
+ *              has a positive weight
+ * so the newest sample weighs most and the weight falls linearly to zero at the
+ * far end of the window.  A slot with a negative time is empty.  Arrays are
+ * [n_ctx][stage_stride][n_samples] (samples in any order), now_us is [n_ctx],
+ * q_us is [n_ctx][stage_stride].  Returns 0, or -1 on bad input. */
+int oracle_queue_delay(uint32_t n_ctx, int32_t stage_stride, const int64_t* now_us,
+                       const int64_t* sample_time_us, const int32_t* sample_delay_us,
+                       uint32_t n_samples, uint32_t window_us, int64_t* q_us);
+
 #ifdef __cplusplus
 }
 #endif

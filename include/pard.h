@@ -37,6 +37,8 @@ extern "C" {
 #define PARD_MAX_WAIT_SAMPLES (1u << 15)   /* samples per slot in pard_estimate_w      */
 #define PARD_MAX_HISTORY     4096         /* workload samples per queue in pard_update_priority */
 #define PARD_RATE_LIMIT      (1u << 24)   /* arrivals per sampling interval lie in [0, 2^24) */
+#define PARD_MAX_DELAY_SAMPLES (1u << 15) /* queueing-delay samples per queue in pard_update_queue_delay */
+#define PARD_MAX_DELAY_WINDOW_US (1u << 24) /* longest sliding window of pard_update_queue_delay */
 #define PARD_WAIT_LIMIT_US   (1 << 24)    /* recorded batch waits lie in [0, 2^24)  */
 #define PARD_TIME_LIMIT_US   (1ll << 60)  /* every time input lies in [0, 2^60)     */
 #define PARD_LAT_LIMIT_US    (1ll << 40)  /* every profile entry lies in [1, 2^40)  */
@@ -306,6 +308,33 @@ int pard_estimate_w(const pard_pipeline_t* const* pipelines, uint32_t n_pipeline
                     uint32_t lambda_num, uint32_t lambda_den, uint64_t seed, uint32_t mode,
                     int64_t* d_w_us, void* d_workspace, uint64_t workspace_bytes,
                     void* cuda_stream);
+
+/* Recent average queueing delay q_k of the State Planner (Sec. 4.2, first
+ * bullet: monitored with a sliding window, by default a 5 s linear weighted
+ * one).  For every (ctx, stage), over its recorded samples j < n_samples --
+ * taken at time d_sample_time_us[(ctx * stage_stride + stage) * n_samples + j]
+ * with measured queueing delay d_sample_delay_us[same index], in any order --
+ *   weight_j = window_us - (now - t_j)   if 0 <= now - t_j < window_us, else 0
+ *   q        = floor( sum weight_j * delay_j / sum weight_j )
+ * and q = 0 when no sample has a positive weight: the newest sample weighs
+ * most and the weight falls linearly to zero at the far end of the window.
+ * A slot with a negative time is empty; delays lie in [0, PARD_WAIT_LIMIT_US).
+ * The result, int64 [n_ctx][stage_stride], is what pard_queue_state_t.d_q_us
+ * expects; d_now_us is [n_ctx] as in pard_queue_state_t.
+ *   d_sample_time_us   DEVICE, int64, 8-byte aligned
+ *   d_sample_delay_us  DEVICE, int32
+ *   d_workspace        DEVICE, 256-byte aligned, pard_update_queue_delay_workspace_bytes()
+ *   mode               0 or PARD_MODE_NOWAIT (pard_plan_status fetches the status)
+ * n_samples <= PARD_MAX_DELAY_SAMPLES, 1 <= window_us <= PARD_MAX_DELAY_WINDOW_US.
+ * Host-detectable errors come back before anything is launched; a delay out of
+ * range gives PARD_EDATA with unspecified outputs.  One kernel is enqueued on
+ * cuda_stream; nothing is allocated. */
+int pard_update_queue_delay_workspace_bytes(uint64_t* bytes);
+int pard_update_queue_delay(uint32_t n_ctx, int32_t stage_stride, const int64_t* d_now_us,
+                            const int64_t* d_sample_time_us, const int32_t* d_sample_delay_us,
+                            uint32_t n_samples, uint32_t window_us, uint32_t mode,
+                            int64_t* d_q_us, void* d_workspace, uint64_t workspace_bytes,
+                            void* cuda_stream);
 
 /* Adaptive request priority with delayed transition (Sec. 4.3): chooses, for
  * every (ctx, stage) queue, the decision order that pard_plan reads from

@@ -29,13 +29,16 @@ PARD_MAX_WAIT_SAMPLES = 1 << 15
 PARD_WAIT_LIMIT_US = 1 << 24
 PARD_MAX_HISTORY = 4096
 PARD_RATE_LIMIT = 1 << 24
+PARD_MAX_DELAY_SAMPLES = 1 << 15
+PARD_MAX_DELAY_WINDOW_US = 1 << 24
 
 EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pipeline_n_stages",
            "pard_pipeline_n_slots", "pard_pipeline_paths", "pard_plan_workspace_bytes", "pard_plan",
            "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput", "pard_plan_status",
            "pard_plan_kernel_launches", "pard_profile_begin", "pard_profile_end",
            "pard_profile_phase_name", "pard_plan_static", "pard_estimate_w_workspace_bytes",
-           "pard_estimate_w", "pard_update_priority_workspace_bytes", "pard_update_priority"]
+           "pard_estimate_w", "pard_update_priority_workspace_bytes", "pard_update_priority",
+           "pard_update_queue_delay_workspace_bytes", "pard_update_queue_delay"]
 
 
 class PardError(RuntimeError):
@@ -103,6 +106,10 @@ def library() -> C.CDLL:
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32,
                                              C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64,
                                              C.c_void_p]
+        lib.pard_update_queue_delay_workspace_bytes.argtypes = [C.c_void_p]
+        lib.pard_update_queue_delay.argtypes = [C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
+                                                C.c_uint64, C.c_void_p]
         lib.pard_profile_begin.argtypes = [C.c_uint32, C.c_uint32]
         lib.pard_profile_end.argtypes = [C.c_void_p, C.c_void_p]
         lib.pard_profile_phase_name.restype = C.c_char_p
@@ -362,6 +369,24 @@ def pard_update_priority(pipelines: Sequence[Pipeline], d_pipeline_of_ctx, n_ctx
                                         stream or None)
     if check:
         _check(rc, "pard_update_priority")
+    return rc
+
+
+def pard_update_queue_delay_workspace_bytes() -> int:
+    b = C.c_uint64()
+    _check(library().pard_update_queue_delay_workspace_bytes(C.byref(b)), "pard_update_queue_delay_workspace_bytes")
+    return b.value
+
+
+def pard_update_queue_delay(n_ctx: int, stage_stride: int, d_now_us, d_sample_time_us, d_sample_delay_us,
+                            n_samples: int, window_us: int, mode: int, d_q_us, d_workspace,
+                            workspace_bytes: Optional[int] = None, stream: int = 0, check: bool = True) -> int:
+    wb = workspace_bytes if workspace_bytes is not None else d_workspace.numel() * d_workspace.element_size()
+    rc = library().pard_update_queue_delay(n_ctx, stage_stride, _ptr(d_now_us), _ptr(d_sample_time_us),
+                                           _ptr(d_sample_delay_us), n_samples, window_us, mode, _ptr(d_q_us),
+                                           _ptr(d_workspace), wb, stream or None)
+    if check:
+        _check(rc, "pard_update_queue_delay")
     return rc
 
 

@@ -98,3 +98,22 @@ def run_update_priority(pipelines, pipeline_of_ctx, n_ctx, S, batch, workers, ar
     for p in pipes:
         p.free()
     return rc, out
+
+
+def run_queue_delay(now_us, sample_time_us, sample_delay_us, window_us, check=True):
+    """pard_update_queue_delay on cuda:0; returns (status, q [n_ctx, S] as numpy)."""
+    import torch
+    pbuild.build()
+    dev = "cuda:0"
+    t = np.ascontiguousarray(sample_time_us, dtype=np.int64)
+    d = np.ascontiguousarray(sample_delay_us, dtype=np.int32)
+    n_ctx, S, M = t.shape
+    d_t = torch.from_numpy(t).to(dev) if M else None
+    d_d = torch.from_numpy(d).to(dev) if M else None
+    d_now = torch.from_numpy(np.ascontiguousarray(now_us, dtype=np.int64)).to(dev)
+    d_q = torch.full((n_ctx, S), -7, dtype=torch.int64, device=dev)
+    ws = pb.alloc_workspace(pb.pard_update_queue_delay_workspace_bytes(), dev)
+    rc = pb.pard_update_queue_delay(n_ctx, S, d_now, d_t, d_d, M, window_us, 0, d_q, ws,
+                                    stream=torch.cuda.current_stream().cuda_stream, check=check)
+    torch.cuda.synchronize()
+    return rc, d_q.cpu().numpy()

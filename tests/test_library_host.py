@@ -223,3 +223,30 @@ def test_update_priority_argument_checks_happen_before_any_launch():
     # a host-only handle cannot be used on a device (without a device the CUDA call fails first)
     assert call() in (pb.PARD_EINVAL, pb.PARD_ECUDA)
     h.free()
+
+
+def test_update_queue_delay_argument_checks_happen_before_any_launch():
+    lib = pb.library()
+    v = C.c_uint64()
+    assert lib.pard_update_queue_delay_workspace_bytes(None) == pb.PARD_EINVAL
+    assert lib.pard_update_queue_delay_workspace_bytes(C.byref(v)) == pb.PARD_OK and v.value >= 256
+    buf = np.zeros(64, np.int64)
+    a = buf.ctypes.data
+
+    def call(n_ctx=1, S=2, now=a, t=a, d=a, M=8, window=1000, mode=0, q=a, ws=None, wsb=0):
+        return lib.pard_update_queue_delay(n_ctx, S, now, t, d, M, window, mode, q, ws, wsb, None)
+
+    assert call(n_ctx=0) == pb.PARD_EINVAL
+    assert call(S=0) == pb.PARD_EINVAL
+    assert call(now=None) == pb.PARD_EINVAL
+    assert call(q=None) == pb.PARD_EINVAL
+    assert call(t=None) == pb.PARD_EINVAL
+    assert call(d=None) == pb.PARD_EINVAL
+    assert call(window=0) == pb.PARD_EINVAL
+    assert call(mode=pb.PARD_MODE_RAW) == pb.PARD_EINVAL
+    assert call(S=65) == pb.PARD_ERANGE
+    assert call(M=pb.PARD_MAX_DELAY_SAMPLES + 1) == pb.PARD_ERANGE
+    assert call(window=pb.PARD_MAX_DELAY_WINDOW_US + 1) == pb.PARD_ERANGE
+    assert call(t=a + 4) == pb.PARD_EINVAL                 # misaligned timestamps
+    assert call() == pb.PARD_EINVAL                        # no workspace
+    assert call(ws=a + 256 - a % 256, wsb=8) == pb.PARD_EWORKSPACE

@@ -68,6 +68,9 @@ def lib():
         _lib.oracle_queue_delay.restype = C.c_int
         _lib.oracle_queue_delay.argtypes = [C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_uint32, C.c_uint32, C.c_void_p]
+        _lib.oracle_advance_state.restype = C.c_int
+        _lib.oracle_advance_state.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint32, C.c_int32] + \
+            [C.c_void_p] * 7 + [C.c_uint32, C.c_uint32]
     return _lib
 
 
@@ -168,6 +171,27 @@ def queue_delay(now_us, sample_time_us, sample_delay_us, window_us: int) -> np.n
     if rc != 0:
         raise ValueError("oracle_queue_delay: bad input")
     return q
+
+
+def advance_state(pipelines, pipeline_of_ctx, n_ctx: int, stage_stride: int, now_us, batch, workers, seg_kept,
+                  free_at_us, sample_time_us, sample_delay_us, slot: int) -> None:
+    """In place: free_at_us (int64 [n_ctx, S]) and slot `slot` of the sample rings (int64 / int32
+    [n_ctx, S, M]; pass None, None to keep no samples)."""
+    k = _Keep()
+    cps = (_Pipeline * len(pipelines))(*[_c_pipeline(p, k) for p in pipelines])
+    assert free_at_us.dtype == np.int64 and free_at_us.flags.c_contiguous
+    M = 0
+    if sample_time_us is not None:
+        assert sample_time_us.dtype == np.int64 and sample_delay_us.dtype == np.int32
+        assert sample_time_us.flags.c_contiguous and sample_delay_us.flags.c_contiguous
+        M = int(sample_time_us.shape[2])
+    rc = lib().oracle_advance_state(C.addressof(cps), len(pipelines), k.add(pipeline_of_ctx, np.int32), n_ctx,
+                                    stage_stride, k.add(now_us, np.int64), k.add(batch, np.int32),
+                                    k.add(workers, np.int32), k.add(seg_kept, np.uint32), free_at_us.ctypes.data,
+                                    None if M == 0 else sample_time_us.ctypes.data,
+                                    None if M == 0 else sample_delay_us.ctypes.data, M, slot)
+    if rc != 0:
+        raise ValueError("oracle_advance_state: bad input")
 
 
 def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:

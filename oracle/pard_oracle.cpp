@@ -346,3 +346,35 @@ extern "C" int oracle_queue_delay(uint32_t n_ctx, int32_t stage_stride, const in
   }
   return 0;
 }
+
+extern "C" int oracle_advance_state(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                                    const int32_t* pipeline_of_ctx, uint32_t n_ctx, int32_t stage_stride,
+                                    const int64_t* now_us, const int32_t* batch, const int32_t* workers,
+                                    const uint32_t* seg_kept, int64_t* free_at_us,
+                                    int64_t* sample_time_us, int32_t* sample_delay_us,
+                                    uint32_t n_samples, uint32_t slot) {
+  if (n_samples > 0 && slot >= n_samples) return -1;
+  for (uint32_t c = 0; c < n_ctx; ++c) {
+    int32_t pi = pipeline_of_ctx ? pipeline_of_ctx[c] : 0;
+    if (pi < 0 || pi >= n_pipelines) return -1;
+    const oracle_pipeline_t* p = &pipelines[pi];
+    for (int32_t k = 0; k < p->n_stages; ++k) {
+      size_t seg = (size_t)c * stage_stride + k;
+      int32_t B = batch[seg];
+      if (B < 1 || B > p->bmax[k]) return -1;
+      int64_t m = workers ? workers[seg] : 1;
+      if (m < 1) return -1;
+      int64_t cap = (int64_t)B * m;
+      int64_t d = profile_at(p, k, B);
+      int64_t base = std::max(now_us[c], free_at_us[seg]);        /* t_e of the next batch */
+      if (n_samples > 0) {
+        int64_t delay = base - now_us[c];                           /* queueing delay met at `now` */
+        sample_time_us[seg * n_samples + slot] = now_us[c];
+        sample_delay_us[seg * n_samples + slot] = (int32_t)std::min<int64_t>(delay, (1 << 24) - 1);
+      }
+      int64_t rounds = ((int64_t)seg_kept[seg] + cap - 1) / cap;    /* batches run back to back */
+      free_at_us[seg] = base + rounds * d;
+    }
+  }
+  return 0;
+}

@@ -140,6 +140,25 @@ int oracle_queue_delay(uint32_t n_ctx, int32_t stage_stride, const int64_t* now_
                        const int64_t* sample_time_us, const int32_t* sample_delay_us,
                        uint32_t n_samples, uint32_t window_us, int64_t* q_us);
 
+/* Carries the queue state from one decision epoch to the next (closed loop:
+ * what the planner admitted is what the workers will run).  For every (ctx,
+ * stage k of its pipeline), with base = max(now, free_at_k) the start of the
+ * next batch as the planner saw it (Sec. 4.2: t_e, the expected end of the
+ * previous batch):
+ *   - the queueing delay a request dequeued at `now` meets, base - now
+ *     (capped at 2^24 - 1), is recorded with time `now` in slot `slot` of the
+ *     stage's sample ring (the samples oracle_queue_delay averages);
+ *   - the seg_kept[ctx * stage_stride + k] admitted requests run back to back
+ *     in rounds of B_k * m_k, each round d_k(B_k) long, so
+ *     free_at_k = base + ceil(kept / (B_k * m_k)) * d_k(B_k).
+ * Columns of stages the pipeline lacks are left untouched.  Returns 0 or -1. */
+int oracle_advance_state(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                         const int32_t* pipeline_of_ctx, uint32_t n_ctx, int32_t stage_stride,
+                         const int64_t* now_us, const int32_t* batch, const int32_t* workers,
+                         const uint32_t* seg_kept, int64_t* free_at_us,
+                         int64_t* sample_time_us, int32_t* sample_delay_us,
+                         uint32_t n_samples, uint32_t slot);
+
 #ifdef __cplusplus
 }
 #endif

@@ -89,3 +89,56 @@ def random_small_workload(rng, n, n_ctx=1, max_stages=5, keepish=True):
     r = requests(now[rng.integers(0, n_ctx, size=n)] * 0 + rng.integers(900, 2000 + span * S, size=n),
                  stage=rng.integers(0, S, size=n), ctx=rng.integers(0, n_ctx, size=n))
     return inputs.Workload("rand", [p], r, st, n_ctx)
+
+
+# --------------------------------------------------------------------------
+# closed-loop replay: a job (inputs only) and the loop composed of oracle calls
+# --------------------------------------------------------------------------
+def small_replay_job(rng, n_inst, n_epochs, per_epoch, n_samples=8, window_us=200_000):
+    """n_inst independent pipeline instances (one ctx each) observed over
+    n_epochs decision epochs; every epoch brings per_epoch new requests spread
+    over the instances and stages.  Durations are sized so that some stages are
+    overloaded and start dropping after a few epochs."""
+    S = 3
+    tables = [rng.integers(200, 900, size=4).astype(np.int64) for _ in range(S)]
+    p = inputs.make_pipeline(inputs.chain_edges(S), S, [4] * S, tables)
+    R = max(1, inputs.n_slots(p))
+    epoch_len = 20_000
+    now0 = 1_000_000
+    batch = rng.integers(1, 5, size=(n_inst, S)).astype(np.int32)
+    workers = rng.integers(1, 3, size=(n_inst, S)).astype(np.int32)
+    epochs = []
+    for e in range(n_epochs):
+        now = np.full(n_inst, now0 + e * epoch_len, np.int64) + rng.integers(0, 50, size=n_inst)
+        ctx = rng.integers(0, n_inst, size=per_epoch)
+        r = requests(now[ctx] + rng.integers(-2000, 40_000, size=per_epoch),
+                     stage=rng.integers(0, S, size=per_epoch), ctx=ctx)
+        epochs.append((now, r))
+    return {"pipelines": [p], "pipeline_of_ctx": None, "n_ctx": n_inst, "S": S, "R": R, "batch": batch,
+            "workers": workers, "free_at0": np.full((n_inst, S), now0 - 5, np.int64),
+            "w": rng.integers(0, 300, size=(n_inst, R)).astype(np.int64), "epochs": epochs,
+            "n_samples": n_samples, "window_us": window_us, "priority": None}
+
+
+def replay_with_oracle(job):
+    """The closed loop, one epoch after the other, composed of oracle calls only:
+    q from the recorded delays, the plan, then the state carried forward."""
+    from oracle import oracle
+    n_ctx, S, M = job["n_ctx"], job["S"], job["n_samples"]
+    free_at = job["free_at0"].copy()
+    t = np.full((n_ctx, S, M), -1, np.int64)
+    d = np.zeros((n_ctx, S, M), np.int32)
+    total, kept, fa_series, q_series = [], [], [], []
+    for e, (now, req) in enumerate(job["epochs"]):
+        q = oracle.queue_delay(now, t, d, job["window_us"])
+        st = inputs.QueueState(S, job["R"], now, job["batch"], free_at.copy(), q, job["w"], job["workers"],
+                               job["pipeline_of_ctx"], job["priority"])
+        o = oracle.plan(job["pipelines"], req, st, n_ctx)
+        oracle.advance_state(job["pipelines"], job["pipeline_of_ctx"], n_ctx, S, now, job["batch"],
+                             job["workers"], o["seg_kept"], free_at, t, d, e % M)
+        total.append(o["ctx_total"])
+        kept.append(o["ctx_kept"])
+        fa_series.append(free_at.copy())
+        q_series.append(q)
+    return {"total": np.array(total), "kept": np.array(kept), "free_at_series": np.array(fa_series),
+            "q_series": np.array(q_series), "free_at": free_at, "sample_time": t, "sample_delay": d}

@@ -336,6 +336,36 @@ int pard_update_queue_delay(uint32_t n_ctx, int32_t stage_stride, const int64_t*
                             int64_t* d_q_us, void* d_workspace, uint64_t workspace_bytes,
                             void* cuda_stream);
 
+/* Carries the queue state from one decision epoch to the next, for replaying a
+ * workload in closed loop: what pard_plan admitted is what the workers will
+ * run.  (The paper's system measures this state on live workers, Sec. 4.1
+ * step 1; a replay has to derive it, and does so with the planner's own model
+ * of Sec. 4.2: t_e is the expected end of the previous batch, and batches run
+ * back to back.)  For every (ctx, stage k of its pipeline), with
+ * base = max(now, free_at_k):
+ *   - the queueing delay met by a request dequeued at `now`, base - now (capped
+ *     at PARD_WAIT_LIMIT_US - 1), is stored with time `now` in slot `slot` of
+ *     the stage's sample ring, the arrays pard_update_queue_delay reads
+ *     ([n_ctx][stage_stride][n_samples]; n_samples = 0 keeps no samples);
+ *   - free_at_k = base + ceil(kept / (B_k * m_k)) * d_k(B_k), with kept =
+ *     d_seg_kept[ctx * stage_stride + k] as written by pard_plan.
+ * d_free_at_us is read and written in place; columns of stages the ctx's
+ * pipeline lacks are left untouched.  All arrays are DEVICE memory laid out as
+ * in pard_queue_state_t (d_workers NULL => 1).  d_workspace: 256-byte aligned,
+ * pard_advance_state_workspace_bytes().  mode: 0 or PARD_MODE_NOWAIT.
+ * Host-detectable errors come back before anything is launched; a batch size,
+ * worker count or time out of range (also a new free_at beyond
+ * PARD_TIME_LIMIT_US) gives PARD_EDATA.  One kernel is enqueued; nothing is
+ * allocated. */
+int pard_advance_state_workspace_bytes(uint32_t n_pipelines, uint64_t* bytes);
+int pard_advance_state(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+                       const int32_t* d_pipeline_of_ctx, uint32_t n_ctx, int32_t stage_stride,
+                       const int64_t* d_now_us, const int32_t* d_batch, const int32_t* d_workers,
+                       const uint32_t* d_seg_kept, int64_t* d_free_at_us,
+                       int64_t* d_sample_time_us, int32_t* d_sample_delay_us,
+                       uint32_t n_samples, uint32_t slot, uint32_t mode,
+                       void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+
 /* Adaptive request priority with delayed transition (Sec. 4.3): chooses, for
  * every (ctx, stage) queue, the decision order that pard_plan reads from
  * pard_queue_state_t.d_priority.  With

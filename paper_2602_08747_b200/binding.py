@@ -38,7 +38,8 @@ EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pi
            "pard_plan_kernel_launches", "pard_profile_begin", "pard_profile_end",
            "pard_profile_phase_name", "pard_plan_static", "pard_estimate_w_workspace_bytes",
            "pard_estimate_w", "pard_update_priority_workspace_bytes", "pard_update_priority",
-           "pard_update_queue_delay_workspace_bytes", "pard_update_queue_delay"]
+           "pard_update_queue_delay_workspace_bytes", "pard_update_queue_delay",
+           "pard_advance_state_workspace_bytes", "pard_advance_state"]
 
 
 class PardError(RuntimeError):
@@ -110,6 +111,9 @@ def library() -> C.CDLL:
         lib.pard_update_queue_delay.argtypes = [C.c_uint32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                                 C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
                                                 C.c_uint64, C.c_void_p]
+        lib.pard_advance_state_workspace_bytes.argtypes = [C.c_uint32, C.c_void_p]
+        lib.pard_advance_state.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_int32] + \
+            [C.c_void_p] * 7 + [C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p, C.c_uint64, C.c_void_p]
         lib.pard_profile_begin.argtypes = [C.c_uint32, C.c_uint32]
         lib.pard_profile_end.argtypes = [C.c_void_p, C.c_void_p]
         lib.pard_profile_phase_name.restype = C.c_char_p
@@ -387,6 +391,27 @@ def pard_update_queue_delay(n_ctx: int, stage_stride: int, d_now_us, d_sample_ti
                                            _ptr(d_workspace), wb, stream or None)
     if check:
         _check(rc, "pard_update_queue_delay")
+    return rc
+
+
+def pard_advance_state_workspace_bytes(n_pipelines: int) -> int:
+    b = C.c_uint64()
+    _check(library().pard_advance_state_workspace_bytes(n_pipelines, C.byref(b)), "pard_advance_state_workspace_bytes")
+    return b.value
+
+
+def pard_advance_state(pipelines: Sequence[Pipeline], d_pipeline_of_ctx, n_ctx: int, stage_stride: int, d_now_us,
+                       d_batch, d_workers, d_seg_kept, d_free_at_us, d_sample_time_us, d_sample_delay_us,
+                       n_samples: int, slot: int, mode: int, d_workspace, workspace_bytes: Optional[int] = None,
+                       stream: int = 0, check: bool = True) -> int:
+    hs = _handles(pipelines)
+    wb = workspace_bytes if workspace_bytes is not None else d_workspace.numel() * d_workspace.element_size()
+    rc = library().pard_advance_state(hs, len(pipelines), _ptr(d_pipeline_of_ctx), n_ctx, stage_stride,
+                                      _ptr(d_now_us), _ptr(d_batch), _ptr(d_workers), _ptr(d_seg_kept),
+                                      _ptr(d_free_at_us), _ptr(d_sample_time_us), _ptr(d_sample_delay_us),
+                                      n_samples, slot, mode, _ptr(d_workspace), wb, stream or None)
+    if check:
+        _check(rc, "pard_advance_state")
     return rc
 
 

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpard.so")
 SOURCES = ["pard_pipeline.cu", "pard_plan.cu", "pard_goodput.cu", "pard_host.cu",
-           "pard_static.cu", "pard_wait.cu", "pard_priority.cu", "pard_qdelay.cu"]
+           "pard_static.cu", "pard_wait.cu", "pard_priority.cu", "pard_qdelay.cu", "pard_replay.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
 

@@ -250,3 +250,33 @@ def test_update_queue_delay_argument_checks_happen_before_any_launch():
     assert call(t=a + 4) == pb.PARD_EINVAL                 # misaligned timestamps
     assert call() == pb.PARD_EINVAL                        # no workspace
     assert call(ws=a + 256 - a % 256, wsb=8) == pb.PARD_EWORKSPACE
+
+
+def test_advance_state_argument_checks_happen_before_any_launch():
+    p = inputs.make_pipeline(inputs.chain_edges(2), 2, [1, 1], [[5], [5]])
+    h = pb.pard_load_pipeline(p, host_only=True)
+    lib = pb.library()
+    v = C.c_uint64()
+    assert lib.pard_advance_state_workspace_bytes(0, C.byref(v)) == pb.PARD_EINVAL
+    assert lib.pard_advance_state_workspace_bytes(2, C.byref(v)) == pb.PARD_OK and v.value >= 256 + 16
+    hs = (C.c_void_p * 1)(h.handle)
+    a = np.zeros(64, np.int64).ctypes.data
+
+    def call(pipes=hs, n_pipes=1, poc=None, n_ctx=1, S=2, now=a, batch=a, workers=None, kept=a, fa=a, t=a, d=a,
+             M=4, slot=0, mode=0):
+        return lib.pard_advance_state(pipes, n_pipes, poc, n_ctx, S, now, batch, workers, kept, fa, t, d, M, slot,
+                                      mode, None, 0, None)
+
+    assert call(pipes=None) == pb.PARD_EINVAL
+    assert call(now=None) == pb.PARD_EINVAL
+    assert call(batch=None) == pb.PARD_EINVAL
+    assert call(kept=None) == pb.PARD_EINVAL
+    assert call(fa=None) == pb.PARD_EINVAL
+    assert call(t=None) == pb.PARD_EINVAL                  # a ring is announced but missing
+    assert call(slot=4) == pb.PARD_EINVAL
+    assert call(n_ctx=0) == pb.PARD_EINVAL
+    assert call(mode=pb.PARD_MODE_SCAN) == pb.PARD_EINVAL
+    assert call(n_pipes=2) == pb.PARD_EINVAL
+    assert call(S=65) == pb.PARD_ERANGE
+    assert call(M=pb.PARD_MAX_DELAY_SAMPLES + 1, slot=0) == pb.PARD_ERANGE
+    h.free()

@@ -310,6 +310,150 @@ def run_e2e(wl, dev, steps, dist):
     return sec, h2d, d2h
 
 
+
+def run_aux(dev, peak):
+    """Device time of the State Planner's input kernels and of the planner with
+    mixed priorities, on seeded synthetic inputs larger than the L2 where a
+    bandwidth figure is given.  CUDA events, 3 warm-ups, 10 timed calls."""
+    import torch
+    from paper_2602_08747_b200 import binding as pb
+    from paper_2602_08747_b200 import replay as rp
+    stream = torch.cuda.current_stream().cuda_stream
+    out = {}
+
+    def timed(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 1e3 / reps
+
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    # the 256 random DAG instances of the what-if sweep carry the per-queue state
+    wl = inputs.make("C5b", n_inst=256, per_inst=256)
+    st = wl.state
+    S, R, n_ctx = st.stage_stride, st.slot_stride, wl.n_ctx
+    pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
+    ds = pb.device_state(st, dev)
+    n_slots = int(sum(inputs.n_slots(wl.pipelines[int(c)]) for c in st.pipeline_of_ctx))
+    path_stages = int(sum(sum(len(pth) for pth in _paths(wl.pipelines[int(c)])) for c in st.pipeline_of_ctx))
+
+    # batch-wait estimate: M = 10,000 samples per (stage, downstream path) slot (Sec. 4.2)
+    M = 10_000
+    samples = torch.randint(0, 8000, (n_ctx, S, M), dtype=torch.int32, device=dev, generator=g)
+    d_w = torch.zeros((n_ctx, R), dtype=torch.int64, device=dev)
+    ws = pb.alloc_workspace(pb.pard_estimate_w_workspace_bytes(len(pipes)), dev)
+    sec = timed(lambda: pb.pard_estimate_w(pipes, ds.pipeline_of_ctx, n_ctx, S, R, samples, M, 1, 10, 5,
+                                           pb.PARD_MODE_NOWAIT, d_w, ws, stream=stream))
+    assert pb.pard_plan_status(ws, stream) == 0
+    out["pard_estimate_w"] = {"workload": "256 random DAG instances, M=10000, lambda=0.1", "slots": n_slots,
+                              "ms": 1e3 * sec, "slots_per_s": n_slots / sec, "draws_per_s": path_stages * M / sec,
+                              "algorithmic_gbs": 4.0 * path_stages * M / sec / 1e9, "bound": "alu/shared memory"}
+    del samples
+
+    # priority update: 2,048 workload samples per queue
+    H, W = 2048, 5
+    x = torch.randint(0, 4000, (n_ctx * 16, S, H), dtype=torch.int32, device=dev, generator=g)
+    big_ctx = n_ctx * 16
+    poc = ds.pipeline_of_ctx.repeat(16)
+    batch, workers = ds.batch.repeat(16, 1), ds.workers.repeat(16, 1)
+    prio = torch.zeros((big_ctx, S), dtype=torch.uint8, device=dev)
+    ws = pb.alloc_workspace(pb.pard_update_priority_workspace_bytes(len(pipes)), dev)
+    sec = timed(lambda: pb.pard_update_priority(pipes, poc, big_ctx, S, batch, workers, x, H, W, 1_000_000,
+                                                pb.PARD_MODE_NOWAIT, prio, ws, stream=stream))
+    assert pb.pard_plan_status(ws, stream) == 0
+    queues = int(sum(wl.pipelines[int(c)].n_stages for c in st.pipeline_of_ctx)) * 16
+    gbs = 4.0 * H * queues / sec / 1e9
+    out["pard_update_priority"] = {"workload": "%d queues x %d samples, window %d" % (queues, H, W), "ms": 1e3 * sec,
+                                   "queues_per_s": queues / sec, "algorithmic_gbs": gbs, "frac": gbs / peak,
+                                   "bound": "hbm"}
+    del x
+
+    # queueing-delay window: 2,048 samples per queue
+    Mq = 2048
+    now = torch.full((big_ctx,), 10**9, dtype=torch.int64, device=dev)
+    t = now[:, None, None] - torch.randint(0, 8_000_000, (big_ctx, S, Mq), dtype=torch.int64, device=dev, generator=g)
+    dly = torch.randint(0, 1 << 20, (big_ctx, S, Mq), dtype=torch.int32, device=dev, generator=g)
+    q = torch.zeros((big_ctx, S), dtype=torch.int64, device=dev)
+    ws = pb.alloc_workspace(pb.pard_update_queue_delay_workspace_bytes(), dev)
+    sec = timed(lambda: pb.pard_update_queue_delay(big_ctx, S, now, t, dly, Mq, 5_000_000, pb.PARD_MODE_NOWAIT, q, ws,
+                                                   stream=stream))
+    assert pb.pard_plan_status(ws, stream) == 0
+    rows = big_ctx * S
+    gbs = 12.0 * Mq * rows / sec / 1e9
+    out["pard_update_queue_delay"] = {"workload": "%d rows x %d samples, window 5 s" % (rows, Mq), "ms": 1e3 * sec,
+                                      "rows_per_s": rows / sec, "algorithmic_gbs": gbs, "frac": gbs / peak,
+                                      "bound": "hbm"}
+    del t, dly
+    for p in pipes:
+        p.free()
+
+    # the planner with every second queue served high budget first
+    wlh = inputs.make(WORKLOAD + "b", seed=2)
+    rng = np.random.default_rng(3)
+    wlh.state.priority = rng.integers(0, 2, size=(wlh.n_ctx, wlh.state.stage_stride)).astype(np.uint8)
+    plan = DevicePlan(wlh, dev)
+    sec, _ = timed_steps(plan, 40, 5, None)
+    out["pard_plan_mixed_priority"] = {"workload": WORKLOAD + "b, priorities drawn per queue", "ms": 1e3 * sec / 40,
+                                       "requests_per_s": wlh.n * 40 / sec}
+    del plan
+
+    # closed-loop replay: 16 instances, 64 epochs of 65,536 requests
+    job_rng = np.random.default_rng(11)
+    inst, n_ep, per = 16, 64, 65536
+    wl5 = inputs.make("C5b", n_inst=inst, per_inst=per)
+    st5 = wl5.state
+    pipes = [pb.pard_load_pipeline(p) for p in wl5.pipelines]
+    epochs = []
+    for e in range(n_ep):
+        r = wl5.requests.copy()
+        r["deadline_us"] += e * 200_000 + job_rng.integers(0, 2000, size=r.shape[0])
+        epochs.append((st5.now_us + e * 200_000, r))
+    R5 = rp.Replay(pipes, st5.pipeline_of_ctx, inst, st5.stage_stride, st5.slot_stride, st5.batch, st5.workers,
+                   st5.free_at_us, st5.w_us, None, 64, 5_000_000, wl5.n, dev)
+    d_now = torch.from_numpy(np.stack([e[0] for e in epochs])).to(dev)
+    d_req = [pb.device_requests(e[1], dev) for e in epochs]
+    total = torch.zeros((n_ep, inst), dtype=torch.int64, device=dev)
+    kept = torch.zeros((n_ep, inst), dtype=torch.int64, device=dev)
+
+    def one_replay():
+        for i in range(n_ep):
+            R5.step(d_now[i], d_req[i], wl5.n, total[i], kept[i])
+
+    sec = timed(one_replay, reps=3)
+    assert R5.statuses() == 0
+    out["replay"] = {"workload": "%d instances, %d epochs x %d requests" % (inst, n_ep, wl5.n), "ms_per_epoch": 1e3 * sec / n_ep,
+                     "epochs_per_s": n_ep / sec, "requests_per_s": wl5.n * n_ep / sec,
+                     "kept_fraction_last_run": float(kept.sum().item()) / float(max(1, total.sum().item()))}
+    for p in pipes:
+        p.free()
+    return out
+
+
+def _paths(p):
+    """Downstream paths of every stage of a pipeline (input structure only), for counting."""
+    out = []
+
+    def rec(k, prefix):
+        prefix = prefix + (int(k),)
+        succ = [int(j) for j in p.successors(k)]
+        if not succ:
+            out.append(prefix)
+        for j in succ:
+            rec(j, prefix)
+
+    for k in range(p.n_stages):
+        for j in p.successors(k):
+            rec(j, ())
+    return out
+
+
 def run_ours(args):
     import torch
     from paper_2602_08747_b200 import build as pbuild
@@ -385,6 +529,7 @@ def run_ours(args):
                                         "keep_fraction": kf,
                                         "kernels": kernel_table(prof2, wlb.n, kf, peak, prof2c)}
             del pl2
+        aux = {} if args.no_variants else run_aux(dev, peak)
         t_cpu, _ = time_oracle(wl, 2)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -405,6 +550,7 @@ def run_ours(args):
                              "sample": "the full %s snapshot (%d requests), best of 2 runs" % (WORKLOAD, wl.n),
                              "host_cores": os.cpu_count()},
             "variants": variants,
+            "state_planner_kernels": aux,
         }
         print(json.dumps(line))
     if dist is not None:

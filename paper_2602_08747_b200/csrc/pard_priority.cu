@@ -3,8 +3,8 @@
  * [1 - eps, 1 + eps], eps = sum |T_in - T_s| / sum T_in with T_s the input
  * workload smoothed by a sliding-window average.
  *
- * One warp per queue.  The lanes walk the queue's workload samples 32 at a
- * time; the window sum of sample j is the difference of two running prefix
+ * One warp per queue.  The lanes walk the queue's workload samples 256 at a
+ * time, eight consecutive ones per lane; the window sum of sample j is the difference of two running prefix
  * sums, one over the samples and one over the samples that have left the
  * window (the same row read `window` places back), so the work is linear in
  * the history length for any window.  All quantities are integers; the two
@@ -62,30 +62,55 @@ k_update_priority(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipel
   const unsigned long long d = (unsigned long long)p->lat_us[p->lat_offsets[k] + B - 1];
   const unsigned long long cap = (unsigned long long)B * (unsigned long long)m;   /* T_m = cap / d */
 
-  /* sums over the samples j >= W - 1:  sum_x = sum x_j,  dev = sum |W * x_j - (x_{j-W+1} + ... + x_j)| */
+  /* sums over the samples j >= W - 1:  sum_x = sum x_j,  dev = sum |W * x_j - (x_{j-W+1} + ... + x_j)|.
+   * A lane owns kRun consecutive samples of every chunk of 32 * kRun: running sums inside the
+   * lane, one warp scan of the lanes' totals per chunk. */
+  constexpr uint32_t kRun = 8;
   const uint32_t* x = arrivals + (size_t)seg * H;
+  const bool vec = (((uintptr_t)x) & 15) == 0;                         /* 16-byte loads of the own samples */
   unsigned long long carry_in = 0, carry_out = 0, sum_x = 0, dev = 0;
   bool bad = false;
-  for (uint32_t j0 = 0; j0 < H; j0 += 32) {
-    const uint32_t j = j0 + lane;
-    const uint32_t xj = j < H ? __ldg(&x[j]) : 0u;
-    const uint32_t xo = (j >= W && j < H) ? __ldg(&x[j - W]) : 0u;     /* the sample that left the window */
-    bad |= xj >= PARD_RATE_LIMIT;
-    unsigned long long pin = xj, pout = xo;                            /* inclusive prefix sums over the lanes */
+  for (uint32_t j0 = 0; j0 < H; j0 += 32 * kRun) {
+    const uint32_t jl = j0 + lane * kRun;                              /* first sample of this lane */
+    uint32_t xin[kRun], xout[kRun];
+    if (vec && jl + kRun <= H) {
+      const uint4 a = __ldg(reinterpret_cast<const uint4*>(x + jl));
+      const uint4 b = __ldg(reinterpret_cast<const uint4*>(x + jl + 4));
+      xin[0] = a.x; xin[1] = a.y; xin[2] = a.z; xin[3] = a.w;
+      xin[4] = b.x; xin[5] = b.y; xin[6] = b.z; xin[7] = b.w;
+    } else {
+#pragma unroll
+      for (uint32_t i = 0; i < kRun; ++i) xin[i] = jl + i < H ? __ldg(&x[jl + i]) : 0u;
+    }
+    unsigned long long tin = 0, tout = 0;
+#pragma unroll
+    for (uint32_t i = 0; i < kRun; ++i) {
+      const uint32_t j = jl + i;
+      xout[i] = (j >= W && j < H) ? __ldg(&x[j - W]) : 0u;             /* the sample that left the window */
+      bad |= xin[i] >= PARD_RATE_LIMIT;
+      tin += xin[i];
+      tout += xout[i];
+    }
+    unsigned long long pin = tin, pout = tout;                         /* inclusive over the lanes' totals */
     for (int o = 1; o < 32; o <<= 1) {
       const unsigned long long a = __shfl_up_sync(0xffffffffu, pin, o);
       const unsigned long long b = __shfl_up_sync(0xffffffffu, pout, o);
       if (lane >= (uint32_t)o) { pin += a; pout += b; }
     }
-    pin += carry_in;
-    pout += carry_out;
-    if (j + 1 >= W && j < H) {
-      const unsigned long long win = pin - pout, wx = (unsigned long long)W * xj;
-      dev += wx > win ? wx - win : win - wx;
-      sum_x += xj;
+    unsigned long long run_in = carry_in + pin - tin, run_out = carry_out + pout - tout;   /* before this lane */
+#pragma unroll
+    for (uint32_t i = 0; i < kRun; ++i) {
+      const uint32_t j = jl + i;
+      run_in += xin[i];
+      run_out += xout[i];
+      if (j + 1 >= W && j < H) {
+        const unsigned long long win = run_in - run_out, wx = (unsigned long long)W * xin[i];
+        dev += wx > win ? wx - win : win - wx;
+        sum_x += xin[i];
+      }
     }
-    carry_in = __shfl_sync(0xffffffffu, pin, 31);
-    carry_out = __shfl_sync(0xffffffffu, pout, 31);
+    carry_in += __shfl_sync(0xffffffffu, pin, 31);
+    carry_out += __shfl_sync(0xffffffffu, pout, 31);
   }
   if (__any_sync(0xffffffffu, bad)) {
     if (lane == 0) atomicMax(&hdr->status, (uint32_t)(-PARD_EDATA));

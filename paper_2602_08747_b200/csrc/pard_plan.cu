@@ -56,14 +56,13 @@ struct PlanHeader {
   uint32_t aborted;           /* 1: a bounded wait ran out; the sort is incomplete and every later kernel returns */
   uint32_t big_total;         /* window-table entries that belong to long queues */
   uint32_t agg_done;          /* blocks of k_tile_agg that have stored their aggregates */
-  uint32_t dec_done;          /* blocks of k_decide that have stored their queues' kept counts */
-  uint32_t pad[64 - 13 - (kMaxPasses + 1)];
+  uint32_t pad[64 - 12 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
-  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, lookback, zero_end,
+  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, hist, lookback, zero_end,
       pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
@@ -96,7 +95,6 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.ctx_dmax = o;  o = al(o + 8ull * n_ctx);
   L.seg_off = o;   o = al(o + 4ull * (L.n_seg + 1));
   L.seg_kept = o;  o = al(o + 4ull * L.n_seg);
-  L.win_done = o;  o = al(o + 4ull * L.n_seg);
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
   L.lookback = o;  o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);   /* two arrays, used in turn */
   L.zero_end = o;
@@ -129,6 +127,19 @@ __device__ __forceinline__ void set_aborted(PlanHeader* hdr) {
   hdr->aborted = 1;
   __threadfence();
   atomicExch(&hdr->status, (uint32_t)(-PARD_ETIMEOUT));
+}
+
+/* True in every thread of exactly one block: the one whose arrival at `counter` is the last of
+ * the grid.  Every thread's earlier global writes are visible to that block afterwards. */
+__device__ __forceinline__ bool last_block_done(uint32_t* counter) {
+  __shared__ uint32_t s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  const bool last = s_last != 0;
+  if (last) __threadfence();
+  return last;
 }
 
 /* ------------------------------------------------------------------------ */
@@ -238,6 +249,14 @@ __global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
   }
 }
 
+/* The device tables of the call's pipelines: handed over inside the kernel arguments when they
+ * are few (no copy to enqueue), else through a table in the workspace. */
+constexpr int kFewPipelines = 8;
+struct PipeTable {
+  const PardPipeDev* few[kFewPipelines];
+  const PardPipeDev* const* many;
+};
+
 /* floor(2^64 / d) + 1 for d >= 2 */
 __device__ __forceinline__ unsigned long long magic64(unsigned long long d) {
   unsigned long long q = ~0ull / d;
@@ -249,7 +268,7 @@ __device__ __forceinline__ unsigned long long magic64(unsigned long long d) {
  * downstream paths (the path table of the pipeline lists, for every stage,
  * each stage sequence from a successor to a sink). */
 __global__ void __launch_bounds__(128)
-k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
+k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
             pard_queue_state_t st, uint32_t n_ctx,
             const unsigned long long* __restrict__ ctx_dmin_inv,
             const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
@@ -268,7 +287,7 @@ k_seg_const(const PardPipeDev* const* __restrict__ pipes, uint32_t n_pipelines,
   if (pi < 0 || (uint32_t)pi >= n_pipelines) {
     bad = true;
   } else {
-    const PardPipeDev* p = pipes[pi];
+    const PardPipeDev* p = n_pipelines <= (uint32_t)kFewPipelines ? pipes.few[pi] : pipes.many[pi];
     const int64_t* qrow = st.d_q_us + (size_t)c * S;
     const int32_t* brow = st.d_batch + (size_t)c * S;
     if (k >= (uint32_t)p->n_stages) {
@@ -815,19 +834,6 @@ __device__ void tile_scan_block(const unsigned long long* tile_agg, uint32_t n_t
   }
 }
 
-/* True in every thread of exactly one block: the one whose arrival at `counter` is the last of
- * the grid.  Every thread's earlier global writes are visible to that block afterwards. */
-__device__ __forceinline__ bool last_block_done(uint32_t* counter) {
-  __shared__ uint32_t s_last;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) s_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1u : 0u;
-  __syncthreads();
-  const bool last = s_last != 0;
-  if (last) __threadfence();
-  return last;
-}
-
 /* Tile aggregates: the segmented reduction over each tile of kDecTile sorted
  * elements.  Tiles are independent; the block that finishes last scans the
  * aggregates into the value carried into every tile, so that the decision
@@ -890,7 +896,7 @@ __device__ void kept_scan_block(const uint32_t* seg_kept, uint32_t n_seg, uint32
     uint32_t v[PER], c[PER], x = 0, y = 0;
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
-      v[k] = i0 + k < n_seg ? __ldcg(&seg_kept[i0 + k]) : 0;
+      v[k] = i0 + k < n_seg ? seg_kept[i0 + k] : 0;
       c[k] = (v[k] + kCompactChunk - 1) / kCompactChunk;
       if (out_seg_kept && i0 + k < n_seg) out_seg_kept[i0 + k] = v[k];
       x += v[k];
@@ -944,19 +950,12 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
          const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
          const uint32_t* __restrict__ win_off, const int32_t* __restrict__ carry,
          uint8_t* __restrict__ out_keep, long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
-         uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept, uint32_t n_seg,
-         uint32_t* __restrict__ kept_base, uint32_t* __restrict__ chunk_base,
-         uint32_t* __restrict__ out_seg_kept, unsigned long long* __restrict__ out_n_kept) {
+         uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept) {
   pdl_wait();
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide || hdr->aborted || !hdr->use_scan) {
-    /* the window-table kernel has decided (or nothing could be): only the scan of the queues'
-     * kept counts is left, and one block does it */
-    if (blockIdx.x == 0) kept_scan_block<kDecThreads>(seg_kept, n_seg, kept_base, chunk_base, out_seg_kept, out_n_kept);
-    return;
-  }
+  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
@@ -1091,8 +1090,14 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
   }
   __syncthreads();
   }
-  if (last_block_done(&const_cast<PlanHeader*>(hdr)->dec_done))
-    kept_scan_block<kDecThreads>(seg_kept, n_seg, kept_base, chunk_base, out_seg_kept, out_n_kept);
+}
+
+__global__ void __launch_bounds__(1024)
+k_kept_scan(const uint32_t* __restrict__ seg_kept, uint32_t n_seg, uint32_t* __restrict__ kept_base,
+            uint32_t* __restrict__ chunk_base, uint32_t* __restrict__ out_seg_kept,
+            unsigned long long* __restrict__ out_n_kept) {
+  pdl_wait();
+  kept_scan_block<1024>(seg_kept, n_seg, kept_base, chunk_base, out_seg_kept, out_n_kept);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -1234,8 +1239,8 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
   }
 }
 
-/* E and Kp of the table entries of one queue, once all their P are known: the warp runs over
- * the queue's windows, 32 at a time. */
+/* E and Kp of the table entries of one queue: the warp runs over the queue's windows, 32 at a
+ * time. */
 __device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* __restrict__ ktab,
                                                 const uint32_t* __restrict__ win_off,
                                                 const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab,
@@ -1244,7 +1249,7 @@ __device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* 
   if (cnt == 0) return;
   const uint32_t cap = ktab[s].cap;
   WinEntry* tab = wtab + w0;
-  const uint32_t P0 = __ldcg(&tab[0].P);
+  const uint32_t P0 = tab[0].P;
   int32_t e_carry = P0 > 0 ? -(int32_t)(P0 - 1) : kWinInf;     /* the expired run: u = 0 */
   uint32_t k_carry = 0;
   if (lane == 0) { tab[0].E = e_carry; tab[0].Kp = 0; }
@@ -1253,7 +1258,7 @@ __device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* 
     int32_t val = kWinInf;
     uint32_t kept = 0;
     if (b + 1 < cnt) {
-      const uint32_t p = __ldcg(&tab[b].P), q = __ldcg(&tab[b + 1].P);
+      const uint32_t p = tab[b].P, q = tab[b + 1].P;
       if (q > p) {
         const uint32_t u = win_u(b, cap);
         val = (int32_t)u - (int32_t)(q - 1);
@@ -1275,51 +1280,36 @@ __device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* 
 }
 
 /* The window tables.  P of every entry: a search in the queue's sorted elements, by one lane
- * (short queue) or by a whole warp with 32 probes per step (long queue).  Every finished entry
- * is counted per queue; the warp that finishes a queue's last entry goes on to the queue's
- * prefix pass (E, Kp), so the tables are complete when the kernel ends. */
+ * (short queue) or by a whole warp with 32 probes per step (long queue).  (Counting finished
+ * entries per queue so that the last finisher could run the queue's prefix pass in the same
+ * kernel was tried: the fence and the atomic per entry cost more than the launch they saved
+ * once there are thousands of queues.) */
 __global__ void __launch_bounds__(256)
 k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
              const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
-             const uint32_t* __restrict__ win_own, const uint32_t* __restrict__ win_big,
-             uint32_t* __restrict__ win_done, WinEntry* __restrict__ wtab) {
+             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_own,
+             const uint32_t* __restrict__ win_big, WinEntry* __restrict__ wtab) {
   pdl_wait();
   if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t lane = threadIdx.x & 31;
   const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
   const uint32_t dbits = hdr->dbits;
   const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
-  /* entries of short queues: one lane each, plain binary search; the warp stays together */
+  /* entries of short queues: one lane each, plain binary search */
   {
     const uint32_t total = hdr->win_total, step = gridDim.x * blockDim.x;
-    for (uint32_t e0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; e0 < total; e0 += step) {
-      const uint32_t e = e0 + lane;
-      uint32_t s = 0;
-      bool finished = false;
-      if (e < total) {
-        s = win_own[e];
-        uint32_t lo = seg_off[s], hi = seg_off[s + 1];
-        if (hi - lo <= kWinLongQueue) {
-          const uint32_t first = lo;
-          const long long thr = ktab[s].A_rel + (long long)(e - win_off[s]) * ktab[s].d;
-          while (lo < hi) {
-            const uint32_t mid = lo + (hi - lo) / 2;
-            if ((long long)((__ldg(src + mid) >> ibits) & dmask) < thr) lo = mid + 1; else hi = mid;
-          }
-          wtab[e].P = lo - first;
-          __threadfence();
-          finished = atomicAdd(&win_done[s], 1u) + 1 == win_cnt[s];
-        }
+    for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += step) {
+      const uint32_t s = win_own[e];
+      uint32_t lo = seg_off[s], hi = seg_off[s + 1];
+      if (hi - lo > kWinLongQueue) continue;
+      const uint32_t first = lo;
+      const long long thr = ktab[s].A_rel + (long long)(e - win_off[s]) * ktab[s].d;
+      while (lo < hi) {
+        const uint32_t mid = lo + (hi - lo) / 2;
+        if ((long long)((__ldg(src + mid) >> ibits) & dmask) < thr) lo = mid + 1; else hi = mid;
       }
-      uint32_t fin = __ballot_sync(0xffffffffu, finished);
-      if (fin) __threadfence();
-      while (fin) {                                  /* queues completed by this warp, one after the other */
-        const uint32_t sq = __shfl_sync(0xffffffffu, s, __ffs(fin) - 1);
-        win_prefix_warp(sq, ktab, win_off, win_cnt, wtab, lane);
-        fin &= fin - 1;
-      }
+      wtab[e].P = lo - first;
     }
   }
   /* entries of long queues: one warp each, 32 probes per step */
@@ -1341,17 +1331,20 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
       if (k > 0) lo = p_below + 1;
       if (k < 32) hi = p_at;
     }
-    uint32_t finished = 0;
-    if (lane == 0) {
-      wtab[e].P = lo - first;
-      __threadfence();
-      finished = atomicAdd(&win_done[s], 1u) + 1 == win_cnt[s] ? 1u : 0u;
-    }
-    if (__shfl_sync(0xffffffffu, finished, 0)) {
-      __threadfence();
-      win_prefix_warp(s, ktab, win_off, win_cnt, wtab, lane);
-    }
+    if (lane == 0) wtab[e].P = lo - first;
   }
+}
+
+/* E and Kp of every table entry: one warp per queue runs over its windows, 32 at a time. */
+__global__ void __launch_bounds__(256)
+k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
+             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
+             WinEntry* __restrict__ wtab) {
+  pdl_wait();
+  if (hdr->use_scan || hdr->wide || hdr->aborted) return;
+  const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (s >= n_seg) return;                          /* whole warps leave together */
+  win_prefix_warp(s, ktab, win_off, win_cnt, wtab, threadIdx.x & 31);
 }
 
 /* Decision pass from the window tables: every request on its own.  HF: some
@@ -1606,7 +1599,6 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   uint32_t* win_cnt = (uint32_t*)(ws + L.win_cnt);
   uint32_t* win_own = (uint32_t*)(ws + L.win_own);
   uint32_t* win_big = (uint32_t*)(ws + L.win_big);
-  uint32_t* win_done = (uint32_t*)(ws + L.win_done);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -1625,7 +1617,12 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   mark();
   /* ---- clear the scratch that must start at zero: one contiguous region ---- */
   PARD_CUDA_OK(cudaMemsetAsync(ws + L.hdr, 0, n > 0 ? L.zero_end : L.lookback, stream));
-  PARD_CUDA_OK(cudaMemcpyAsync(d_pipes, h_pipes.data(), 8ull * n_pipelines, cudaMemcpyHostToDevice, stream));
+  PipeTable pipe_table = {};
+  pipe_table.many = d_pipes;
+  if (n_pipelines <= (uint32_t)kFewPipelines)
+    for (uint32_t i = 0; i < n_pipelines; ++i) pipe_table.few[i] = h_pipes[i];
+  else
+    PARD_CUDA_OK(cudaMemcpyAsync(d_pipes, h_pipes.data(), 8ull * n_pipelines, cudaMemcpyHostToDevice, stream));
 
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -1641,7 +1638,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   mark();
   if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
   launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr);
-  launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, d_pipes, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab, hdr);
+  launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab, hdr);
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
@@ -1664,34 +1661,33 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     const bool raw = mode & PARD_MODE_RAW;
     /* window tables, and the decision from them */
     launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream, 
-        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_own, win_big, wtab);
+    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, win_off, win_cnt, wtab);
     mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
                           : (state->d_priority ? k_decide_win<false, true> : k_decide_win<false, false>);
     launch_pdl(decide_win, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, wtab,
                out->d_keep, est, out->d_perm, tmp, seg_kept);
-    /* fallback when a queue has too many batch windows: the same decision by scanning (the
-     * aggregate kernel returns at once otherwise) */
+    /* fallback when a queue has too many batch windows: the same decision by scanning (these two
+     * return at once otherwise) */
     const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3);
-    if (raw)
+    if (raw) {
       launch_pdl(k_tile_agg<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg,
                  tile_carry);
-    else
+      launch_pdl(k_decide<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
+                 tile_carry, out->d_keep, est, out->d_perm, tmp, seg_kept);
+    } else {
       launch_pdl(k_tile_agg<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg,
                  tile_carry);
+      launch_pdl(k_decide<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
+                 tile_carry, out->d_keep, est, out->d_perm, tmp, seg_kept);
+    }
   }
-  /* the scan path's decision kernel; whichever path decided, it ends with the scan of the queues'
-   * kept counts (first output slot of every queue, copy jobs, total) */
-  {
-    if (n == 0) mark();
-    const uint32_t scan_grid = std::max<uint32_t>(1u, std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3));
-    auto decide = (mode & PARD_MODE_RAW) ? k_decide<true> : k_decide<false>;
-    launch_pdl(decide, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, tile_carry,
-               out->d_keep, (long long*)out->d_est_us, out->d_perm, out->d_kept_idx ? kept_tmp : nullptr, seg_kept,
-               L.n_seg, kept_base, chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept);
-  }
+  if (n == 0) mark();
   mark();
+  launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+             (unsigned long long*)out->d_n_kept);
   if (n > 0 && out->d_kept_idx)
     launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
                                                (uint32_t)sms * 8), 256, 0, stream, 
@@ -1718,10 +1714,10 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* key_width, seg_const, seg_win and the scan path's decision kernel (which ends with the scan of
-   * the kept counts) always; prepass, ctx_span, pack, the passes, win_bounds, decide_win, tile_agg
-   * and kept_move (when the compacted indices are requested) when n > 0 */
-  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 4 : 4;
+  /* key_width, seg_const, seg_win and kept_scan always; prepass, ctx_span, pack, the passes,
+   * win_bounds, win_prefix, decide_win, tile_agg, decide and kept_move (when the compacted indices
+   * are requested) when n > 0 */
+  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 6 : 4;
   return PARD_OK;
 }
 

@@ -311,7 +311,7 @@ def run_e2e(wl, dev, steps, dist):
 
 
 
-def run_aux(dev, peak):
+def run_aux(dev, peak, kernels_only=False):
     """Device time of the State Planner's input kernels and of the planner with
     mixed priorities, on seeded synthetic inputs larger than the L2 where a
     bandwidth figure is given.  CUDA events, 3 warm-ups, 10 timed calls."""
@@ -393,6 +393,8 @@ def run_aux(dev, peak):
     del t, dly
     for p in pipes:
         p.free()
+    if kernels_only:
+        return out
 
     # the planner with every second queue served high budget first
     wlh = inputs.make(WORKLOAD + "b", seed=2)
@@ -471,6 +473,10 @@ def run_ours(args):
         dist_mod.init_process_group("nccl", device_id=torch.device(dev))
         dist = dist_mod
 
+    if args.only_aux:
+        peak, _ = measured_peaks()
+        print(json.dumps({"only_aux": True, "state_planner_kernels": run_aux(dev, peak, kernels_only=True)}))
+        return
     if args.only_device:
         kw = {"n": args.n} if args.n else {}
         wl = inputs.make(args.workload or WORKLOAD, **kw)
@@ -567,6 +573,9 @@ def main():
     ap.add_argument("--no-variants", action="store_true")
     ap.add_argument("--only-device", action="store_true",
                     help="run warm-up and timed steps of the device path only and print a short line "
+                         "(for use under a profiler; not a bench value)")
+    ap.add_argument("--only-aux", action="store_true",
+                    help="run only the State Planner kernels' timings and print them "
                          "(for use under a profiler; not a bench value)")
     ap.add_argument("--workload", default=None, help="with --only-device: another workload name, e.g. C3b")
     ap.add_argument("--n", type=int, default=None, help="with --only-device: number of requests")

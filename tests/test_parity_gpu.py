@@ -201,13 +201,14 @@ def test_workspace_too_small_and_foreign_handle():
 def test_host_buffer_entry_point_matches():
     import torch
     wl = inputs.make("C2b", n=150_001)
+    wl.state.priority = np.random.default_rng(5).integers(0, 2, size=(wl.n_ctx, wl.state.stage_stride)).astype(np.uint8)
     want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
     pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
     st = wl.state
     S, R = st.stage_stride, st.slot_stride
     n_seg = wl.n_ctx * S
     hs = pb.QueueStateArrays(S, R, st.now_us, st.batch, st.free_at_us, st.q_us, st.w_us, st.workers,
-                             st.pipeline_of_ctx)
+                             st.pipeline_of_ctx, st.priority)
     out = pb.PlanOut(np.zeros(wl.n, np.uint8), np.zeros(wl.n, np.int64), np.zeros(wl.n, np.uint32),
                      np.zeros(wl.n, np.uint32), np.zeros(1, np.uint64),
                      np.zeros(n_seg + 1, np.uint32), np.zeros(n_seg, np.uint32))

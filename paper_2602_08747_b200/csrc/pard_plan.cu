@@ -891,14 +891,30 @@ __device__ void kept_scan_block(const uint32_t* seg_kept, uint32_t n_seg, uint32
   if (threadIdx.x == 0) { s_ca = 0; s_cb = 0; }
   __syncthreads();
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  /* a thread's eight entries as two 16-byte accesses where the arrays allow it */
+  const bool vec_in = ((uintptr_t)seg_kept & 15) == 0;
+  const bool vec_out = (((uintptr_t)kept_base | (uintptr_t)chunk_base) & 15) == 0;
+  const bool vec_user = out_seg_kept && ((uintptr_t)out_seg_kept & 15) == 0;
   for (uint32_t base = 0; base < n_seg + 1; base += THREADS * PER) {
     const uint32_t i0 = base + threadIdx.x * PER;
     uint32_t v[PER], c[PER], x = 0, y = 0;
+    if (vec_in && i0 + PER <= n_seg) {
+      const uint4 a = *reinterpret_cast<const uint4*>(seg_kept + i0), b = *reinterpret_cast<const uint4*>(seg_kept + i0 + 4);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+#pragma unroll
+      for (int k = 0; k < PER; ++k) v[k] = i0 + k < n_seg ? seg_kept[i0 + k] : 0;
+    }
+    if (vec_user && i0 + PER <= n_seg) {
+      *reinterpret_cast<uint4*>(out_seg_kept + i0) = make_uint4(v[0], v[1], v[2], v[3]);
+      *reinterpret_cast<uint4*>(out_seg_kept + i0 + 4) = make_uint4(v[4], v[5], v[6], v[7]);
+    } else if (out_seg_kept) {
+#pragma unroll
+      for (int k = 0; k < PER; ++k) if (i0 + k < n_seg) out_seg_kept[i0 + k] = v[k];
+    }
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
-      v[k] = i0 + k < n_seg ? seg_kept[i0 + k] : 0;
       c[k] = (v[k] + kCompactChunk - 1) / kCompactChunk;
-      if (out_seg_kept && i0 + k < n_seg) out_seg_kept[i0 + k] = v[k];
       x += v[k];
       y += c[k];
     }
@@ -921,11 +937,21 @@ __device__ void kept_scan_block(const uint32_t* seg_kept, uint32_t n_seg, uint32
     }
     __syncthreads();
     uint32_t ea = s_ca + s_a[warp] + x - tx, eb = s_cb + s_b[warp] + y - ty;   /* exclusive, before this thread's queues */
+    uint32_t oa[PER], ob[PER];
 #pragma unroll
     for (int k = 0; k < PER; ++k) {
-      if (i0 + k <= n_seg) { kept_base[i0 + k] = ea; chunk_base[i0 + k] = eb; }
+      oa[k] = ea; ob[k] = eb;
       ea += v[k];
       eb += c[k];
+    }
+    if (vec_out && i0 + PER <= n_seg + 1) {
+      *reinterpret_cast<uint4*>(kept_base + i0) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+      *reinterpret_cast<uint4*>(kept_base + i0 + 4) = make_uint4(oa[4], oa[5], oa[6], oa[7]);
+      *reinterpret_cast<uint4*>(chunk_base + i0) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+      *reinterpret_cast<uint4*>(chunk_base + i0 + 4) = make_uint4(ob[4], ob[5], ob[6], ob[7]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < PER; ++k) if (i0 + k <= n_seg) { kept_base[i0 + k] = oa[k]; chunk_base[i0 + k] = ob[k]; }
     }
     __syncthreads();
     if (threadIdx.x == THREADS - 1) { s_ca = ea; s_cb = eb; }
@@ -1127,6 +1153,7 @@ struct __align__(16) WinEntry {
 };
 constexpr int32_t kWinInf = 0x7fffffff;
 constexpr uint32_t kWinMaxPerSeg = 4096;
+constexpr uint32_t kManyQueues = 8192;     /* from this many queues on a lane, not a warp, handles a queue in k_seg_win_many */
 constexpr uint32_t kWinLongQueue = 8192;   /* above this a window boundary is searched by a whole warp, else by one lane */
 
 
@@ -1236,6 +1263,84 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
     if (lane == 0) at = atomicAdd(&hdr->big_total, w);
     at = __shfl_sync(0xffffffffu, at, 0);
     for (uint32_t e = lane; e < w; e += 32) win_big[at + e] = first + e;
+  }
+}
+
+/* The same for calls with thousands of queues, where a warp per queue means more probes than a
+ * pass over the elements: here a LANE owns a queue.  Lane i of a warp finds the first element
+ * of queue s0 + i by a plain binary search (the lanes' early probes coincide, so they cost one
+ * sector), takes the end of its queue from lane i + 1, and the warp draws its queues' table
+ * entries from the shared counter with one addition. */
+__global__ void __launch_bounds__(256)
+k_seg_win_many(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
+               const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t n_seg,
+               const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
+               uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
+               uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
+               uint32_t force_scan) {
+  pdl_wait();
+  const uint32_t warp_g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t s0 = warp_g * 31u;              /* queues s0 .. s0+30, boundaries s0 .. s0+31 */
+  if (s0 > n_seg) return;                        /* whole warps leave together */
+  if (warp_g == 0 && lane == 0 && force_scan) hdr->use_scan = 1;
+  const uint32_t s = s0 + lane;
+  const bool wide = hdr->wide != 0 || hdr->aborted != 0;   /* nothing usable was sorted */
+  const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
+  const uint32_t dbits = hdr->dbits;
+  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  uint32_t lo = 0;                               /* first element whose segment id is >= s */
+  if (!wide && n > 0 && s <= n_seg) {
+    const uint32_t kshift = ibits + dbits;
+    uint32_t hi = n;
+    while (lo < hi) {
+      const uint32_t mid = lo + (hi - lo) / 2;
+      if ((uint32_t)(__ldg(src + mid) >> kshift) < s) lo = mid + 1; else hi = mid;
+    }
+  }
+  if (lane < 31 && s <= n_seg) {                 /* boundary s0+31 belongs to the next warp */
+    seg_off[s] = lo;
+    if (out_seg_off) out_seg_off[s] = lo;
+  }
+  const uint32_t end = __shfl_down_sync(0xffffffffu, lo, 1);
+  const bool mine = lane < 31 && s < n_seg;
+  uint32_t w = 0;
+  bool high_first = false;
+  if (mine && end > lo && !wide) {
+    const PardSegConst K = ktab[s];
+    if (K.narrow & kSegNoStage) {
+      set_status(hdr, PARD_EDATA);               /* requests queued at a stage the pipeline lacks */
+    } else if (K.narrow & kSegHighFirst) {       /* length of the kept prefix (see k_seg_win) */
+      high_first = true;
+      uint32_t a = lo, b = end;
+      while (a < b) {
+        const uint32_t mid = a + (b - a) / 2;
+        if (mid - lo < threshold_u(slack_of((__ldg(src + mid) >> ibits) & dmask, K), K)) a = mid + 1; else b = mid;
+      }
+      win_off[s] = a - lo;
+      win_cnt[s] = 0;
+    } else {
+      const long long X = (long long)((src[end - 1] >> ibits) & dmask) - K.A_rel;   /* latest deadline of the queue */
+      const unsigned long long nb = X < 0 ? 0 : win_of((unsigned long long)X, K) + 1;
+      if (nb >= kWinMaxPerSeg) hdr->use_scan = 1;
+      else w = (uint32_t)nb + 1;
+    }
+  }
+  uint32_t incl = w;                             /* the warp's queues take consecutive table entries */
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= (uint32_t)o) incl += t;
+  }
+  uint32_t base = 0;
+  if (lane == 31 && incl) base = atomicAdd(&hdr->win_total, incl);
+  base = __shfl_sync(0xffffffffu, base, 31);
+  uint32_t first = base + incl - w;
+  if (w && first + w > capacity) { hdr->use_scan = 1; w = 0; }
+  if (mine && !high_first) { win_off[s] = w ? first : 0u; win_cnt[s] = w; }
+  for (uint32_t e = 0; e < w; ++e) win_own[first + e] = s;
+  if (w && end - lo > kWinLongQueue) {           /* long queue: list its entries for the warp-wide search */
+    const uint32_t at = atomicAdd(&hdr->big_total, w);
+    for (uint32_t e = 0; e < w; ++e) win_big[at + e] = first + e;
   }
 }
 
@@ -1652,9 +1757,14 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
           n32, ibits, (p == 0 && (mode & PARD_MODE_TEST_STALL)) ? 1u : 0u);
   }
   mark();
-  launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
-                                                        out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-                                                        (mode & PARD_MODE_SCAN) ? 1u : 0u);
+  if (L.n_seg >= kManyQueues)
+    launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
+               seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
+               (mode & PARD_MODE_SCAN) ? 1u : 0u);
+  else
+    launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
+               out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
+               (mode & PARD_MODE_SCAN) ? 1u : 0u);
   if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
     long long* est = (long long*)out->d_est_us;

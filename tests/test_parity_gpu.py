@@ -34,6 +34,8 @@ def both(wl, mode=0):
     ("C3", {"n": 70_001}), ("C3b", {"n": 300_007}),
     ("C4", {"n_epochs": 37, "per_epoch": 1000}), ("C4b", {"n_epochs": 64, "per_epoch": 8192}),
     ("C5", {"n_inst": 9, "per_inst": 5001}), ("C5b", {"n_inst": 16, "per_inst": 65536}),
+    # thousands of queues: the lane-per-queue form of the segment search
+    ("C4b", {"n_epochs": 1100, "per_epoch": 200}), ("C5b", {"n_inst": 600, "per_inst": 301}),
 ])
 @pytest.mark.parametrize("mode", [0, 1])
 def test_configs_reduced(name, kw, mode):

@@ -36,6 +36,7 @@ def with_priority(wl, rng=None, value=None):
     ("C1", {}), ("C1b", {}), ("C1b", {"n": 12345}),
     ("C2b", {"n": 100_003}), ("C3b", {"n": 300_007}),
     ("C4b", {"n_epochs": 64, "per_epoch": 8192}), ("C5b", {"n_inst": 16, "per_inst": 65536}),
+    ("C4b", {"n_epochs": 1100, "per_epoch": 200}), ("C5b", {"n_inst": 600, "per_inst": 301}),
 ])
 @pytest.mark.parametrize("mode", [0, 1])
 def test_configs_reduced_with_mixed_priorities(name, kw, mode):

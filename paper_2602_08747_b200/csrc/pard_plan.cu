@@ -62,7 +62,7 @@ static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
-  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, hist, lookback, zero_end,
+  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, lookback, zero_end,
       pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
@@ -95,6 +95,7 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.ctx_dmax = o;  o = al(o + 8ull * n_ctx);
   L.seg_off = o;   o = al(o + 4ull * (L.n_seg + 1));
   L.seg_kept = o;  o = al(o + 4ull * L.n_seg);
+  L.win_done = o;  o = al(o + 4ull * L.n_seg);
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
   L.lookback = o;  o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);   /* two arrays, used in turn */
   L.zero_end = o;
@@ -1180,7 +1181,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
           const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
           uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
           uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
-          uint32_t force_scan) {
+          uint32_t force_scan, const uint32_t* __restrict__ hist, uint32_t sbits) {
   pdl_wait();
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1190,7 +1191,21 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
   const bool wide = hdr->wide != 0 || hdr->aborted != 0;   /* nothing usable was sorted */
   const unsigned long long* src = (hdr->npass & 1) ? buf_b : buf_a;
   const uint32_t dbits = hdr->dbits;
-  if (!wide && n > 0) {
+  const uint32_t npass = hdr->npass;
+  const uint32_t top_bits = npass ? hdr->keybits - 8 * (npass - 1) : 0;   /* width of the last pass's digit */
+  if (!wide && n > 0 && npass && sbits <= top_bits) {
+    /* the segment id is the upper part of the last pass's digit: the queue starts where the
+     * digits below (s << (top_bits - sbits)) end, and the digit counts of that pass are known */
+    const uint32_t* h = hist + (npass - 1) * kBins;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const uint32_t limit = min((s + q) << (top_bits - sbits), (uint32_t)kBins);
+      uint32_t sum = 0;
+      for (uint32_t d = lane; d < limit; d += 32) sum += h[d];
+      for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      lo[q] = sum;
+    }
+  } else if (!wide && n > 0) {
     const uint32_t kshift = ibits + dbits;
     uint32_t hi[2] = {n, n};                     /* answers: first element whose segment id is >= s, >= s+1 */
     while (lo[0] < hi[0] || lo[1] < hi[1]) {
@@ -1354,7 +1369,7 @@ __device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* 
   if (cnt == 0) return;
   const uint32_t cap = ktab[s].cap;
   WinEntry* tab = wtab + w0;
-  const uint32_t P0 = tab[0].P;
+  const uint32_t P0 = __ldcg(&tab[0].P);          /* other blocks may have written the P (long queues) */
   int32_t e_carry = P0 > 0 ? -(int32_t)(P0 - 1) : kWinInf;     /* the expired run: u = 0 */
   uint32_t k_carry = 0;
   if (lane == 0) { tab[0].E = e_carry; tab[0].Kp = 0; }
@@ -1363,7 +1378,7 @@ __device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* 
     int32_t val = kWinInf;
     uint32_t kept = 0;
     if (b + 1 < cnt) {
-      const uint32_t p = tab[b].P, q = tab[b + 1].P;
+      const uint32_t p = __ldcg(&tab[b].P), q = __ldcg(&tab[b + 1].P);
       if (q > p) {
         const uint32_t u = win_u(b, cap);
         val = (int32_t)u - (int32_t)(q - 1);
@@ -1393,8 +1408,9 @@ __global__ void __launch_bounds__(256)
 k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
              const unsigned long long* __restrict__ buf_b, uint32_t ibits, uint32_t n_seg,
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_own,
-             const uint32_t* __restrict__ win_big, WinEntry* __restrict__ wtab) {
+             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
+             const uint32_t* __restrict__ win_own, const uint32_t* __restrict__ win_big,
+             uint32_t* __restrict__ win_done, WinEntry* __restrict__ wtab) {
   pdl_wait();
   if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t lane = threadIdx.x & 31;
@@ -1436,19 +1452,32 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
       if (k > 0) lo = p_below + 1;
       if (k < 32) hi = p_at;
     }
-    if (lane == 0) wtab[e].P = lo - first;
+    /* a long queue has few hundred entries at most, spread over as many warps: they are counted,
+     * and the warp that stores the last one goes on to the queue's prefix pass */
+    uint32_t last = 0;
+    if (lane == 0) {
+      wtab[e].P = lo - first;
+      __threadfence();
+      last = atomicAdd(&win_done[s], 1u) + 1 == win_cnt[s] ? 1u : 0u;
+    }
+    if (__shfl_sync(0xffffffffu, last, 0)) {
+      __threadfence();
+      win_prefix_warp(s, ktab, win_off, win_cnt, wtab, lane);
+    }
   }
 }
 
-/* E and Kp of every table entry: one warp per queue runs over its windows, 32 at a time. */
+/* E and Kp of the table entries of the short queues: one warp per queue runs over its windows,
+ * 32 at a time. */
 __global__ void __launch_bounds__(256)
 k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
-             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
-             WinEntry* __restrict__ wtab) {
+             const uint32_t* __restrict__ seg_off, const uint32_t* __restrict__ win_off,
+             const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab) {
   pdl_wait();
   if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (s >= n_seg) return;                          /* whole warps leave together */
+  if (seg_off[s + 1] - seg_off[s] > kWinLongQueue) return;   /* done by k_win_bounds */
   win_prefix_warp(s, ktab, win_off, win_cnt, wtab, threadIdx.x & 31);
 }
 
@@ -1704,6 +1733,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   uint32_t* win_cnt = (uint32_t*)(ws + L.win_cnt);
   uint32_t* win_own = (uint32_t*)(ws + L.win_own);
   uint32_t* win_big = (uint32_t*)(ws + L.win_big);
+  uint32_t* win_done = (uint32_t*)(ws + L.win_done);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -1764,15 +1794,15 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   else
     launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
                out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-               (mode & PARD_MODE_SCAN) ? 1u : 0u);
+               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits);
   if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
     long long* est = (long long*)out->d_est_us;
     const bool raw = mode & PARD_MODE_RAW;
     /* window tables, and the decision from them */
     launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream, 
-        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_own, win_big, wtab);
-    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, win_off, win_cnt, wtab);
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
+    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab);
     mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)

@@ -32,7 +32,7 @@ constexpr int kSortThreads = 512;
 constexpr int kLoWarps = 8;                        /* warps 0..7 also do the look-back (one thread per digit) */
 constexpr int kItemsLo = 10, kItemsHi = 22;        /* rounds of 32 elements per warp: look-back warps / others (measured best) */
 constexpr int kSortTile = 32 * (kLoWarps * kItemsLo + (kSortThreads / 32 - kLoWarps) * kItemsHi);
-constexpr int kDecThreads = 256;
+constexpr int kDecThreads = 128;                   /* small blocks: a short tail when the grid drains (measured against 64 and 256) */
 constexpr int kDecItems = 8;
 constexpr int kDecTile = kDecThreads * kDecItems;
 constexpr int kCompactChunk = 1024;                /* indices moved by one warp of k_kept_move */
@@ -61,7 +61,8 @@ struct PlanHeader {
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
-  /* [hdr, zero_end) must be zero when the first kernel starts: one memset */
+  /* [hdr, zero_end) must be zero when the first kernel starts: cleared by k_clear (of the two
+   * look-back arrays only the first: every sort pass clears the array of the pass after it) */
   uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, lookback, zero_end,
       pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
@@ -97,8 +98,8 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.seg_kept = o;  o = al(o + 4ull * L.n_seg);
   L.win_done = o;  o = al(o + 4ull * L.n_seg);
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
-  L.lookback = o;  o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);   /* two arrays, used in turn */
-  L.zero_end = o;
+  L.lookback = o;  L.zero_end = al(o + 4ull * kBins * (uint64_t)L.sort_tiles);
+  o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);                    /* two arrays, used in turn */
   L.pipes = o;     o = al(o + 8ull * kMaxPipelinesPerCall);
   L.ktab = o;      o = al(o + sizeof(PardSegConst) * (uint64_t)L.n_seg);
   L.kept_base = o; o = al(o + 4ull * (L.n_seg + 1));
@@ -141,6 +142,17 @@ __device__ __forceinline__ bool last_block_done(uint32_t* counter) {
   const bool last = s_last != 0;
   if (last) __threadfence();
   return last;
+}
+
+/* Clears the part of the scratch that must start at zero.  A kernel rather than a memset: it is
+ * launched like every other kernel of the call, so its blocks are placed while the previous
+ * work of the stream drains. */
+__global__ void __launch_bounds__(256)
+k_clear(uint4* __restrict__ p, unsigned long long n16) {
+  pdl_wait();
+  const unsigned long long step = (unsigned long long)gridDim.x * blockDim.x;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += step)
+    p[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -1484,7 +1496,7 @@ k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegCo
 /* Decision pass from the window tables: every request on its own.  HF: some
  * queue may be served high budget first (the caller gave priorities). */
 template <bool RAW, bool HF>
-__global__ void __launch_bounds__(kDecThreads, 4)
+__global__ void __launch_bounds__(kDecThreads, 8)
 k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
              const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
@@ -1751,7 +1763,13 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   };
   mark();
   /* ---- clear the scratch that must start at zero: one contiguous region ---- */
-  PARD_CUDA_OK(cudaMemsetAsync(ws + L.hdr, 0, n > 0 ? L.zero_end : L.lookback, stream));
+  int sms = 148;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  {
+    const unsigned long long n16 = (n > 0 ? L.zero_end : L.lookback) / 16;   /* offsets are multiples of 256 */
+    launch_pdl(k_clear, (uint32_t)std::min<unsigned long long>((n16 + 255) / 256, (unsigned long long)sms * 4), 256, 0,
+               stream, (uint4*)(ws + L.hdr), n16);
+  }
   PipeTable pipe_table = {};
   pipe_table.many = d_pipes;
   if (n_pipelines <= (uint32_t)kFewPipelines)
@@ -1759,8 +1777,6 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   else
     PARD_CUDA_OK(cudaMemcpyAsync(d_pipes, h_pipes.data(), 8ull * n_pipelines, cudaMemcpyHostToDevice, stream));
 
-  int sms = 148;
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   rc = allow_sort_smem(dev);
   if (rc != PARD_OK) return rc;
   const uint4* req4 = (const uint4*)d_requests;
@@ -1854,10 +1870,10 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* key_width, seg_const, seg_win and kept_scan always; prepass, ctx_span, pack, the passes,
+  /* clear, key_width, seg_const, seg_win and kept_scan always; prepass, ctx_span, pack, the passes,
    * win_bounds, win_prefix, decide_win, tile_agg, decide and kept_move (when the compacted indices
    * are requested) when n > 0 */
-  *launches = n > 0 ? 4 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 6 : 4;
+  *launches = n > 0 ? 5 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 6 : 5;
   return PARD_OK;
 }
 

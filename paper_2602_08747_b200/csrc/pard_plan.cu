@@ -26,6 +26,7 @@ constexpr uint32_t kMaxPipelinesPerCall = 65536;
 constexpr uint32_t kSegNarrow = 1u;                /* bits of PardSegConst::narrow */
 constexpr uint32_t kSegNoStage = 2u;
 constexpr uint32_t kSegHighFirst = 4u;
+constexpr uint32_t kFoldSegs = 1024;              /* up to this many queues the key width is found inside k_seg_const */
 constexpr uint32_t kSpinLimit = 1u << 18;          /* polling rounds (about a microsecond each) before giving up */
 
 constexpr int kSortThreads = 512;
@@ -56,7 +57,8 @@ struct PlanHeader {
   uint32_t aborted;           /* 1: a bounded wait ran out; the sort is incomplete and every later kernel returns */
   uint32_t big_total;         /* window-table entries that belong to long queues */
   uint32_t agg_done;          /* blocks of k_tile_agg that have stored their aggregates */
-  uint32_t pad[64 - 12 - (kMaxPasses + 1)];
+  uint32_t seg_done;          /* blocks of k_seg_const that have stored their constants */
+  uint32_t pad[64 - 13 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
@@ -285,12 +287,12 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
             pard_queue_state_t st, uint32_t n_ctx,
             const unsigned long long* __restrict__ ctx_dmin_inv,
             const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
-            PlanHeader* hdr) {
+            PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width) {
   pdl_wait();
   const uint32_t S = (uint32_t)st.stage_stride;
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t seg = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (seg >= n_ctx * S) return;                          /* whole warps leave together */
+  if (seg < n_ctx * S) {                                 /* whole warps take the same side */
   const uint32_t c = seg / S, k = seg % S;
   PardSegConst out;
   out.A = 0; out.A_rel = 0; out.d = 1; out.cap = 1; out.d_magic = 0; out.cap_magic = 0;
@@ -354,6 +356,36 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
   }
   if (bad) set_status(hdr, PARD_EDATA);
   if (lane == 0) ktab[seg] = out;
+  }
+  /* With few queues the block that finishes last also finds the widest deadline span and with
+   * it the width of the sort key (the work of k_ctx_span and k_key_width, without their launches). */
+  if (!with_key_width) return;
+  if (!last_block_done(&hdr->seg_done)) return;
+  __shared__ unsigned long long s_span[4];
+  unsigned long long span = 0;
+  for (uint32_t c = threadIdx.x; c < n_ctx; c += blockDim.x) {
+    const unsigned long long lo = ~ctx_dmin_inv[c], hi = ctx_dmax[c];
+    if (lo <= hi && hi - lo > span) span = hi - lo;
+  }
+  for (int o = 16; o; o >>= 1) {
+    const unsigned long long a = __shfl_xor_sync(0xffffffffu, span, o);
+    span = a > span ? a : span;
+  }
+  if (lane == 0) s_span[threadIdx.x >> 5] = span;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (uint32_t w = 1; w < blockDim.x / 32; ++w) span = s_span[w] > span ? s_span[w] : span;
+    const uint32_t dbits = bit_width64(span);
+    hdr->span_max = span;
+    hdr->dbits = dbits;
+    hdr->keybits = sbits + dbits;
+    hdr->npass = (sbits + dbits + 7) / 8;
+    if (sbits + dbits + ibits > 64) {
+      hdr->npass = 0;
+      hdr->wide = 1;
+      set_status(hdr, PARD_ERANGE);
+    }
+  }
 }
 
 /* request -> sort element; digit histograms of every pass */
@@ -1787,9 +1819,13 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     launch_pdl(k_prepass, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, hdr);
   }
   mark();
-  if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
-  launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr);
-  launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab, hdr);
+  const bool fold_width = L.n_seg <= kFoldSegs;          /* few queues: k_seg_const's last block finds the key width */
+  if (!fold_width) {
+    if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
+    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr);
+  }
+  launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
+             hdr, sbits, ibits, fold_width ? 1u : 0u);
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
@@ -1870,10 +1906,13 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* clear, key_width, seg_const, seg_win and kept_scan always; prepass, ctx_span, pack, the passes,
+  /* clear, seg_const, seg_win and kept_scan always, key_width (and, when n > 0, ctx_span) with many
+   * queues; prepass, ctx_span, pack, the passes,
    * win_bounds, win_prefix, decide_win, tile_agg, decide and kept_move (when the compacted indices
    * are requested) when n > 0 */
-  *launches = n > 0 ? 5 + 3 + make_layout(n, n_ctx, stage_stride).max_passes + 6 : 5;
+  const uint32_t width_kernels = (uint64_t)n_ctx * (uint64_t)stage_stride <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
+  *launches = n > 0 ? 4 + width_kernels + 2 + width_kernels + make_layout(n, n_ctx, stage_stride).max_passes + 6
+                    : 4 + width_kernels;
   return PARD_OK;
 }
 

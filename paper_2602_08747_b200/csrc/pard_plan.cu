@@ -58,7 +58,9 @@ struct PlanHeader {
   uint32_t big_total;         /* window-table entries that belong to long queues */
   uint32_t agg_done;          /* blocks of k_tile_agg that have stored their aggregates */
   uint32_t seg_done;          /* blocks of k_seg_const that have stored their constants */
-  uint32_t pad[64 - 13 - (kMaxPasses + 1)];
+  uint32_t unsorted;          /* 1: some request's ctx is smaller than its predecessor's */
+  uint32_t ctx_too_big;       /* 1: some ctx holds more requests than one sort tile */
+  uint32_t pad[64 - 15 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
@@ -66,7 +68,7 @@ struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: cleared by k_clear (of the two
    * look-back arrays only the first: every sort pass clears the array of the pass after it) */
   uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, lookback, zero_end,
-      pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
+      ctx_start, pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
 };
@@ -102,6 +104,7 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
   L.lookback = o;  L.zero_end = al(o + 4ull * kBins * (uint64_t)L.sort_tiles);
   o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);                    /* two arrays, used in turn */
+  L.ctx_start = o; o = al(o + 4ull * ((uint64_t)n_ctx + 1));
   L.pipes = o;     o = al(o + 8ull * kMaxPipelinesPerCall);
   L.ktab = o;      o = al(o + sizeof(PardSegConst) * (uint64_t)L.n_seg);
   L.kept_base = o; o = al(o + 4ull * (L.n_seg + 1));
@@ -131,6 +134,11 @@ __device__ __forceinline__ void set_aborted(PlanHeader* hdr) {
   hdr->aborted = 1;
   __threadfence();
   atomicExch(&hdr->status, (uint32_t)(-PARD_ETIMEOUT));
+}
+
+/* See k_sort_local: the call's requests come grouped by ctx and no ctx exceeds a tile. */
+__device__ __forceinline__ bool sort_is_local(const PlanHeader* hdr, uint32_t candidate) {
+  return candidate && !hdr->unsorted && !hdr->ctx_too_big && !hdr->wide;
 }
 
 /* True in every thread of exactly one block: the one whose arrival at `counter` is the last of
@@ -393,11 +401,13 @@ __global__ void __launch_bounds__(256)
 k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
        const unsigned long long* __restrict__ ctx_dmin_inv, const unsigned long long* __restrict__ ctx_dmax,
        const uint8_t* __restrict__ priority, uint32_t ibits,
-       const PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
-       uint32_t* __restrict__ hist) {
+       PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
+       uint32_t* __restrict__ hist, const uint32_t* __restrict__ ctx_start) {
   pdl_wait();
   __shared__ uint32_t s_hist[kMaxPasses * kBins];
   if (hdr->wide) return;
+  bool out_of_range = false;                   /* ctx_start != nullptr: is every request inside its ctx's range? */
+  const bool with_hist = ctx_start == nullptr; /* else the digit counts are only needed if the global passes run: k_hist */
   const uint32_t npass = hdr->npass, dbits = hdr->dbits;
   for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
   __syncthreads();
@@ -415,11 +425,37 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
       const bool high_first = priority && __ldg(&priority[seg]) != 0;
       unsigned long long off = (high_first ? ctx_dmax[ctx] - D : D - ~ctx_dmin_inv[ctx]) & dmask;
       e = ((((unsigned long long)seg << dbits) | off) << ibits) | j;
+      if (ctx_start) out_of_range |= j < ctx_start[ctx] || j >= ctx_start[ctx + 1];
     } else {
       e = j;                                  /* flagged by the prepass; keep indices in range */
     }
     dst[j] = e;
     unsigned long long key = e >> ibits;
+    if (with_hist)
+      for (uint32_t p = 0; p < npass; ++p) atomicAdd(&s_hist[p * kBins + ((key >> (8 * p)) & 255u)], 1u);
+  }
+  if (out_of_range) hdr->unsorted = 1;         /* the requests are not grouped by ascending ctx */
+  __syncthreads();
+  if (with_hist)
+    for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x)
+      if (s_hist[i]) atomicAdd(&hist[i], s_hist[i]);
+}
+
+/* Digit counts of every pass from the packed elements: only for calls that were candidates for
+ * the block-local sort (k_pack then leaves the counting out) and turned out to need the global
+ * passes after all. */
+__global__ void __launch_bounds__(256)
+k_hist(const PlanHeader* __restrict__ hdr, uint32_t candidate, const unsigned long long* __restrict__ src, uint32_t n,
+       uint32_t ibits, uint32_t* __restrict__ hist) {
+  pdl_wait();
+  __shared__ uint32_t s_hist[kMaxPasses * kBins];
+  if (hdr->wide || hdr->aborted || sort_is_local(hdr, candidate)) return;
+  const uint32_t npass = hdr->npass;
+  for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
+  __syncthreads();
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += stride) {
+    const unsigned long long key = src[j] >> ibits;
     for (uint32_t p = 0; p < npass; ++p) atomicAdd(&s_hist[p * kBins + ((key >> (8 * p)) & 255u)], 1u);
   }
   __syncthreads();
@@ -482,8 +518,8 @@ __device__ __forceinline__ void sort_load_count(unsigned long long (&key)[kItems
 }
 
 /* one warp's share of step 4 */
-template <int ITEMS>
-__device__ __forceinline__ void sort_rank_drop(const unsigned long long (&key)[kItemsHi], uint32_t shift,
+template <int ITEMS, int CAP>
+__device__ __forceinline__ void sort_rank_drop(const unsigned long long (&key)[CAP], uint32_t shift,
                                                uint32_t* slot_row, uint32_t* match_row, unsigned long long* keys,
                                                uint32_t lanebit) {
 #pragma unroll
@@ -504,23 +540,29 @@ __device__ __forceinline__ void sort_rank_drop(const unsigned long long (&key)[k
   }
 }
 
+template <bool PERSIST>
 __global__ void __launch_bounds__(kSortThreads, 2)
 k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf_a,
             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ hist,
             uint32_t* __restrict__ lookback, uint32_t* __restrict__ lookback_next, uint32_t n,
-            uint32_t ibits, uint32_t stall) {
+            uint32_t ibits, uint32_t stall, uint32_t local_candidate) {
   pdl_wait();
   constexpr int WARPS = kSortThreads / 32;
   static_assert(kLoWarps * 32 == kBins, "one look-back thread per digit");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SortSmem& S = *reinterpret_cast<SortSmem*>(smem_raw);
 
-  if (pass >= hdr->npass || hdr->aborted) return;
+  if (pass >= hdr->npass || hdr->aborted || sort_is_local(hdr, local_candidate)) return;
   const unsigned long long* src = (pass & 1) ? buf_b : buf_a;
   unsigned long long* dst = (pass & 1) ? buf_a : buf_b;
   hist += pass * kBins;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lanebit = 1u << lane;
+  const uint32_t n_tiles = (uint32_t)(((uint64_t)n + kSortTile - 1) / kSortTile);
+  /* PERSIST: a small grid whose blocks take tile after tile (used where the pass is launched
+   * only as the fallback of the block-local sort and will almost always return at once);
+   * otherwise one tile per block */
+  for (;;) {
   if (tid == 0) {
     S.tile = atomicAdd(&hdr->ticket[pass], 1u);
     S.abort = 0;
@@ -532,6 +574,7 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   const uint32_t gh = tid < kBins ? hist[tid] : 0;     /* global count of digit tid, needed in step 2 */
   __syncthreads();
   const uint32_t tile = S.tile;
+  if (PERSIST && tile >= n_tiles) return;
   const uint64_t base = (uint64_t)tile * kSortTile;
   const uint32_t shift = ibits + 8 * pass;
 
@@ -613,8 +656,8 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   }
 
   /* 4. rank and drop into the tile buffer */
-  if (lo_warp) sort_rank_drop<kItemsLo>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
-  else sort_rank_drop<kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
+  if (lo_warp) sort_rank_drop<kItemsLo, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
+  else sort_rank_drop<kItemsHi, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
   __syncthreads();
   if (S.abort) {
     if (tid == 0) set_aborted(hdr);
@@ -629,6 +672,136 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
     const uint32_t d = (uint32_t)(k >> shift) & 255u;
     dst[S.gofs[d] + pos] = k;
   }
+  if (!PERSIST) return;
+  __syncthreads();                                     /* the tile buffer and the tables are reused */
+  }
+}
+
+/* ------------------------------------------------------------------------ */
+/* calls whose requests come grouped by ctx, every ctx within one tile       */
+/* ------------------------------------------------------------------------ */
+/* Batched decision epochs and small what-if instances arrive as one array with the requests of
+ * a ctx side by side.  If no ctx holds more than a tile, nothing has to move between ctxs: a
+ * block sorts "its" ctx in shared memory -- radix passes over the stage and deadline bits only,
+ * no global scatter, no look-back -- and the global passes do not run.  `candidate` is the
+ * host's part of the test (at least two ctxs, between kSortTile / 4 and kSortTile requests per
+ * ctx on average); the device adds what only it can see. */
+/* Where every ctx would begin if the requests came in ascending ctx order: the first request
+ * whose ctx is >= c, by a 32-ary search, one warp per ctx.  Whether they do come in that order
+ * is settled by k_pack, which checks every request against the range of its ctx; that test is
+ * complete as long as the boundaries themselves never step back, which is checked here. */
+__global__ void __launch_bounds__(256)
+k_ctx_ranges(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t* __restrict__ ctx_start,
+             PlanHeader* hdr) {
+  pdl_wait();
+  const uint32_t c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t lane = threadIdx.x & 31;
+  if (c > n_ctx) return;                         /* whole warps leave together */
+  uint32_t lo[2] = {0, 0}, hi[2] = {n, n};       /* first request whose ctx is >= c, >= c + 1 */
+  while (lo[0] < hi[0] || lo[1] < hi[1]) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      if (lo[q] < hi[q]) {                       /* uniform across the warp */
+        const uint32_t span = hi[q] - lo[q];
+        const uint32_t p = lo[q] + (uint32_t)(((unsigned long long)(lane + 1) * span) / 33u);   /* lo <= p < hi */
+        const bool less = __ldg(&req[p]).z < c + q;
+        const uint32_t k = __popc(__ballot_sync(0xffffffffu, less));
+        const uint32_t p_below = __shfl_sync(0xffffffffu, p, k > 0 ? k - 1 : 0);
+        const uint32_t p_at = __shfl_sync(0xffffffffu, p, k < 32 ? k : 31);
+        if (k > 0) lo[q] = p_below + 1;
+        if (k < 32) hi[q] = p_at;
+      }
+    }
+  }
+  if (lane != 0) return;
+  ctx_start[c] = lo[0];
+  if (c < n_ctx) {
+    if (lo[1] < lo[0]) hdr->unsorted = 1;
+    else if (lo[1] - lo[0] > (uint32_t)kSortTile) hdr->ctx_too_big = 1;
+  }
+}
+
+/* One block per ctx: the ctx's elements, as k_pack wrote them, sorted in shared memory and
+ * written to the buffer the global passes would have ended in.  Inside a ctx only the stage
+ * and the deadline offset differ; the ctx's own contribution to the segment field is taken off
+ * on the way in and put back on the way out, so that the passes see a plain bit field. */
+__global__ void __launch_bounds__(kSortThreads, 2)
+k_sort_local(const PlanHeader* __restrict__ hdr, uint32_t candidate, const unsigned long long* __restrict__ buf_a,
+             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ ctx_start, uint32_t S,
+             uint32_t stage_bits, uint32_t ibits) {
+  pdl_wait();
+  constexpr int WARPS = kSortThreads / 32;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  SortSmem& Sm = *reinterpret_cast<SortSmem*>(smem_raw);
+  if (!sort_is_local(hdr, candidate) || hdr->aborted) return;
+  const uint32_t c = blockIdx.x;
+  const uint32_t first = ctx_start[c], cnt = ctx_start[c + 1] - first;
+  if (cnt == 0) return;
+  unsigned long long* dst = (hdr->npass & 1) ? buf_b : const_cast<unsigned long long*>(buf_a);
+  const uint32_t dbits = hdr->dbits;
+  const uint32_t local_bits = dbits + stage_bits;
+  const uint32_t passes = (local_bits + 7) / 8;
+  const unsigned long long ctx_part = (unsigned long long)c * S << (dbits + ibits);   /* < 2^64: the key fits */
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lanebit = 1u << lane;
+  constexpr int kItems = kSortTile / kSortThreads;       /* every warp owns the same share here: nothing else to do meanwhile */
+  static_assert(kItems * kSortThreads == kSortTile, "the tile divides evenly");
+  const uint32_t wfirst = warp * (32 * kItems);
+
+  unsigned long long key[kItems];
+#pragma unroll
+  for (int i = 0; i < kItems; ++i) {
+    const uint32_t pos = wfirst + i * 32 + lane;
+    key[i] = pos < cnt ? buf_a[first + pos] - ctx_part : ~0ull;   /* padding sorts last */
+  }
+  for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) (&Sm.match[0][0])[i] = 0;   /* ranking leaves it clear */
+  for (uint32_t p = 0; p < passes; ++p) {
+    const uint32_t shift = ibits + 8 * p;
+    for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) (&Sm.slot[0][0])[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kItems; ++i) atomicAdd(&Sm.slot[warp][(uint32_t)(key[i] >> shift) & 255u], 1u);
+    __syncthreads();
+    uint32_t count = 0, x = 0;
+    if (tid < kBins) {                                  /* thread d owns digit d */
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) {
+        const uint32_t t = Sm.slot[w][tid];
+        Sm.slot[w][tid] = count;                        /* exclusive over the warps */
+        count += t;
+      }
+      x = count;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= (uint32_t)o) x += y;
+      }
+      if (lane == 31) Sm.scan[0][warp] = x;
+    }
+    __syncthreads();
+    if (tid < kBins) {
+      uint32_t wx = 0;
+#pragma unroll
+      for (int w = 0; w < kBins / 32; ++w)
+        if (w < (int)warp) wx += Sm.scan[0][w];
+      const uint32_t dstart = wx + x - count;           /* first slot of digit tid */
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) Sm.slot[w][tid] += dstart;
+    }
+    __syncthreads();
+    sort_rank_drop<kItems, kItems>(key, shift, Sm.slot[warp], Sm.match[warp], Sm.keys, lanebit);
+    __syncthreads();
+    if (p + 1 < passes) {
+#pragma unroll
+      for (int i = 0; i < kItems; ++i) key[i] = Sm.keys[wfirst + i * 32 + lane];
+      __syncthreads();
+    }
+  }
+  if (passes == 0) {                                    /* nothing differs inside a ctx: index order stands */
+#pragma unroll
+    for (int i = 0; i < kItems; ++i) Sm.keys[wfirst + i * 32 + lane] = key[i];
+    __syncthreads();
+  }
+  for (uint32_t pos = tid; pos < cnt; pos += kSortThreads) dst[first + pos] = Sm.keys[pos] + ctx_part;
 }
 
 /* ------------------------------------------------------------------------ */
@@ -1225,7 +1398,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
           const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
           uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
           uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
-          uint32_t force_scan, const uint32_t* __restrict__ hist, uint32_t sbits) {
+          uint32_t force_scan, const uint32_t* __restrict__ hist, uint32_t sbits, uint32_t local_candidate) {
   pdl_wait();
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1237,7 +1410,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
   const uint32_t dbits = hdr->dbits;
   const uint32_t npass = hdr->npass;
   const uint32_t top_bits = npass ? hdr->keybits - 8 * (npass - 1) : 0;   /* width of the last pass's digit */
-  if (!wide && n > 0 && npass && sbits <= top_bits) {
+  if (!wide && n > 0 && npass && sbits <= top_bits && !sort_is_local(hdr, local_candidate)) {
     /* the segment id is the upper part of the last pass's digit: the queue starts where the
      * digits below (s << (top_bits - sbits)) end, and the digit counts of that pass are known */
     const uint32_t* h = hist + (npass - 1) * kBins;
@@ -1691,11 +1864,19 @@ int allow_sort_smem(int dev) {
   std::lock_guard<std::mutex> lock(mu);
   if (dev < 0 || dev >= 64) return PARD_ERANGE;
   if (!done[dev]) {
-    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(SortSmem)));
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(SortSmem)));
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_local, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
     done[dev] = true;
   }
   return PARD_OK;
+}
+
+bool local_sort_candidate(uint64_t n, uint32_t n_ctx) {
+  return n_ctx >= 2 && n >= (uint64_t)n_ctx * (kSortTile / 4) && n <= (uint64_t)n_ctx * kSortTile;
 }
 
 int check_state(const pard_queue_state_t* st, uint32_t n_ctx) {
@@ -1786,6 +1967,9 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   const uint32_t sbits = ceil_log2(L.n_seg);
 
   bool prof_coarse = false;
+  /* requests grouped by ctx, no ctx beyond a tile: worth testing for when the sizes allow it */
+  const uint32_t local_cand = local_sort_candidate(n, n_ctx) ? 1u : 0u;
+  uint32_t* ctx_start = (uint32_t*)(ws + L.ctx_start);
   cudaEvent_t* evs = profile_acquire(&prof_coarse);
   int phase = 0;
   auto mark = [&]() {                      /* boundary between two phases */
@@ -1826,17 +2010,26 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   }
   launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
              hdr, sbits, ibits, fold_width ? 1u : 0u);
+  if (local_cand) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
-    launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, ibits, hdr, buf_a, hist);
+    launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, ibits, hdr, buf_a, hist,
+               local_cand ? (const uint32_t*)ctx_start : (const uint32_t*)nullptr);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
+    if (p == 0 && local_cand) {                  /* every ctx inside one tile: sorted block by block (else returns at once) */
+      launch_pdl(k_sort_local, n_ctx, kSortThreads, sizeof(SortSmem), stream, hdr, local_cand, buf_a, buf_b, ctx_start, S,
+                 ceil_log2(S), ibits);
+      launch_pdl(k_hist, (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8), 256, 0, stream, hdr, local_cand,
+                 buf_a, n32, ibits, hist);
+    }
     if (n > 0 && p < L.max_passes)
-      launch_pdl(k_sort_pass, L.sort_tiles, kSortThreads, sizeof(SortSmem), stream, 
+      launch_pdl(local_cand ? k_sort_pass<true> : k_sort_pass<false>,
+                 local_cand ? std::min<uint32_t>(L.sort_tiles, 2u * (uint32_t)sms) : L.sort_tiles, kSortThreads, sizeof(SortSmem), stream,
           p, hdr, buf_a, buf_b, hist, lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words,
-          n32, ibits, (p == 0 && (mode & PARD_MODE_TEST_STALL)) ? 1u : 0u);
+          n32, ibits, (p == 0 && (mode & PARD_MODE_TEST_STALL)) ? 1u : 0u, local_cand);
   }
   mark();
   if (L.n_seg >= kManyQueues)
@@ -1846,7 +2039,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   else
     launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
                out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits);
+               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits, local_cand);
   if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
     long long* est = (long long*)out->d_est_us;
@@ -1911,7 +2104,9 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
    * win_bounds, win_prefix, decide_win, tile_agg, decide and kept_move (when the compacted indices
    * are requested) when n > 0 */
   const uint32_t width_kernels = (uint64_t)n_ctx * (uint64_t)stage_stride <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
-  *launches = n > 0 ? 4 + width_kernels + 2 + width_kernels + make_layout(n, n_ctx, stage_stride).max_passes + 6
+  const uint32_t local_kernels = local_sort_candidate(n, n_ctx) ? 3 : 0;   /* ctx_ranges, sort_local, hist */
+  *launches = n > 0 ? 4 + width_kernels + 2 + width_kernels + local_kernels +
+                          make_layout(n, n_ctx, stage_stride).max_passes + 6
                     : 4 + width_kernels;
   return PARD_OK;
 }

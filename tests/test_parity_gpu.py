@@ -260,3 +260,65 @@ def test_window_count_limits():
         dl = rng.integers(0, span_windows * d, size=50_000)
         dl[0] = span_windows * d - 1                      # the last window is occupied
         both(_one_stage(len(dl), dl, d=d, B=3))
+
+
+# --------------------------------------------------------------------------
+# requests grouped by ctx, every ctx within one sort tile: the block-local sort
+# --------------------------------------------------------------------------
+def _grouped(n_epochs=40, seed=0, keep_lo=0.3):
+    """C4b with a random share of every epoch's requests removed (order kept):
+    contexts of ragged sizes, still grouped by ascending ctx."""
+    rng = np.random.default_rng(seed)
+    wl = inputs.make("C4b", n_epochs=n_epochs, per_epoch=8192)
+    share = rng.uniform(keep_lo, 1.0, size=wl.n_ctx)
+    share[rng.integers(0, wl.n_ctx)] = 1.0                       # one ctx fills its tile exactly
+    keep = rng.random(wl.n) < share[wl.requests["ctx"]]
+    wl.requests = np.ascontiguousarray(wl.requests[keep])
+    return wl, rng
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_grouped_contexts_take_the_local_sort(mode):
+    wl, rng = _grouped(seed=1)
+    both(wl, mode)
+    # some contexts empty, one with a single request
+    wl, rng = _grouped(seed=2, keep_lo=0.5)
+    r = wl.requests
+    drop = np.isin(r["ctx"], [3, 4, 17]) | ((r["ctx"] == 9) & (np.arange(wl.n) != np.flatnonzero(r["ctx"] == 9)[0]))
+    wl.requests = np.ascontiguousarray(r[~drop])
+    both(wl, mode)
+    # queues served high budget first among them
+    wl, rng = _grouped(seed=3)
+    wl.state.priority = rng.integers(0, 2, size=(wl.n_ctx, wl.state.stage_stride)).astype(np.uint8)
+    both(wl, mode)
+
+
+def test_grouped_contexts_fall_back_when_the_device_says_no():
+    """Same sizes, but the device finds a reason against the local sort: requests
+    out of ctx order, or one ctx larger than a tile.  Results are the oracle's
+    either way."""
+    wl, rng = _grouped(seed=4)
+    r = wl.requests.copy()
+    i, j = 5, wl.n - 7
+    r[[i, j]] = r[[j, i]]                                        # two requests far from their ctx's group
+    wl.requests = r
+    both(wl)
+    wl, rng = _grouped(seed=5, keep_lo=0.9)
+    r = wl.requests.copy()
+    r["ctx"][r["ctx"] == 21] = 20                                # ctx 20 now holds two epochs, ctx 21 none
+    wl.requests = r
+    both(wl)
+    # shuffled completely
+    wl, rng = _grouped(seed=6)
+    wl.requests = np.ascontiguousarray(wl.requests[rng.permutation(wl.n)])
+    both(wl)
+
+
+def test_grouped_contexts_with_equal_deadlines_and_one_stage():
+    """No bit differs inside a ctx (one stage, all deadlines of a ctx equal): index order stands."""
+    p = util.pipeline([], 1, [10], bmax=2)
+    n_ctx, per = 6, 3000
+    ctx = np.repeat(np.arange(n_ctx), per)
+    dl = 1000 + 50 * ctx
+    st = util.state(n_ctx, 1, 0, 900, 2)
+    both(inputs.Workload("flat", [p], util.requests(dl, stage=0, ctx=ctx), st, n_ctx))

@@ -174,7 +174,9 @@ typedef struct pard_plan_out {
                                    later tiles wait for, so their waits run out (after
                                    about a third of a second) and the call returns
                                    PARD_ETIMEOUT with unspecified outputs; the CUDA
-                                   context stays usable                               */
+                                   context stays usable.  Calls that the library sorts
+                                   block by block (requests grouped by ctx, no ctx above
+                                   8,192 requests) have no such wait and are unaffected */
 
 /* Device scratch pard_plan needs for n requests in n_ctx contexts. */
 int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,

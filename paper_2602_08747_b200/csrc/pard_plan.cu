@@ -402,12 +402,13 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
        const unsigned long long* __restrict__ ctx_dmin_inv, const unsigned long long* __restrict__ ctx_dmax,
        const uint8_t* __restrict__ priority, uint32_t ibits,
        PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
-       uint32_t* __restrict__ hist, const uint32_t* __restrict__ ctx_start) {
+       uint32_t* __restrict__ hist, const uint32_t* __restrict__ ctx_start, uint32_t with_hist) {
   pdl_wait();
   __shared__ uint32_t s_hist[kMaxPasses * kBins];
   if (hdr->wide) return;
   bool out_of_range = false;                   /* ctx_start != nullptr: is every request inside its ctx's range? */
-  const bool with_hist = ctx_start == nullptr; /* else the digit counts are only needed if the global passes run: k_hist */
+  /* with_hist == 0: the call is sorted block by block; the digit counts are only needed if the
+   * global passes run after all, and k_hist makes them up then */
   const uint32_t npass = hdr->npass, dbits = hdr->dbits;
   for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
   __syncthreads();
@@ -684,8 +685,10 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
  * a ctx side by side.  If no ctx holds more than a tile, nothing has to move between ctxs: a
  * block sorts "its" ctx in shared memory -- radix passes over the stage and deadline bits only,
  * no global scatter, no look-back -- and the global passes do not run.  `candidate` is the
- * host's part of the test (at least two ctxs, between kSortTile / 4 and kSortTile requests per
- * ctx on average); the device adds what only it can see. */
+ * host's part of the test (between kSortTile / 4 and kSortTile requests per ctx on average);
+ * the device adds what only it can see.  A call with a single ctx of at most kSortTile requests
+ * needs no test at all: its one block is certain, and neither the range search nor the global
+ * passes are launched -- the case of one module's queue planned every few milliseconds. */
 /* Where every ctx would begin if the requests came in ascending ctx order: the first request
  * whose ctx is >= c, by a 32-ary search, one warp per ctx.  Whether they do come in that order
  * is settled by k_pack, which checks every request against the range of its ctx; that test is
@@ -727,15 +730,16 @@ k_ctx_ranges(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t
  * on the way in and put back on the way out, so that the passes see a plain bit field. */
 __global__ void __launch_bounds__(kSortThreads, 2)
 k_sort_local(const PlanHeader* __restrict__ hdr, uint32_t candidate, const unsigned long long* __restrict__ buf_a,
-             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ ctx_start, uint32_t S,
-             uint32_t stage_bits, uint32_t ibits) {
+             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ ctx_start, uint32_t n,
+             uint32_t S, uint32_t stage_bits, uint32_t ibits) {
   pdl_wait();
   constexpr int WARPS = kSortThreads / 32;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SortSmem& Sm = *reinterpret_cast<SortSmem*>(smem_raw);
   if (!sort_is_local(hdr, candidate) || hdr->aborted) return;
   const uint32_t c = blockIdx.x;
-  const uint32_t first = ctx_start[c], cnt = ctx_start[c + 1] - first;
+  const uint32_t first = ctx_start ? ctx_start[c] : 0u;              /* no table: the call has one ctx */
+  const uint32_t cnt = ctx_start ? ctx_start[c + 1] - first : n;
   if (cnt == 0) return;
   unsigned long long* dst = (hdr->npass & 1) ? buf_b : const_cast<unsigned long long*>(buf_a);
   const uint32_t dbits = hdr->dbits;
@@ -1876,7 +1880,8 @@ int allow_sort_smem(int dev) {
 }
 
 bool local_sort_candidate(uint64_t n, uint32_t n_ctx) {
-  return n_ctx >= 2 && n >= (uint64_t)n_ctx * (kSortTile / 4) && n <= (uint64_t)n_ctx * kSortTile;
+  if (n_ctx == 1) return n > 0 && n <= (uint64_t)kSortTile;         /* certain: one ctx inside one tile */
+  return n >= (uint64_t)n_ctx * (kSortTile / 4) && n <= (uint64_t)n_ctx * kSortTile;
 }
 
 int check_state(const pard_queue_state_t* st, uint32_t n_ctx) {
@@ -1969,6 +1974,8 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   bool prof_coarse = false;
   /* requests grouped by ctx, no ctx beyond a tile: worth testing for when the sizes allow it */
   const uint32_t local_cand = local_sort_candidate(n, n_ctx) ? 1u : 0u;
+  /* one ctx that fits a tile: the local sort is certain, no range search, no order check, no fallback passes */
+  const bool local_sure = local_cand && n_ctx == 1;
   uint32_t* ctx_start = (uint32_t*)(ws + L.ctx_start);
   cudaEvent_t* evs = profile_acquire(&prof_coarse);
   int phase = 0;
@@ -2010,22 +2017,23 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   }
   launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
              hdr, sbits, ibits, fold_width ? 1u : 0u);
-  if (local_cand) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
+  if (local_cand && !local_sure) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
   mark();
   if (n > 0) {
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
     launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, ibits, hdr, buf_a, hist,
-               local_cand ? (const uint32_t*)ctx_start : (const uint32_t*)nullptr);
+               (local_cand && !local_sure) ? (const uint32_t*)ctx_start : (const uint32_t*)nullptr, local_cand ? 0u : 1u);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
     if (p == 0 && local_cand) {                  /* every ctx inside one tile: sorted block by block (else returns at once) */
-      launch_pdl(k_sort_local, n_ctx, kSortThreads, sizeof(SortSmem), stream, hdr, local_cand, buf_a, buf_b, ctx_start, S,
-                 ceil_log2(S), ibits);
-      launch_pdl(k_hist, (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8), 256, 0, stream, hdr, local_cand,
-                 buf_a, n32, ibits, hist);
+      launch_pdl(k_sort_local, n_ctx, kSortThreads, sizeof(SortSmem), stream, hdr, local_cand, buf_a, buf_b,
+                 local_sure ? (const uint32_t*)nullptr : (const uint32_t*)ctx_start, n32, S, ceil_log2(S), ibits);
+      if (!local_sure)
+        launch_pdl(k_hist, (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8), 256, 0, stream, hdr, local_cand,
+                   buf_a, n32, ibits, hist);
     }
-    if (n > 0 && p < L.max_passes)
+    if (n > 0 && p < L.max_passes && !local_sure)
       launch_pdl(local_cand ? k_sort_pass<true> : k_sort_pass<false>,
                  local_cand ? std::min<uint32_t>(L.sort_tiles, 2u * (uint32_t)sms) : L.sort_tiles, kSortThreads, sizeof(SortSmem), stream,
           p, hdr, buf_a, buf_b, hist, lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words,
@@ -2104,10 +2112,10 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
    * win_bounds, win_prefix, decide_win, tile_agg, decide and kept_move (when the compacted indices
    * are requested) when n > 0 */
   const uint32_t width_kernels = (uint64_t)n_ctx * (uint64_t)stage_stride <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
-  const uint32_t local_kernels = local_sort_candidate(n, n_ctx) ? 3 : 0;   /* ctx_ranges, sort_local, hist */
-  *launches = n > 0 ? 4 + width_kernels + 2 + width_kernels + local_kernels +
-                          make_layout(n, n_ctx, stage_stride).max_passes + 6
-                    : 4 + width_kernels;
+  const bool local_cand = local_sort_candidate(n, n_ctx), local_sure = local_cand && n_ctx == 1;
+  const uint32_t local_kernels = local_sure ? 1 : local_cand ? 3 : 0;       /* sort_local (, ctx_ranges, hist) */
+  const uint32_t passes = local_sure ? 0 : make_layout(n, n_ctx, stage_stride).max_passes;
+  *launches = n > 0 ? 4 + width_kernels + 2 + width_kernels + local_kernels + passes + 6 : 4 + width_kernels;
   return PARD_OK;
 }
 

@@ -439,8 +439,8 @@ def run_aux(dev, peak, kernels_only=False):
     epochs = []
     for e in range(n_ep):
         r = wl5.requests.copy()
-        r["deadline_us"] += e * 200_000 + job_rng.integers(0, 2000, size=r.shape[0])
-        epochs.append((st5.now_us + e * 200_000, r))
+        r["deadline_us"] += e * 600_000 + job_rng.integers(0, 2000, size=r.shape[0])
+        epochs.append((st5.now_us + e * 600_000, r))
     R5 = rp.Replay(pipes, st5.pipeline_of_ctx, inst, st5.stage_stride, st5.slot_stride, st5.batch, st5.workers,
                    st5.free_at_us, st5.w_us, None, 64, 5_000_000, wl5.n, dev)
     d_now = torch.from_numpy(np.stack([e[0] for e in epochs])).to(dev)
@@ -448,7 +448,12 @@ def run_aux(dev, peak, kernels_only=False):
     total = torch.zeros((n_ep, inst), dtype=torch.int64, device=dev)
     kept = torch.zeros((n_ep, inst), dtype=torch.int64, device=dev)
 
+    fa0 = R5.state.free_at_us.clone()
+
     def one_replay():
+        R5.state.free_at_us.copy_(fa0)                    # every run starts from the same state
+        R5.sample_time.fill_(-1)
+        R5.epoch = 0
         for i in range(n_ep):
             R5.step(d_now[i], d_req[i], wl5.n, total[i], kept[i])
 
@@ -456,6 +461,7 @@ def run_aux(dev, peak, kernels_only=False):
     assert R5.statuses() == 0
     out["replay"] = {"workload": "%d instances, %d epochs x %d requests" % (inst, n_ep, wl5.n), "ms_per_epoch": 1e3 * sec / n_ep,
                      "epochs_per_s": n_ep / sec, "requests_per_s": wl5.n * n_ep / sec,
+                     "epoch_spacing_us": 600_000,
                      "kept_fraction_last_run": float(kept.sum().item()) / float(max(1, total.sum().item()))}
     for p in pipes:
         p.free()
@@ -561,6 +567,18 @@ def run_ours(args):
                                         "kernels": kernel_table(prof2, wlb.n, kf, peak, prof2c)}
             del pl2
         aux = {} if args.no_variants else run_aux(dev, peak)
+        others = {}
+        if not args.no_variants:
+            # the other configurations of the workload list, device-resident, for the record
+            for name in ("C1", "C2", "C4", "C5"):
+                wlo = inputs.make(name)
+                plo = DevicePlan(wlo, dev)
+                plo.step(nowait=False)
+                kfo = float(plo.out.n_kept.cpu()[0]) / wlo.n
+                so, _ = timed_steps(plo, 50, 5, None)
+                others[name] = {"requests": wlo.n, "contexts": wlo.n_ctx, "us_per_step": 1e6 * so / 50,
+                                "requests_per_s": wlo.n * 50 / so, "keep_fraction": kfo}
+                del plo, wlo
         t_cpu, _ = time_oracle(wl, 2)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -587,6 +605,7 @@ def run_ours(args):
                              "host_cores": os.cpu_count()},
             "variants": variants,
             "state_planner_kernels": aux,
+            "other_workloads": others,
         }
         print(json.dumps(line))
     if dist is not None:

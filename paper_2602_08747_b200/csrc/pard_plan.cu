@@ -402,13 +402,10 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
        const unsigned long long* __restrict__ ctx_dmin_inv, const unsigned long long* __restrict__ ctx_dmax,
        const uint8_t* __restrict__ priority, uint32_t ibits,
        PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
-       uint32_t* __restrict__ hist, const uint32_t* __restrict__ ctx_start, uint32_t with_hist) {
+       uint32_t* __restrict__ hist, uint32_t local_candidate) {
   pdl_wait();
   __shared__ uint32_t s_hist[kMaxPasses * kBins];
-  if (hdr->wide) return;
-  bool out_of_range = false;                   /* ctx_start != nullptr: is every request inside its ctx's range? */
-  /* with_hist == 0: the call is sorted block by block; the digit counts are only needed if the
-   * global passes run after all, and k_hist makes them up then */
+  if (hdr->wide || sort_is_local(hdr, local_candidate)) return;   /* sorted block by block: k_sort_local read the requests itself */
   const uint32_t npass = hdr->npass, dbits = hdr->dbits;
   for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
   __syncthreads();
@@ -426,37 +423,11 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
       const bool high_first = priority && __ldg(&priority[seg]) != 0;
       unsigned long long off = (high_first ? ctx_dmax[ctx] - D : D - ~ctx_dmin_inv[ctx]) & dmask;
       e = ((((unsigned long long)seg << dbits) | off) << ibits) | j;
-      if (ctx_start) out_of_range |= j < ctx_start[ctx] || j >= ctx_start[ctx + 1];
     } else {
       e = j;                                  /* flagged by the prepass; keep indices in range */
     }
     dst[j] = e;
     unsigned long long key = e >> ibits;
-    if (with_hist)
-      for (uint32_t p = 0; p < npass; ++p) atomicAdd(&s_hist[p * kBins + ((key >> (8 * p)) & 255u)], 1u);
-  }
-  if (out_of_range) hdr->unsorted = 1;         /* the requests are not grouped by ascending ctx */
-  __syncthreads();
-  if (with_hist)
-    for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x)
-      if (s_hist[i]) atomicAdd(&hist[i], s_hist[i]);
-}
-
-/* Digit counts of every pass from the packed elements: only for calls that were candidates for
- * the block-local sort (k_pack then leaves the counting out) and turned out to need the global
- * passes after all. */
-__global__ void __launch_bounds__(256)
-k_hist(const PlanHeader* __restrict__ hdr, uint32_t candidate, const unsigned long long* __restrict__ src, uint32_t n,
-       uint32_t ibits, uint32_t* __restrict__ hist) {
-  pdl_wait();
-  __shared__ uint32_t s_hist[kMaxPasses * kBins];
-  if (hdr->wide || hdr->aborted || sort_is_local(hdr, candidate)) return;
-  const uint32_t npass = hdr->npass;
-  for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
-  __syncthreads();
-  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-  for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += stride) {
-    const unsigned long long key = src[j] >> ibits;
     for (uint32_t p = 0; p < npass; ++p) atomicAdd(&s_hist[p * kBins + ((key >> (8 * p)) & 255u)], 1u);
   }
   __syncthreads();
@@ -691,8 +662,9 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
  * passes are launched -- the case of one module's queue planned every few milliseconds. */
 /* Where every ctx would begin if the requests came in ascending ctx order: the first request
  * whose ctx is >= c, by a 32-ary search, one warp per ctx.  Whether they do come in that order
- * is settled by k_pack, which checks every request against the range of its ctx; that test is
- * complete as long as the boundaries themselves never step back, which is checked here. */
+ * is settled by k_sort_local, where every block checks that its range holds requests of its ctx
+ * only; that test is complete as long as the boundaries never step back and the ranges cover
+ * all requests, which is checked here. */
 __global__ void __launch_bounds__(256)
 k_ctx_ranges(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t* __restrict__ ctx_start,
              PlanHeader* hdr) {
@@ -718,18 +690,22 @@ k_ctx_ranges(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t
   }
   if (lane != 0) return;
   ctx_start[c] = lo[0];
+  if (c == n_ctx && lo[0] != n) hdr->unsorted = 1;      /* requests past the last ctx's range (ctx out of range) */
   if (c < n_ctx) {
     if (lo[1] < lo[0]) hdr->unsorted = 1;
     else if (lo[1] - lo[0] > (uint32_t)kSortTile) hdr->ctx_too_big = 1;
   }
 }
 
-/* One block per ctx: the ctx's elements, as k_pack wrote them, sorted in shared memory and
- * written to the buffer the global passes would have ended in.  Inside a ctx only the stage
- * and the deadline offset differ; the ctx's own contribution to the segment field is taken off
- * on the way in and put back on the way out, so that the passes see a plain bit field. */
+/* One block per ctx: the ctx's requests, read from the caller's array, turned into the sort
+ * elements k_pack would have made, sorted in shared memory and written to the buffer the global
+ * passes would have ended in (k_pack does not run then).  Inside a ctx only the stage and the
+ * deadline offset differ; the ctx's own contribution to the segment field is left out of the
+ * element while it is sorted and added on the way out, so that the passes see a plain bit field. */
 __global__ void __launch_bounds__(kSortThreads, 2)
-k_sort_local(const PlanHeader* __restrict__ hdr, uint32_t candidate, const unsigned long long* __restrict__ buf_a,
+k_sort_local(PlanHeader* __restrict__ hdr, uint32_t candidate, const uint4* __restrict__ req,
+             const unsigned long long* __restrict__ ctx_dmin_inv, const unsigned long long* __restrict__ ctx_dmax,
+             const uint8_t* __restrict__ priority, unsigned long long* __restrict__ buf_a,
              unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ ctx_start, uint32_t n,
              uint32_t S, uint32_t stage_bits, uint32_t ibits) {
   pdl_wait();
@@ -741,8 +717,10 @@ k_sort_local(const PlanHeader* __restrict__ hdr, uint32_t candidate, const unsig
   const uint32_t first = ctx_start ? ctx_start[c] : 0u;              /* no table: the call has one ctx */
   const uint32_t cnt = ctx_start ? ctx_start[c + 1] - first : n;
   if (cnt == 0) return;
-  unsigned long long* dst = (hdr->npass & 1) ? buf_b : const_cast<unsigned long long*>(buf_a);
+  unsigned long long* dst = (hdr->npass & 1) ? buf_b : buf_a;
   const uint32_t dbits = hdr->dbits;
+  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  const unsigned long long dmin = ~ctx_dmin_inv[c], dmax = ctx_dmax[c];
   const uint32_t local_bits = dbits + stage_bits;
   const uint32_t passes = (local_bits + 7) / 8;
   const unsigned long long ctx_part = (unsigned long long)c * S << (dbits + ibits);   /* < 2^64: the key fits */
@@ -752,11 +730,33 @@ k_sort_local(const PlanHeader* __restrict__ hdr, uint32_t candidate, const unsig
   static_assert(kItems * kSortThreads == kSortTile, "the tile divides evenly");
   const uint32_t wfirst = warp * (32 * kItems);
 
+  /* the ctx's requests, straight from the caller's array, turned into sort elements without the
+   * ctx's share of the segment field (k_pack's element minus ctx_part); a request of another
+   * ctx inside the range means the requests are not grouped after all */
   unsigned long long key[kItems];
+  bool foreign = false;
 #pragma unroll
   for (int i = 0; i < kItems; ++i) {
     const uint32_t pos = wfirst + i * 32 + lane;
-    key[i] = pos < cnt ? buf_a[first + pos] - ctx_part : ~0ull;   /* padding sorts last */
+    key[i] = ~0ull;                                       /* padding sorts last */
+    if (pos < cnt) {
+      const uint32_t j = first + pos;
+      const uint4 r = __ldg(&req[j]);
+      const unsigned long long D = ((unsigned long long)r.y << 32) | r.x;
+      const uint32_t stage = r.w & 0xffffu;
+      foreign |= ctx_start != nullptr && r.z != c;       /* with one ctx there is no other: an input error */
+      if (r.z == c && stage < S) {
+        const bool high_first = priority && __ldg(&priority[c * S + stage]) != 0;
+        const unsigned long long off = (high_first ? dmax - D : D - dmin) & dmask;
+        key[i] = ((((unsigned long long)stage << dbits) | off) << ibits) | j;
+      } else {
+        key[i] = (unsigned long long)j - ctx_part;        /* flagged by the prepass; k_pack's element is j */
+      }
+    }
+  }
+  if (__syncthreads_or(foreign)) {                        /* the global passes take over (k_pack, then k_sort_pass) */
+    if (tid == 0) hdr->unsorted = 1;
+    return;
   }
   for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) (&Sm.match[0][0])[i] = 0;   /* ranking leaves it clear */
   for (uint32_t p = 0; p < passes; ++p) {
@@ -2019,20 +2019,17 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
              hdr, sbits, ibits, fold_width ? 1u : 0u);
   if (local_cand && !local_sure) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
   mark();
-  if (n > 0) {
+  if (local_cand)                                /* every ctx inside one tile: sorted block by block, straight from the requests */
+    launch_pdl(k_sort_local, n_ctx, kSortThreads, sizeof(SortSmem), stream, hdr, local_cand, req4, ctx_dmin, ctx_dmax,
+               state->d_priority, buf_a, buf_b, local_sure ? (const uint32_t*)nullptr : (const uint32_t*)ctx_start, n32, S,
+               ceil_log2(S), ibits);
+  if (n > 0 && !local_sure) {                    /* returns at once when the blocks above did the work */
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
     launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, ibits, hdr, buf_a, hist,
-               (local_cand && !local_sure) ? (const uint32_t*)ctx_start : (const uint32_t*)nullptr, local_cand ? 0u : 1u);
+               local_cand);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
-    if (p == 0 && local_cand) {                  /* every ctx inside one tile: sorted block by block (else returns at once) */
-      launch_pdl(k_sort_local, n_ctx, kSortThreads, sizeof(SortSmem), stream, hdr, local_cand, buf_a, buf_b,
-                 local_sure ? (const uint32_t*)nullptr : (const uint32_t*)ctx_start, n32, S, ceil_log2(S), ibits);
-      if (!local_sure)
-        launch_pdl(k_hist, (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8), 256, 0, stream, hdr, local_cand,
-                   buf_a, n32, ibits, hist);
-    }
     if (n > 0 && p < L.max_passes && !local_sure)
       launch_pdl(local_cand ? k_sort_pass<true> : k_sort_pass<false>,
                  local_cand ? std::min<uint32_t>(L.sort_tiles, 2u * (uint32_t)sms) : L.sort_tiles, kSortThreads, sizeof(SortSmem), stream,
@@ -2113,9 +2110,10 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
    * are requested) when n > 0 */
   const uint32_t width_kernels = (uint64_t)n_ctx * (uint64_t)stage_stride <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
   const bool local_cand = local_sort_candidate(n, n_ctx), local_sure = local_cand && n_ctx == 1;
-  const uint32_t local_kernels = local_sure ? 1 : local_cand ? 3 : 0;       /* sort_local (, ctx_ranges, hist) */
+  const uint32_t local_kernels = local_sure ? 1 : local_cand ? 2 : 0;       /* sort_local (, ctx_ranges) */
   const uint32_t passes = local_sure ? 0 : make_layout(n, n_ctx, stage_stride).max_passes;
-  *launches = n > 0 ? 4 + width_kernels + 2 + width_kernels + local_kernels + passes + 6 : 4 + width_kernels;
+  const uint32_t pack = local_sure ? 0 : 1;
+  *launches = n > 0 ? 4 + width_kernels + 1 + pack + width_kernels + local_kernels + passes + 6 : 4 + width_kernels;
   return PARD_OK;
 }
 

@@ -202,7 +202,11 @@ int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
  * stream); the call then waits for the stream and reads back one status word,
  * so a PARD_EDATA / PARD_ETIMEOUT found on the device is returned here.  The
  * library allocates no device memory in this call.
- * Host-detectable errors are returned before anything is launched. */
+ * Host-detectable errors are returned before anything is launched.
+ * Performance note: requests may come in any order.  When they come grouped by
+ * ascending ctx and no ctx holds more than 8,192 of them (batched decision
+ * epochs, one module's queue), every ctx is sorted by one thread block in
+ * shared memory, which is markedly faster; the result is the same. */
 int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
               const pard_request_t* d_requests, uint64_t n,
               const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,

@@ -120,6 +120,32 @@ def time_oracle(wl, repeats):
     return best, o
 
 
+def _oracle_shard(job):
+    """Worker of the all-cores CPU baseline: draws the (reduced) workload, keeps
+    this worker's share of its contexts and times the oracle on it."""
+    name, kw, world, rank = job
+    from oracle import oracle
+    from paper_2602_08747_b200 import sharding
+    wl = sharding.shard_workload(inputs.make(name, **kw), world, rank)
+    t = time.perf_counter()
+    oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
+    return wl.n, time.perf_counter() - t
+
+
+def oracle_all_cores(name, kw):
+    """The oracle, unchanged, over the contexts of a many-context workload on all
+    host cores: one share of the contexts per process, no exchange (contexts are
+    independent).  Processes are spawned, never forked: the parent holds a CUDA
+    context.  Returns requests per second by the slowest worker's clock."""
+    import multiprocessing as mp
+    cores = max(1, min(os.cpu_count() or 1, 32))
+    with mp.get_context("spawn").Pool(cores) as pool:
+        res = pool.map(_oracle_shard, [(name, kw, cores, r) for r in range(cores)])
+    n = sum(r[0] for r in res)
+    return {"value": n / max(r[1] for r in res), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%s drawn with %s: %d requests, contexts split over %d processes" % (name, kw, n, cores)}
+
+
 def run_reference(args):
     """The oracle, as it stands, on the host cores; each step plans a bounded
     sample (a smaller draw of the same workload)."""
@@ -579,6 +605,9 @@ def run_ours(args):
                 others[name] = {"requests": wlo.n, "contexts": wlo.n_ctx, "us_per_step": 1e6 * so / 50,
                                 "requests_per_s": wlo.n * 50 / so, "keep_fraction": kfo}
                 del plo, wlo
+            # the many-context workloads also against the oracle on all host cores (bounded samples)
+            others["C4"]["cpu_baseline_all_cores"] = oracle_all_cores("C4", {"n_epochs": 512, "per_epoch": 8192})
+            others["C5"]["cpu_baseline_all_cores"] = oracle_all_cores("C5", {"n_inst": 64, "per_inst": 65536})
         t_cpu, _ = time_oracle(wl, 2)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -196,13 +196,13 @@ class DevicePlan:
         self.total = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
         self.kept = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
         self.stream = torch.cuda.current_stream().cuda_stream
-        self.launches = pb.pard_plan_kernel_launches(wl.n, wl.n_ctx, self.S) + 2
+        self.launches = pb.pard_plan_kernel_launches(wl.n, wl.n_ctx, self.S) + 1   # + the goodput kernel
 
     def step(self, nowait=True):
         pb, wl = self.pb, self.wl
         pb.pard_plan(self.pipes, self.d_req, wl.n, self.d_state, wl.n_ctx,
                      pb.PARD_MODE_NOWAIT if nowait else 0, self.out, self.ws, stream=self.stream)
-        pb.pard_goodput(self.out.keep, self.out.seg_offsets, wl.n, wl.n_ctx, self.S, self.total,
+        pb.pard_goodput(None, self.out.seg_offsets, self.out.seg_kept, wl.n, wl.n_ctx, self.S, self.total,
                         self.kept, stream=self.stream)
 
     def status(self):

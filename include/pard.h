@@ -271,16 +271,23 @@ int pard_plan_host(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines
 
 /* Goodput counters (Sec. 5.1, Metrics): per ctx, the number of queued
  * requests and the number predicted to finish within their SLO (kept);
- * dropped = total - kept, drop rate = dropped / total.  Reads d_keep and
- * d_seg_offsets as produced by pard_plan; writes d_out_total[n_ctx] and
- * d_out_kept[n_ctx] (overwritten, not accumulated).  Enqueued on cuda_stream;
- * does not synchronise. */
+ * dropped = total - kept, drop rate = dropped / total.  Writes
+ * d_out_total[n_ctx] and d_out_kept[n_ctx] (overwritten, not accumulated)
+ * from pard_plan's outputs: d_seg_offsets always, and
+ *   - d_seg_kept, when given: the kept counts of a ctx's queues are added up
+ *     (one small kernel; d_keep is not read and may be NULL), or
+ *   - d_keep, when d_seg_kept is NULL: the keep flags of every ctx are counted
+ *     (16-byte aligned; a block-wide reduction and one atomic per block and
+ *     ctx), for callers that did not ask pard_plan for the per-queue counts.
+ * Both give the same numbers.  Enqueued on cuda_stream; does not synchronise. */
 int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets,
+                 const uint32_t* d_seg_kept,
                  uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                  int64_t* d_out_total, int64_t* d_out_kept, void* cuda_stream);
 
-/* Batch-wait estimate of the State Planner (Sec. 4.2, Batch wait estimation,
- * and Sec. 5.3 Overheads: M = 10,000 samples, refreshed off the critical path).
+/* Batch-wait estimate of the State Planner (Sec. 4.2, Batch wait estimation;
+ * its footnote gives the default M = 10,000 samples; Sec. 5.4, Overheads: the
+ * estimate is refreshed off the critical path).
  * For every ctx and every (stage k, downstream path P) slot of its pipeline,
  *   w[ctx][slot] = F^{-1}(lambda),   lambda = lambda_num / lambda_den in [0, 1],
  * where F is the empirical distribution of n_samples draws of the batch wait

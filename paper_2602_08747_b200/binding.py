@@ -93,7 +93,7 @@ def library() -> C.CDLL:
                      C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
         lib.pard_plan.argtypes = plan_args
         lib.pard_plan_host.argtypes = plan_args
-        lib.pard_goodput.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32,
+        lib.pard_goodput.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p]
         lib.pard_plan_static.argtypes = plan_args[:8] + [C.c_void_p]
         lib.pard_plan_status.argtypes = [C.c_void_p, C.c_void_p]
@@ -324,9 +324,9 @@ def pard_profile_end() -> dict:
     return {"n_samples": k.value, "ms": {names[i]: float(ms[i]) for i in range(PARD_N_PHASES)}}
 
 
-def pard_goodput(d_keep, d_seg_offsets, n: int, n_ctx: int, stage_stride: int, d_out_total,
+def pard_goodput(d_keep, d_seg_offsets, d_seg_kept, n: int, n_ctx: int, stage_stride: int, d_out_total,
                  d_out_kept, stream: int = 0, check: bool = True) -> int:
-    rc = library().pard_goodput(_ptr(d_keep), _ptr(d_seg_offsets), n, n_ctx, stage_stride,
+    rc = library().pard_goodput(_ptr(d_keep), _ptr(d_seg_offsets), _ptr(d_seg_kept), n, n_ctx, stage_stride,
                                 _ptr(d_out_total), _ptr(d_out_kept), stream or None)
     if check:
         _check(rc, "pard_goodput")

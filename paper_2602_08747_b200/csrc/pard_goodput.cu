@@ -111,17 +111,43 @@ k_goodput_count(const uint8_t* __restrict__ keep, const uint32_t* __restrict__ s
   }
 }
 
+/* Both counters of a ctx from the per-queue figures the planner has already produced: the
+ * ctx's first and last position, and the kept counts of its queues added up.  One warp per
+ * ctx, lanes over its queues; the keep flags are not read. */
+__global__ void __launch_bounds__(kThreads)
+k_goodput_from_queues(const uint32_t* __restrict__ seg_off, const uint32_t* __restrict__ seg_kept,
+                      uint32_t n_ctx, uint32_t S, long long* __restrict__ out_total,
+                      long long* __restrict__ out_kept) {
+  pdl_wait();
+  const uint32_t c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (c >= n_ctx) return;                          /* whole warps leave together */
+  unsigned long long sum = 0;
+  for (uint32_t k = lane; k < S; k += 32) sum += seg_kept[(size_t)c * S + k];
+  for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) {
+    out_total[c] = (long long)seg_off[(size_t)(c + 1) * S] - (long long)seg_off[(size_t)c * S];
+    out_kept[c] = (long long)sum;
+  }
+}
+
 }  // namespace
 
-extern "C" int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets, uint64_t n,
+extern "C" int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets,
+                            const uint32_t* d_seg_kept, uint64_t n,
                             uint32_t n_ctx, int32_t stage_stride, int64_t* d_out_total,
                             int64_t* d_out_kept, void* cuda_stream) {
   if (!d_seg_offsets || !d_out_total || !d_out_kept || n_ctx < 1 || stage_stride < 1) return PARD_EINVAL;
-  if (n > 0 && (!d_keep || ((uintptr_t)d_keep & 15))) return PARD_EINVAL;
+  if (!d_seg_kept && n > 0 && (!d_keep || ((uintptr_t)d_keep & 15))) return PARD_EINVAL;
   if (n >= PARD_MAX_REQUESTS || stage_stride > PARD_MAX_STAGES ||
       (uint64_t)n_ctx * (uint64_t)stage_stride > PARD_MAX_SEGMENTS)
     return PARD_ERANGE;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (d_seg_kept) {
+    launch_pdl(k_goodput_from_queues, (n_ctx + kThreads / 32 - 1) / (kThreads / 32), kThreads, 0, stream, d_seg_offsets,
+               d_seg_kept, n_ctx, (uint32_t)stage_stride, (long long*)d_out_total, (long long*)d_out_kept);
+    PARD_CUDA_OK(cudaGetLastError());
+    return PARD_OK;
+  }
   launch_pdl(k_goodput_init, (n_ctx + 255) / 256, 256, 0, stream, d_seg_offsets, n_ctx, (uint32_t)stage_stride,
                                                           (long long*)d_out_total, (long long*)d_out_kept);
   if (n > 0) {

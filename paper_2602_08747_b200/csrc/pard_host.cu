@@ -110,7 +110,9 @@ extern "C" int pard_plan_host(const pard_pipeline_t* const* pipelines, uint32_t 
   dout.d_seg_offsets = out->d_seg_offsets ? (uint32_t*)(ws + L.seg_off) : nullptr;
   dout.d_seg_kept = out->d_seg_kept ? (uint32_t*)(ws + L.seg_kept) : nullptr;
 
-  rc = pard_plan(pipelines, n_pipelines, d_req, n, &d, n_ctx, mode, &dout, ws + L.plan,
+  /* this call drains the stream anyway, so the status is always read here: PARD_MODE_NOWAIT would
+   * only hide a device-detected error behind the downloads */
+  rc = pard_plan(pipelines, n_pipelines, d_req, n, &d, n_ctx, mode & ~PARD_MODE_NOWAIT, &dout, ws + L.plan,
                  L.plan_bytes, cuda_stream);
   if (rc != PARD_OK) return rc;
 

@@ -12,6 +12,7 @@
  *             position c, estimate, keep flag, compaction, per-segment counts
  */
 #include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <mutex>
 
@@ -50,17 +51,17 @@ struct PlanHeader {
   uint32_t keybits;           /* segment bits + dbits                      */
   uint32_t npass;             /* radix passes that run                     */
   unsigned long long span_max;
+  unsigned long long win_total;   /* window-table entries asked for (64 bits: 2^24 queues of up to 4,097 entries) */
   uint32_t ticket[kMaxPasses + 1];
   uint32_t wide;              /* 1: segment, deadline and index bits exceed 64; nothing is sorted */
   uint32_t use_scan;          /* 1: too many batch windows for the window tables: decide by scanning */
-  uint32_t win_total;         /* window-table entries handed out */
   uint32_t aborted;           /* 1: a bounded wait ran out; the sort is incomplete and every later kernel returns */
   uint32_t big_total;         /* window-table entries that belong to long queues */
   uint32_t agg_done;          /* blocks of k_tile_agg that have stored their aggregates */
   uint32_t seg_done;          /* blocks of k_seg_const that have stored their constants */
   uint32_t unsorted;          /* 1: some request's ctx is smaller than its predecessor's */
   uint32_t ctx_too_big;       /* 1: some ctx holds more requests than one sort tile */
-  uint32_t pad[64 - 15 - (kMaxPasses + 1)];
+  uint32_t pad[64 - 16 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
@@ -1497,8 +1498,9 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
         hdr->use_scan = 1;
       } else {
         w = (uint32_t)nb + 1;
-        first = atomicAdd(&hdr->win_total, w);
-        if (first + w > capacity) { hdr->use_scan = 1; w = 0; }
+        const unsigned long long at = atomicAdd(&hdr->win_total, (unsigned long long)w);
+        if (at + w > (unsigned long long)capacity) { hdr->use_scan = 1; w = 0; }
+        else first = (uint32_t)at;
       }
     }
   }
@@ -1579,11 +1581,12 @@ k_seg_win_many(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
     const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= (uint32_t)o) incl += t;
   }
-  uint32_t base = 0;
-  if (lane == 31 && incl) base = atomicAdd(&hdr->win_total, incl);
+  unsigned long long base = 0;
+  if (lane == 31 && incl) base = atomicAdd(&hdr->win_total, (unsigned long long)incl);
   base = __shfl_sync(0xffffffffu, base, 31);
-  uint32_t first = base + incl - w;
-  if (w && first + w > capacity) { hdr->use_scan = 1; w = 0; }
+  const unsigned long long first64 = base + incl - w;        /* 64 bits: the counter may pass 2^32 on legal input */
+  if (w && first64 + w > (unsigned long long)capacity) { hdr->use_scan = 1; w = 0; }
+  const uint32_t first = w ? (uint32_t)first64 : 0u;
   if (mine && !high_first) { win_off[s] = w ? first : 0u; win_cnt[s] = w; }
   for (uint32_t e = 0; e < w; ++e) win_own[first + e] = s;
   if (w && end - lo > kWinLongQueue) {           /* long queue: list its entries for the warp-wide search */
@@ -1652,7 +1655,8 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
   const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
   /* entries of short queues: one lane each, plain binary search */
   {
-    const uint32_t total = hdr->win_total, step = gridDim.x * blockDim.x;
+    /* without use_scan every request for entries was granted, so the counter is within the table */
+    const uint32_t total = (uint32_t)hdr->win_total, step = gridDim.x * blockDim.x;
     for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += step) {
       const uint32_t s = win_own[e];
       uint32_t lo = seg_off[s], hi = seg_off[s + 1];
@@ -1721,7 +1725,8 @@ __global__ void __launch_bounds__(kDecThreads, 8)
 k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
              const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-             const uint32_t* __restrict__ win_off, const WinEntry* __restrict__ wtab,
+             const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
+             const WinEntry* __restrict__ wtab,
              uint8_t* __restrict__ out_keep, long long* __restrict__ out_est,
              uint32_t* __restrict__ out_perm, uint32_t* __restrict__ kept_tmp,
              uint32_t* __restrict__ seg_kept) {
@@ -1741,7 +1746,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
   }
   uint32_t cur_seg = (uint32_t)(e[0] >> T.kshift);
   PardSegConst K = ktab[cur_seg];
-  uint32_t sstart = seg_off[cur_seg], send = seg_off[cur_seg + 1], woff = win_off[cur_seg];
+  uint32_t sstart = seg_off[cur_seg], send = seg_off[cur_seg + 1], woff = win_off[cur_seg], wcnt = win_cnt[cur_seg];
   const bool narrow = T.narrow && (K.narrow & (kSegNarrow | kSegNoStage)) == kSegNarrow && full &&
                       cur_seg == (uint32_t)(e[kDecItems - 1] >> T.kshift);
 
@@ -1766,6 +1771,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
           sstart = seg_off[sg];
           send = seg_off[sg + 1];
           woff = win_off[sg];
+          wcnt = win_cnt[sg];
         }
         X = HF ? slack_of((e[i] >> T.ibits) & T.dmask, K) : (long long)((e[i] >> T.ibits) & T.dmask) - K.A_rel;
       }
@@ -1776,7 +1782,17 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
         ahead = min(r, woff);
         c = RAW ? r : ahead;
       } else if (X >= 0) {                            /* window b of the request and its table entry */
-        const uint32_t b = (uint32_t)win_of((unsigned long long)X, K);
+        const unsigned long long b64 = win_of((unsigned long long)X, K);
+        /* The queue's table has an entry for every window up to its latest deadline's.  A queue
+         * without a table (input errors: a stage its pipeline lacks, constants left at their
+         * defaults) must not index one: its requests count as dropped, the call reports PARD_EDATA. */
+        if (b64 >= (unsigned long long)wcnt) {
+          set_status(T.hdr, PARD_EDATA);
+          est[i] = K.A;
+          if ((uint32_t)j + 1 == send) seg_kept[cur_seg] = 0;
+          continue;
+        }
+        const uint32_t b = (uint32_t)b64;
         u = win_u(b, K.cap);
         const WinEntry w = wtab[woff + b];
         if (RAW) {
@@ -1855,7 +1871,8 @@ constexpr int kEventsPerSample = PARD_N_PHASES + 1;
 static_assert(PARD_N_PHASES == 4 + kMaxPasses + 3, "phase list");
 struct Profiler {
   std::mutex mu;
-  bool on = false, coarse = false;
+  std::atomic<bool> on{false};       /* read without the lock by every pard_plan call */
+  bool coarse = false;
   uint32_t every = 1, max_samples = 0, calls = 0, n_samples = 0;
   std::vector<cudaEvent_t> ev;
 };
@@ -1865,8 +1882,9 @@ constexpr int kPhaseTables = 4 + kMaxPasses;       /* "tables", then "decide", "
 
 /* events of this call if it is a sampled one, else nullptr */
 cudaEvent_t* profile_acquire(bool* coarse) {
+  if (!g_prof.on.load(std::memory_order_acquire)) return nullptr;   /* the usual case: no lock taken */
   std::lock_guard<std::mutex> lock(g_prof.mu);
-  if (!g_prof.on) return nullptr;
+  if (!g_prof.on.load(std::memory_order_relaxed)) return nullptr;
   *coarse = g_prof.coarse;
   uint32_t call = g_prof.calls++;
   if (call % g_prof.every != 0 || g_prof.n_samples >= g_prof.max_samples) return nullptr;
@@ -1876,17 +1894,18 @@ cudaEvent_t* profile_acquire(bool* coarse) {
 /* the sort pass needs more dynamic shared memory than the default limit: opt in once per device */
 int allow_sort_smem(int dev) {
   static std::mutex mu;
-  static bool done[64];
-  std::lock_guard<std::mutex> lock(mu);
+  static std::atomic<bool> done[64];
   if (dev < 0 || dev >= 64) return PARD_ERANGE;
-  if (!done[dev]) {
+  if (done[dev].load(std::memory_order_acquire)) return PARD_OK;    /* every call but the first on a device */
+  std::lock_guard<std::mutex> lock(mu);
+  if (!done[dev].load(std::memory_order_relaxed)) {
     PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
     PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
     PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_local, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
-    done[dev] = true;
+    done[dev].store(true, std::memory_order_release);
   }
   return PARD_OK;
 }
@@ -2069,7 +2088,7 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
                           : (state->d_priority ? k_decide_win<false, true> : k_decide_win<false, false>);
-    launch_pdl(decide_win, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, wtab,
+    launch_pdl(decide_win, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, win_cnt, wtab,
                out->d_keep, est, out->d_perm, tmp, seg_kept);
     /* fallback when a queue has too many batch windows: the same decision by scanning (these two
      * return at once otherwise) */
@@ -2134,7 +2153,7 @@ extern "C" int pard_profile_begin(uint32_t every, uint32_t max_samples) {
   every &= ~PARD_PROFILE_COARSE;
   if (every < 1 || max_samples < 1 || max_samples > 65536) return PARD_EINVAL;
   std::lock_guard<std::mutex> lock(g_prof.mu);
-  if (g_prof.on) return PARD_EINVAL;
+  if (g_prof.on.load()) return PARD_EINVAL;
   g_prof.ev.assign((size_t)max_samples * kEventsPerSample, nullptr);
   for (auto& e : g_prof.ev)
     if (cudaEventCreate(&e) != cudaSuccess) {
@@ -2147,13 +2166,13 @@ extern "C" int pard_profile_begin(uint32_t every, uint32_t max_samples) {
   g_prof.max_samples = max_samples;
   g_prof.calls = 0;
   g_prof.n_samples = 0;
-  g_prof.on = true;
+  g_prof.on.store(true, std::memory_order_release);
   return PARD_OK;
 }
 
 extern "C" int pard_profile_end(float* ms_sum, uint32_t* n_samples) {
   std::lock_guard<std::mutex> lock(g_prof.mu);
-  if (!g_prof.on) return PARD_EINVAL;
+  if (!g_prof.on.load()) return PARD_EINVAL;
   int rc = PARD_OK;
   if (ms_sum) for (int i = 0; i < PARD_N_PHASES; ++i) ms_sum[i] = 0.f;
   for (uint32_t s = 0; s < g_prof.n_samples; ++s) {
@@ -2171,7 +2190,7 @@ extern "C" int pard_profile_end(float* ms_sum, uint32_t* n_samples) {
   if (n_samples) *n_samples = g_prof.n_samples;
   for (auto& e : g_prof.ev) cudaEventDestroy(e);
   g_prof.ev.clear();
-  g_prof.on = false;
+  g_prof.on.store(false, std::memory_order_release);
   return rc;
 }
 

@@ -68,7 +68,7 @@ class Replay:
         pb.pard_update_queue_delay(self.n_ctx, self.S, d_now_us, self.sample_time, self.sample_delay,
                                    self.M, self.window, nw, st.q_us, self.ws_q, stream=self.stream)
         pb.pard_plan(self.pipes, d_requests, n, st, self.n_ctx, nw, self.out, self.ws_plan, stream=self.stream)
-        pb.pard_goodput(self.out.keep, self.out.seg_offsets, n, self.n_ctx, self.S, d_total_row, d_kept_row,
+        pb.pard_goodput(None, self.out.seg_offsets, self.out.seg_kept, n, self.n_ctx, self.S, d_total_row, d_kept_row,
                         stream=self.stream)
         pb.pard_advance_state(self.pipes, self.poc, self.n_ctx, self.S, d_now_us, st.batch, st.workers,
                               self.out.seg_kept, st.free_at_us, self.sample_time, self.sample_delay, self.M,

@@ -25,11 +25,16 @@ def run_library(wl, mode=0, check=True):
         return rc, None
     total = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
     kept = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)
-    pb.pard_goodput(out.keep, out.seg_offsets, wl.n, wl.n_ctx, S, total, kept, stream=stream)
+    # the counters both ways: from the per-queue kept counts, and by counting the keep flags
+    pb.pard_goodput(None, out.seg_offsets, out.seg_kept, wl.n, wl.n_ctx, S, total, kept, stream=stream)
+    total2, kept2 = torch.empty_like(total), torch.empty_like(kept)
+    pb.pard_goodput(out.keep, out.seg_offsets, None, wl.n, wl.n_ctx, S, total2, kept2, stream=stream)
     torch.cuda.synchronize()
     res = pb.out_to_numpy(out, wl.n)
     res["ctx_total"] = total.cpu().numpy()
     res["ctx_kept"] = kept.cpu().numpy()
+    res["ctx_total_from_flags"] = total2.cpu().numpy()
+    res["ctx_kept_from_flags"] = kept2.cpu().numpy()
     for p in pipes:
         p.free()
     return rc, res
@@ -40,6 +45,9 @@ KEYS = ["seg_offsets", "perm", "keep", "est_us", "n_kept", "kept_idx", "seg_kept
 
 def assert_identical(got, want):
     """Bit-exact comparison of every output (all of them are integers)."""
+    for k in ("ctx_total", "ctx_kept"):           # the second way of counting, against the oracle too
+        if k + "_from_flags" in got:
+            assert np.array_equal(got[k + "_from_flags"], want[k]), k + "_from_flags"
     for k in KEYS:
         g, w = got[k], want[k]
         if isinstance(w, (int, np.integer)):

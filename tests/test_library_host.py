@@ -156,7 +156,7 @@ def test_plan_argument_checks_happen_before_any_launch():
     bad = pb.QueueStateArrays(2, 1, None, dummy, dummy, dummy).c_struct()
     assert lib.pard_plan(hs, 1, None, 0, C.byref(bad), 1, 0, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
     assert lib.pard_plan(hs, 1, None, 5, C.byref(cst), 1, 0, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
-    assert lib.pard_goodput(None, None, 0, 1, 2, None, None, None) == pb.PARD_EINVAL
+    assert lib.pard_goodput(None, None, None, 0, 1, 2, None, None, None) == pb.PARD_EINVAL
 
 
 def test_estimate_w_argument_checks_happen_before_any_launch():

@@ -160,6 +160,13 @@ def test_device_detected_errors():
     r["stage"][7] = 2
     rc, _ = run_library(inputs.Workload("bad", [p], r, util.state(1, 3, 1, 10, 1), 1), check=False)
     assert rc == pb.PARD_EDATA
+    # the same with a deadline far from the queue's start: the request's batch window (offset 2,500
+    # with the default duration of 1) lies beyond every window table (1,133 entries here); it must be
+    # reported, not looked up (the offset stays below n, i.e. inside the caller's workspace)
+    r = good.copy()
+    r["stage"][2500] = 2
+    rc, _ = run_library(inputs.Workload("bad", [p], r, util.state(1, 3, 1, 10, 1), 1), check=False)
+    assert rc == pb.PARD_EDATA
     # the context still works afterwards
     both(inputs.Workload("ok", [p], good, st, 1))
 

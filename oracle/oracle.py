@@ -55,9 +55,14 @@ def lib():
         _lib.oracle_slot_base.argtypes = [C.c_void_p, C.c_int32]
         _lib.oracle_lsub.restype = C.c_int64
         _lib.oracle_lsub.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib.oracle_lsub_masked.restype = C.c_int64
+        _lib.oracle_lsub_masked.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint16]
         _lib.oracle_plan.restype = C.c_int
         _lib.oracle_plan.argtypes = ([C.c_void_p, C.c_int32, C.c_void_p, C.c_uint64,
                                       C.c_void_p, C.c_uint32, C.c_uint32] + [C.c_void_p] * 9)
+        _lib.oracle_plan_policy.restype = C.c_int
+        _lib.oracle_plan_policy.argtypes = ([C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_uint64,
+                                             C.c_void_p, C.c_uint32, C.c_uint32] + [C.c_void_p] * 9)
         _lib.oracle_estimate_w.restype = C.c_int
         _lib.oracle_estimate_w.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_uint32, C.c_int32, C.c_int32,
                                            C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_void_p]
@@ -120,6 +125,14 @@ def lsub(p, stage: int, batch_row, q_row, w_row=None) -> int:
     cp = _c_pipeline(p, k)
     return int(lib().oracle_lsub(C.addressof(cp), stage, k.add(batch_row, np.int32),
                                  k.add(q_row, np.int64), k.add(w_row, np.int64)))
+
+
+def lsub_masked(p, stage: int, batch_row, q_row, w_row, mask: int) -> int:
+    """L_sub over the downstream paths whose bit is set in `mask` (0 = all); -1 if none exists."""
+    k = _Keep()
+    cp = _c_pipeline(p, k)
+    return int(lib().oracle_lsub_masked(C.addressof(cp), stage, k.add(batch_row, np.int32),
+                                        k.add(q_row, np.int64), k.add(w_row, np.int64), mask))
 
 
 def estimate_w(pipelines, pipeline_of_ctx, n_ctx: int, stage_stride: int, slot_stride: int, wait_samples,
@@ -194,8 +207,12 @@ def advance_state(pipelines, pipeline_of_ctx, n_ctx: int, stage_stride: int, now
         raise ValueError("oracle_advance_state: bad input")
 
 
-def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:
-    """Runs the oracle planner; returns a dict of numpy outputs."""
+MODE_RAW, MODE_PATH_MASK, MODE_FCFS, MODE_NEXUS, MODE_CLIPPER = 1, 16, 32, 64, 128
+
+
+def plan(pipelines, requests, state, n_ctx: int, mode: int = 0, arrivals=None) -> dict:
+    """Runs the oracle planner; returns a dict of numpy outputs.  `arrivals` (records of
+    two int64: arrive_us, slo_us) is needed by MODE_CLIPPER only."""
     k = _Keep()
     cps = (_Pipeline * len(pipelines))(*[_c_pipeline(p, k) for p in pipelines])
     req = np.ascontiguousarray(requests)
@@ -216,7 +233,11 @@ def plan(pipelines, requests, state, n_ctx: int, mode: int = 0) -> dict:
         "seg_kept": np.zeros(n_ctx * S, np.uint32),
         "ctx_total": np.zeros(n_ctx, np.int64), "ctx_kept": np.zeros(n_ctx, np.int64),
     }
-    rc = lib().oracle_plan(C.addressof(cps), len(pipelines), req.ctypes.data, n,
+    arr = None
+    if arrivals is not None:
+        arr = np.ascontiguousarray(arrivals)
+        assert arr.dtype.itemsize == 16 and arr.shape[0] == n
+    rc = lib().oracle_plan_policy(C.addressof(cps), len(pipelines), req.ctypes.data, _ptr(arr), n,
                            C.addressof(cst), n_ctx, mode,
                            *[out[key].ctypes.data for key in
                              ("keep", "est_us", "perm", "kept_idx", "n_kept",

@@ -18,6 +18,8 @@
  *   Rule:   drop when the estimate exceeds the latency objective (Sec. 5.3)
  *   Counts: goodput / drop rate                                 (Sec. 5.1)
  *   w_k:    quantile lambda of the sampled aggregated batch wait  (Sec. 4.2)
+ *   Other rules on the same queues: dynamic-path requests (Sec. 5.2), arrival
+ *           order (Table 1, Sec. 5.3), Nexus and Clipper++ (Sec. 5.1 Baseline)
  *
  * Readings where the paper is silent (each also listed in the design notes):
  *   - Snapshot: the Request Broker loop is run over the whole queue at the
@@ -116,6 +118,42 @@ extern "C" int64_t oracle_lsub(const oracle_pipeline_t* p, int32_t stage,
 
 namespace {
 
+/* As walk(), but a complete path counts only if the bit of its rank among the
+ * stage's downstream paths (`rank` runs 0, 1, ... in lexicographic order) is
+ * set in `mask`.  Returns -1 when no path below `stage` counts (every path sum
+ * is at least one execution duration, so -1 cannot be a sum). */
+int64_t walk_masked(const oracle_pipeline_t* p, int32_t stage, int64_t acc,
+                    const int32_t* batch_row, const int64_t* q_row, const int64_t* w_row,
+                    int64_t slot_base, int64_t* rank, uint16_t mask) {
+  acc += q_row[stage] + profile_at(p, stage, batch_row[stage]);
+  std::vector<int32_t> s = successors_ascending(p, stage);
+  if (s.empty()) {
+    int64_t r = *rank;
+    *rank += 1;
+    if (r >= 16 || !((mask >> r) & 1)) return -1;           /* not a path this request can take */
+    return acc + (w_row ? w_row[slot_base + r] : 0);
+  }
+  int64_t best = -1;
+  for (int32_t j : s) best = std::max(best, walk_masked(p, j, acc, batch_row, q_row, w_row, slot_base, rank, mask));
+  return best;
+}
+
+}  // namespace
+
+extern "C" int64_t oracle_lsub_masked(const oracle_pipeline_t* p, int32_t stage,
+                                      const int32_t* batch_row, const int64_t* q_row,
+                                      const int64_t* w_row, uint16_t mask) {
+  if (mask == 0) return oracle_lsub(p, stage, batch_row, q_row, w_row);   /* path unknown: all of them */
+  std::vector<int32_t> s = successors_ascending(p, stage);
+  if (s.empty()) return 0;
+  int64_t rank = 0, best = -1;
+  for (int32_t j : s)
+    best = std::max(best, walk_masked(p, j, 0, batch_row, q_row, w_row, oracle_slot_base(p, stage), &rank, mask));
+  return best;
+}
+
+namespace {
+
 /* splitmix64 (Steele, Lea, Flood: "Fast splittable pseudorandom number generators") */
 uint64_t splitmix64(uint64_t x) {
   uint64_t z = x + 0x9E3779B97F4A7C15ull;
@@ -182,6 +220,23 @@ extern "C" int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelin
                            uint32_t* kept_idx, uint64_t* n_kept,
                            uint32_t* seg_offsets, uint32_t* seg_kept,
                            int64_t* ctx_total, int64_t* ctx_kept) {
+  return oracle_plan_policy(pipelines, n_pipelines, requests, nullptr, n, st, n_ctx, mode, keep, est_us,
+                            perm, kept_idx, n_kept, seg_offsets, seg_kept, ctx_total, ctx_kept);
+}
+
+extern "C" int oracle_plan_policy(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                                  const oracle_request_t* requests, const oracle_arrival_t* arrivals,
+                                  uint64_t n, const oracle_state_t* st, uint32_t n_ctx, uint32_t mode,
+                                  uint8_t* keep, int64_t* est_us, uint32_t* perm,
+                                  uint32_t* kept_idx, uint64_t* n_kept,
+                                  uint32_t* seg_offsets, uint32_t* seg_kept,
+                                  int64_t* ctx_total, int64_t* ctx_kept) {
+  const bool nexus = mode & ORACLE_MODE_NEXUS, clipper = mode & ORACLE_MODE_CLIPPER;
+  const bool masked = mode & ORACLE_MODE_PATH_MASK;
+  const bool arrival_order = (mode & ORACLE_MODE_FCFS) || nexus || clipper;
+  if (nexus && clipper) return -1;
+  if ((nexus || clipper) && (masked || (mode & 1u))) return -1;
+  if (clipper && n > 0 && !arrivals) return -1;
   const int64_t S = st->stage_stride;
   /* one queue per (ctx, stage), filled in arrival (index) order */
   std::vector<std::vector<uint32_t>> queue((size_t)n_ctx * S);
@@ -226,9 +281,11 @@ extern "C" int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelin
       /* the remaining budget of a request is its deadline minus the same `now`
        * for the whole queue, so budget order is deadline order.
        * low budget first: smallest deadline first; high budget first: largest
-       * deadline first; ties in index order either way */
+       * deadline first; ties in index order either way.  Arrival order (PARD-FCFS,
+       * Nexus, Clipper++) leaves the queue as it was filled. */
       bool high_first = st->priority && st->priority[(size_t)c * S + k] != 0;
-      if (high_first)
+      if (arrival_order) {
+      } else if (high_first)
         std::stable_sort(qk.begin(), qk.end(), [&](uint32_t a, uint32_t b) {
           return requests[a].deadline_us > requests[b].deadline_us;
         });
@@ -238,21 +295,76 @@ extern "C" int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelin
         });
 
       int64_t kept = 0, raw = 0;
-      for (uint32_t i : qk) {                    /* the Request Broker, one request at a time */
-        int64_t ahead = (mode & 1u) ? raw : kept;
-        int64_t t_e = base + (ahead / cap) * d;  /* its batch starts when the previous one ends */
-        int64_t est = t_e + d + lsub;            /* t_s + L of Eq. 3 */
-        bool k_ = est <= requests[i].deadline_us;
-        if (keep) keep[pos] = k_ ? 1 : 0;
-        if (est_us) est_us[pos] = est;
-        if (perm) perm[pos] = i;
-        if (k_) {
-          if (kept_idx) kept_idx[kept_all] = i;
-          ++kept_all;
-          ++kept;
+      if (nexus) {
+        /* Sec. 5.1 Baseline, Nexus: a window of one batch round slides over the queue in
+         * arrival order; t is when the batch being formed would start */
+        int64_t t = base;
+        size_t window_start = 0;                 /* first request of the window being tried */
+        std::vector<uint8_t> in_batch(qk.size(), 0);
+        std::vector<int64_t> tested_end(qk.size(), 0);
+        for (size_t r = 0; r < qk.size(); ++r) {
+          const bool fits = t + d <= requests[qk[r]].deadline_us;   /* enough budget left for this module */
+          tested_end[r] = t + d;
+          if (!fits) {
+            window_start = r + 1;                /* no window that holds r can be the batch: all before it go too */
+          } else if ((int64_t)(r - window_start + 1) == cap) {
+            for (size_t j = window_start; j <= r; ++j) in_batch[j] = 1;
+            t += d;                              /* the next batch starts when this one ends */
+            window_start = r + 1;
+          }
         }
-        ++raw;
-        ++pos;
+        /* what is left behind the last full batch fits and runs as a partly filled batch */
+        for (size_t j = window_start; j < qk.size(); ++j) in_batch[j] = 1;
+        for (size_t r = 0; r < qk.size(); ++r) {
+          if (keep) keep[pos] = in_batch[r];
+          if (est_us) est_us[pos] = tested_end[r];
+          if (perm) perm[pos] = qk[r];
+          if (in_batch[r]) {
+            if (kept_idx) kept_idx[kept_all] = qk[r];
+            ++kept_all;
+            ++kept;
+          }
+          ++raw;
+          ++pos;
+        }
+      } else {
+        int64_t dsum = 0;                        /* Clipper++: sum of d_i over the pipeline's modules */
+        if (clipper) for (int32_t i = 0; i < p->n_stages; ++i) {
+          if (batch_row[i] < 1 || batch_row[i] > p->bmax[i]) return -1;
+          dsum += profile_at(p, i, batch_row[i]);
+        }
+        for (uint32_t i : qk) {                    /* the Request Broker, one request at a time */
+          int64_t ahead = (mode & 1u) ? raw : kept;
+          int64_t t_e = base + (ahead / cap) * d;  /* its batch starts when the previous one ends */
+          int64_t est;
+          bool k_;
+          if (clipper) {
+            /* Sec. 5.1 Baseline, Clipper++: SLO_k = SLO * d_k / sum d_i; dropped iff the request has
+             * already used up that share when its inference would start */
+            if (arrivals[i].slo_us < 0) return -1;
+            int64_t share = (int64_t)(((__int128)arrivals[i].slo_us * d) / dsum);
+            est = t_e + d;
+            k_ = t_e - arrivals[i].arrive_us <= share;
+          } else {
+            int64_t lsub_i = lsub;
+            if (masked) {
+              lsub_i = oracle_lsub_masked(p, k, batch_row, q_row, w_row, requests[i].flags);
+              if (lsub_i < 0) return -1;
+            }
+            est = t_e + d + lsub_i;                /* t_s + L of Eq. 3 */
+            k_ = est <= requests[i].deadline_us;
+          }
+          if (keep) keep[pos] = k_ ? 1 : 0;
+          if (est_us) est_us[pos] = est;
+          if (perm) perm[pos] = i;
+          if (k_) {
+            if (kept_idx) kept_idx[kept_all] = i;
+            ++kept_all;
+            ++kept;
+          }
+          ++raw;
+          ++pos;
+        }
       }
       if (seg_kept) seg_kept[(size_t)c * S + k] = (uint32_t)kept;
       total_c += raw;

@@ -67,8 +67,54 @@ int64_t oracle_lsub(const oracle_pipeline_t* p, int32_t stage,
                     const int32_t* batch_row, const int64_t* q_row,
                     const int64_t* w_row);
 
+/* L_sub for a request whose downstream path is (partly) known -- the dynamic-path
+ * DAGs of Sec. 5.2, where a request takes one of several branches: the maximum
+ * is taken only over the stage's downstream paths j (in the lexicographic
+ * enumeration, j = 0, 1, ...) whose bit j is set in `mask`.  mask = 0 means
+ * "unknown": all paths, i.e. oracle_lsub.  A sink gives 0 whatever the mask.
+ * Returns -1 when the mask selects no existing path. */
+int64_t oracle_lsub_masked(const oracle_pipeline_t* p, int32_t stage,
+                           const int32_t* batch_row, const int64_t* q_row,
+                           const int64_t* w_row, uint16_t mask);
+
+/* Decision rules and orders beside the paper's own (Sec. 5.1 Baseline, Sec. 5.2
+ * dynamic paths, Table 1 / Sec. 5.3 FCFS), selected by bits of `mode`:
+ *   ORACLE_MODE_PATH_MASK  request.flags is the path mask of oracle_lsub_masked
+ *   ORACLE_MODE_FCFS       queues are served in arrival order, which is the order
+ *                          of the request array (index order), not budget order;
+ *                          estimate and drop rule unchanged  (PARD-FCFS)
+ *   ORACLE_MODE_NEXUS      Nexus' reactive rule, arrival order: the queue is scanned
+ *                          with a window of one batch round (B*m requests); the
+ *                          batch is the first window whose requests can all finish
+ *                          the CURRENT module by their deadline if the batch starts
+ *                          when the previous one ends; every request before that
+ *                          window is dropped; the scan resumes behind the window one
+ *                          execution duration later.  A last window that the queue
+ *                          cannot fill is run as it is.  est = end of the batch the
+ *                          request was tested against.
+ *   ORACLE_MODE_CLIPPER    Clipper++: arrival order; module k gets the share
+ *                          SLO_k = floor(SLO * d_k / sum_i d_i) of the request's
+ *                          objective (d_i at the current batch sizes, all stages of
+ *                          the pipeline); a request is dropped iff, when its batch
+ *                          starts, it has already spent more than SLO_k in the
+ *                          module: start - arrive > SLO_k.  Needs `arrivals`.
+ *                          est = end of that batch.
+ * NEXUS and CLIPPER exclude each other, PATH_MASK and bit 0. */
+#define ORACLE_MODE_PATH_MASK 16u
+#define ORACLE_MODE_FCFS      32u
+#define ORACLE_MODE_NEXUS     64u
+#define ORACLE_MODE_CLIPPER   128u
+
+/* when the request reached its current module, and its end-to-end objective */
+typedef struct oracle_arrival {
+  int64_t arrive_us;
+  int64_t slo_us;
+} oracle_arrival_t;
+
 /* The planner.  mode bit 0: 0 = a dropped request takes no batch slot,
- * 1 = every request ahead takes one.  Outputs (any may be NULL):
+ * 1 = every request ahead takes one; further bits as above (`arrivals` is
+ * [n], needed by ORACLE_MODE_CLIPPER only; oracle_plan passes NULL).
+ * Outputs (any may be NULL):
  *   keep[n], est_us[n], perm[n]      in service order
  *   kept_idx[n], *n_kept             original indices of kept requests
  *   seg_offsets[n_ctx*stage_stride+1], seg_kept[n_ctx*stage_stride]
@@ -81,6 +127,13 @@ int oracle_plan(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
                 uint32_t* kept_idx, uint64_t* n_kept,
                 uint32_t* seg_offsets, uint32_t* seg_kept,
                 int64_t* ctx_total, int64_t* ctx_kept);
+int oracle_plan_policy(const oracle_pipeline_t* pipelines, int32_t n_pipelines,
+                       const oracle_request_t* requests, const oracle_arrival_t* arrivals,
+                       uint64_t n, const oracle_state_t* state, uint32_t n_ctx, uint32_t mode,
+                       uint8_t* keep, int64_t* est_us, uint32_t* perm,
+                       uint32_t* kept_idx, uint64_t* n_kept,
+                       uint32_t* seg_offsets, uint32_t* seg_kept,
+                       int64_t* ctx_total, int64_t* ctx_kept);
 
 /* Batch-wait estimate w = F^{-1}(lambda) of the State Planner (Sec. 4.2, Batch
  * wait estimation): for every (ctx, stage k, downstream path P) slot, draw M

@@ -24,6 +24,11 @@ REQUEST_DTYPE = np.dtype(
      "formats": ["<i8", "<u4", "<u2", "<u2"],
      "offsets": [0, 8, 12, 14], "itemsize": 16})
 
+# when a request reached its current module, and its end-to-end objective (only
+# the Clipper++ comparison rule reads these)
+ARRIVAL_DTYPE = np.dtype({"names": ["arrive_us", "slo_us"], "formats": ["<i8", "<i8"],
+                          "offsets": [0, 8], "itemsize": 16})
+
 
 @dataclass
 class Pipeline:

@@ -53,6 +53,14 @@ def requests(deadline, stage=0, ctx=0):
     return r
 
 
+def arrivals(arrive, slo):
+    arrive = np.asarray(arrive, dtype=np.int64)
+    a = np.zeros(len(arrive), dtype=inputs.ARRIVAL_DTYPE)
+    a["arrive_us"] = arrive
+    a["slo_us"] = slo
+    return a
+
+
 def explicit_paths(p, stage):
     """Every downstream path of `stage` as a tuple of stage ids, sorted
     lexicographically (written independently of the oracle and the library)."""

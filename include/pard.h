@@ -116,7 +116,8 @@ typedef struct pard_request {
   int64_t  deadline_us;   /* in [0, 2^60)                                            */
   uint32_t ctx;           /* < n_ctx                                                 */
   uint16_t stage;         /* stage whose queue holds the request, < n_stages         */
-  uint16_t flags;         /* reserved, ignored                                       */
+  uint16_t flags;         /* ignored unless PARD_MODE_PATH_MASK: then the downstream
+                             paths the request will take (0 = unknown, all paths)   */
 } pard_request_t;         /* 16 bytes, 16-byte aligned arrays                        */
 
 /* Runtime state the State Planner monitors and synchronises (Sec. 4.1, steps
@@ -178,6 +179,52 @@ typedef struct pard_plan_out {
                                    block by block (requests grouped by ctx, no ctx above
                                    8,192 requests) have no such wait and are unaffected */
 
+/* Other decision orders and rules on the same queues, for comparison with the
+ * planner's own (which stays the default).  Their thresholds do not rise along
+ * a queue, so each queue is walked in order by one warp (32 requests per step)
+ * instead of being decided request by request; they cost a few times the
+ * default rule on long queues.  None combines with PARD_MODE_RAW.
+ *   PARD_MODE_PATH_MASK  requests whose downstream path is known (Sec. 5.2,
+ *       dynamic-path DAGs, where a request takes one of several branches):
+ *       pard_request_t.flags is a mask over the downstream paths of the
+ *       request's stage -- bit j = the stage's j-th path in the order of
+ *       pard_pipeline_paths, j < 16 -- and L_sub is the maximum over the paths
+ *       named.  flags = 0 means "unknown": all paths, as without this mode; at
+ *       a sink the mask is ignored; a mask naming no path of the stage gives
+ *       PARD_EDATA.  Order and rule otherwise unchanged (also with priorities).
+ *   PARD_MODE_FCFS       queues are decided in arrival order -- the order of the
+ *       request array -- instead of budget order (Table 1 and Sec. 5.3,
+ *       PARD-FCFS); estimate and rule unchanged; combines with
+ *       PARD_MODE_PATH_MASK; d_priority must be NULL.
+ *   PARD_MODE_NEXUS      Nexus' reactive rule (Sec. 5.1, Baseline), arrival
+ *       order: a window of one batch round (B_k * m_k requests) slides over the
+ *       queue; the batch is the first window whose requests can all finish the
+ *       CURRENT module by their deadlines if the batch starts when the previous
+ *       one ends (base + b * d for round b); all requests in front of it are
+ *       dropped; the scan goes on behind it, one duration later.  A last window
+ *       that the queue cannot fill runs as it is.  est_us = end of the round
+ *       the request was tested against.  d_priority must be NULL.
+ *   PARD_MODE_CLIPPER    Clipper++ (Sec. 5.1, Baseline), arrival order: module k
+ *       gets the share SLO_k = floor(SLO * d_k / sum_i d_i) of the request's
+ *       objective (d_i at the current batch sizes, all stages of the ctx's
+ *       pipeline), counted from the request's arrival at the module; a request
+ *       is dropped iff its batch would start later than arrive + SLO_k (a
+ *       dropped request takes no batch slot).  Needs pard_plan_policy's
+ *       d_arrivals; deadline_us is not read.  est_us = end of the request's
+ *       batch.  arrive_us in [0, 2^60), slo_us in [0, 2^31), d_k < 2^32, else
+ *       PARD_EDATA.  d_priority must be NULL. */
+#define PARD_MODE_PATH_MASK 16u
+#define PARD_MODE_FCFS      32u
+#define PARD_MODE_NEXUS     64u
+#define PARD_MODE_CLIPPER   128u
+
+/* Per-request input of PARD_MODE_CLIPPER: when the request reached the module
+ * whose queue holds it, and its end-to-end latency objective. */
+typedef struct pard_arrival {
+  int64_t arrive_us;
+  int64_t slo_us;
+} pard_arrival_t;          /* 16 bytes, 16-byte aligned arrays */
+
 /* Device scratch pard_plan needs for n requests in n_ctx contexts. */
 int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                               uint64_t* bytes);
@@ -212,6 +259,15 @@ int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
               const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,
               const pard_plan_out_t* out,
               void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
+
+/* pard_plan with the per-request arrival records that PARD_MODE_CLIPPER reads
+ * (DEVICE, [n], parallel to d_requests; NULL for every other mode, which makes
+ * the call identical to pard_plan). */
+int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+                     const pard_request_t* d_requests, const pard_arrival_t* d_arrivals,
+                     uint64_t n, const pard_queue_state_t* state, uint32_t n_ctx,
+                     uint32_t mode, const pard_plan_out_t* out,
+                     void* d_workspace, uint64_t workspace_bytes, void* cuda_stream);
 
 /* For PARD_MODE_NOWAIT: waits for `cuda_stream`, then returns the status that
  * the most recent pard_plan call on this workspace left there (PARD_OK,

@@ -23,6 +23,7 @@ PARD_EWORKSPACE, PARD_ETIMEOUT, PARD_ECUDA, PARD_EDATA, PARD_ESTATIC = -5, -6, -
 PARD_STATIC_SCRATCH_BYTES = 8 << 20
 PARD_LOAD_HOST_ONLY = 1
 PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT, PARD_MODE_SCAN, PARD_MODE_TEST_STALL = 0, 1, 2, 4, 8
+PARD_MODE_PATH_MASK, PARD_MODE_FCFS, PARD_MODE_NEXUS, PARD_MODE_CLIPPER = 16, 32, 64, 128
 PARD_N_PHASES = 15
 PARD_PROFILE_COARSE = 0x80000000
 PARD_MAX_WAIT_SAMPLES = 1 << 15
@@ -34,7 +35,7 @@ PARD_MAX_DELAY_WINDOW_US = 1 << 24
 
 EXPORTS = ["pard_strerror", "pard_load_pipeline", "pard_free_pipeline", "pard_pipeline_n_stages",
            "pard_pipeline_n_slots", "pard_pipeline_paths", "pard_plan_workspace_bytes", "pard_plan",
-           "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput", "pard_plan_status",
+           "pard_plan_host_workspace_bytes", "pard_plan_host", "pard_goodput", "pard_plan_status", "pard_plan_policy",
            "pard_plan_kernel_launches", "pard_profile_begin", "pard_profile_end",
            "pard_profile_phase_name", "pard_plan_static", "pard_estimate_w_workspace_bytes",
            "pard_estimate_w", "pard_update_priority_workspace_bytes", "pard_update_priority",
@@ -92,6 +93,7 @@ def library() -> C.CDLL:
         plan_args = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32,
                      C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
         lib.pard_plan.argtypes = plan_args
+        lib.pard_plan_policy.argtypes = plan_args[:3] + [C.c_void_p] + plan_args[3:]
         lib.pard_plan_host.argtypes = plan_args
         lib.pard_goodput.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p]
@@ -266,6 +268,19 @@ def pard_plan(pipelines: Sequence[Pipeline], d_requests, n: int, state: QueueSta
                              C.byref(o), _ptr(d_workspace), wb, stream or None)
     if check:
         _check(rc, "pard_plan")
+    return rc
+
+
+def pard_plan_policy(pipelines: Sequence[Pipeline], d_requests, d_arrivals, n: int, state: QueueStateArrays,
+                     n_ctx: int, mode: int, out: PlanOut, d_workspace, workspace_bytes: Optional[int] = None,
+                     stream: int = 0, check: bool = True) -> int:
+    hs = _handles(pipelines)
+    st, o = state.c_struct(), out.c_struct()
+    wb = workspace_bytes if workspace_bytes is not None else d_workspace.numel() * d_workspace.element_size()
+    rc = library().pard_plan_policy(hs, len(pipelines), _ptr(d_requests), _ptr(d_arrivals), n, C.byref(st), n_ctx,
+                                    mode, C.byref(o), _ptr(d_workspace), wb, stream or None)
+    if check:
+        _check(rc, "pard_plan_policy")
     return rc
 
 

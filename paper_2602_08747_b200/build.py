@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpard.so")
-SOURCES = ["pard_pipeline.cu", "pard_plan.cu", "pard_goodput.cu", "pard_host.cu",
+SOURCES = ["pard_pipeline.cu", "pard_plan.cu", "pard_policy.cu", "pard_goodput.cu", "pard_host.cu",
            "pard_static.cu", "pard_wait.cu", "pard_priority.cu", "pard_qdelay.cu", "pard_replay.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
@@ -18,6 +18,7 @@ FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std
 def _inputs():
     files = [os.path.join(CSRC, s) for s in SOURCES]
     files.append(os.path.join(CSRC, "pard_internal.h"))
+    files.append(os.path.join(CSRC, "pard_plan_internal.cuh"))
     files.append(os.path.join(ROOT, "include", "pard.h"))
     return files
 

@@ -45,10 +45,10 @@ struct __align__(16) PardSegConst {
   uint64_t d_magic;  /* floor(2^64 / d) + 1, or 0 when d == 1 or d >= 2^32              */
   uint64_t cap_magic;/* floor(2^64 / cap) + 1, or 0 when cap == 1                       */
   uint32_t cap;      /* min(B_k * m_k, 2^30)                                            */
-  uint32_t narrow;   /* 1: 2 <= d < 2^31 and |A_rel| < 2^29, the 32-bit fields below apply */
-  int32_t a_rel32;   /* A_rel                                                           */
-  uint32_t d32;      /* d                                                               */
-  uint32_t pad[2];
+  uint32_t narrow;   /* bit 0: 2 <= d < 2^31 and |A_rel| < 2^29, so both fit 32-bit arithmetic;
+                        bit 1: the ctx's pipeline has no such stage; bit 2: high budget first */
+  int64_t lsub;      /* L_sub of Eq. 3 (max over all downstream paths): A - lsub = base + d_k(B_k) */
+  int64_t dsum;      /* sum of d_i(B_i) over all stages of the ctx's pipeline (Clipper++ split) */
 };
 static_assert(sizeof(PardSegConst) == 64, "one 64-byte line per segment");
 

@@ -16,54 +16,11 @@
 #include <cstring>
 #include <mutex>
 
-#include "pard_internal.h"
+#include "pard_plan_internal.cuh"
+
+using namespace pard_plan_detail;
 
 namespace {
-
-constexpr int kMaxPasses = 8;
-constexpr int kBins = 256;
-constexpr uint32_t kUClamp = (1u << 30) - 1;       /* >= any request count      */
-constexpr uint32_t kMaxPipelinesPerCall = 65536;
-constexpr uint32_t kSegNarrow = 1u;                /* bits of PardSegConst::narrow */
-constexpr uint32_t kSegNoStage = 2u;
-constexpr uint32_t kSegHighFirst = 4u;
-constexpr uint32_t kFoldSegs = 1024;              /* up to this many queues the key width is found inside k_seg_const */
-constexpr uint32_t kSpinLimit = 1u << 18;          /* polling rounds (about a microsecond each) before giving up */
-
-constexpr int kSortThreads = 512;
-constexpr int kLoWarps = 8;                        /* warps 0..7 also do the look-back (one thread per digit) */
-constexpr int kItemsLo = 10, kItemsHi = 22;        /* rounds of 32 elements per warp: look-back warps / others (measured best) */
-constexpr int kSortTile = 32 * (kLoWarps * kItemsLo + (kSortThreads / 32 - kLoWarps) * kItemsHi);
-constexpr int kDecThreads = 128;                   /* small blocks: a short tail when the grid drains (measured against 64 and 256) */
-constexpr int kDecItems = 8;
-constexpr int kDecTile = kDecThreads * kDecItems;
-constexpr int kCompactChunk = 1024;                /* indices moved by one warp of k_kept_move */
-constexpr int kLookBatch = 8;                      /* earlier tiles inspected per round trip in the sort */
-
-/* look-back word of the sort: [31:30] state, [29:0] count */
-constexpr uint32_t kLbAgg = 1u << 30;
-constexpr uint32_t kLbIncl = 2u << 30;
-constexpr uint32_t kLbMask = (1u << 30) - 1;
-
-struct PlanHeader {
-  uint32_t status;            /* 0, or the positive value of a pard_status */
-  uint32_t dbits;             /* bits of the widest per-ctx deadline span  */
-  uint32_t keybits;           /* segment bits + dbits                      */
-  uint32_t npass;             /* radix passes that run                     */
-  unsigned long long span_max;
-  unsigned long long win_total;   /* window-table entries asked for (64 bits: 2^24 queues of up to 4,097 entries) */
-  uint32_t ticket[kMaxPasses + 1];
-  uint32_t wide;              /* 1: segment, deadline and index bits exceed 64; nothing is sorted */
-  uint32_t use_scan;          /* 1: too many batch windows for the window tables: decide by scanning */
-  uint32_t aborted;           /* 1: a bounded wait ran out; the sort is incomplete and every later kernel returns */
-  uint32_t big_total;         /* window-table entries that belong to long queues */
-  uint32_t agg_done;          /* blocks of k_tile_agg that have stored their aggregates */
-  uint32_t seg_done;          /* blocks of k_seg_const that have stored their constants */
-  uint32_t unsorted;          /* 1: some request's ctx is smaller than its predecessor's */
-  uint32_t ctx_too_big;       /* 1: some ctx holds more requests than one sort tile */
-  uint32_t pad[64 - 16 - (kMaxPasses + 1)];
-};
-static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: cleared by k_clear (of the two
@@ -123,10 +80,6 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.buf_b = o;     o = al(o + 8ull * n);
   L.total = o;
   return L;
-}
-
-__device__ __forceinline__ void set_status(PlanHeader* hdr, int status) {
-  atomicCAS(&hdr->status, 0u, (uint32_t)(-status));
 }
 
 /* A bounded wait ran out: the elements are only partly sorted from here on, so nothing after
@@ -260,9 +213,10 @@ __global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin_inv,
 }
 
 /* Width of the sort key, once the widest deadline span is known. */
-__global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
+__global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr, uint32_t arrival_order) {
   pdl_wait();
-  const uint32_t dbits = bit_width64(hdr->span_max);
+  /* in arrival order the deadline takes no part in the key: the index alone orders a queue */
+  const uint32_t dbits = arrival_order ? 0u : bit_width64(hdr->span_max);
   hdr->dbits = dbits;
   hdr->keybits = sbits + dbits;
   hdr->npass = (sbits + dbits + 7) / 8;
@@ -273,21 +227,6 @@ __global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr) {
   }
 }
 
-/* The device tables of the call's pipelines: handed over inside the kernel arguments when they
- * are few (no copy to enqueue), else through a table in the workspace. */
-constexpr int kFewPipelines = 8;
-struct PipeTable {
-  const PardPipeDev* few[kFewPipelines];
-  const PardPipeDev* const* many;
-};
-
-/* floor(2^64 / d) + 1 for d >= 2 */
-__device__ __forceinline__ unsigned long long magic64(unsigned long long d) {
-  unsigned long long q = ~0ull / d;
-  if (~0ull % d == d - 1) ++q;          /* d divides 2^64 */
-  return q + 1;
-}
-
 /* Per-segment constants; one warp per (ctx, stage), lanes over the stage's
  * downstream paths (the path table of the pipeline lists, for every stage,
  * each stage sequence from a successor to a sink). */
@@ -296,7 +235,7 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
             pard_queue_state_t st, uint32_t n_ctx,
             const unsigned long long* __restrict__ ctx_dmin_inv,
             const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
-            PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width) {
+            PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width, uint32_t arrival_order) {
   pdl_wait();
   const uint32_t S = (uint32_t)st.stage_stride;
   const uint32_t lane = threadIdx.x & 31;
@@ -305,7 +244,7 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
   const uint32_t c = seg / S, k = seg % S;
   PardSegConst out;
   out.A = 0; out.A_rel = 0; out.d = 1; out.cap = 1; out.d_magic = 0; out.cap_magic = 0;
-  out.narrow = 0; out.a_rel32 = 0; out.d32 = 1; out.pad[0] = out.pad[1] = 0;
+  out.narrow = 0; out.lsub = 0; out.dsum = 1;
   int32_t pi = st.d_pipeline_of_ctx ? st.d_pipeline_of_ctx[c] : 0;
   bool bad = false;
   if (pi < 0 || (uint32_t)pi >= n_pipelines) {
@@ -358,8 +297,16 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
         const int64_t lim = (int64_t)1 << 29;
         out.narrow = (out.d_magic != 0 && d < ((int64_t)1 << 31) && out.A_rel > -lim && out.A_rel < lim) ? 1u : 0u;
         if (high_first) out.narrow |= kSegHighFirst;
-        out.a_rel32 = (int32_t)out.A_rel;
-        out.d32 = (uint32_t)d;
+        out.lsub = lsub;
+        /* all stages' durations at their current batch sizes, for the rule that splits the objective
+         * in proportion to them (a batch size out of range is reported by that stage's own warp) */
+        long long dsum = 0;
+        for (int32_t i = (int32_t)lane; i < p->n_stages; i += 32) {
+          const int32_t Bi = brow[i];
+          dsum += p->lat_us[p->lat_offsets[i] + ((Bi >= 1 && Bi <= p->bmax[i]) ? Bi : 1) - 1];
+        }
+        for (int o = 16; o; o >>= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+        out.dsum = dsum;
       }
     }
   }
@@ -384,7 +331,7 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
   __syncthreads();
   if (threadIdx.x == 0) {
     for (uint32_t w = 1; w < blockDim.x / 32; ++w) span = s_span[w] > span ? s_span[w] : span;
-    const uint32_t dbits = bit_width64(span);
+    const uint32_t dbits = arrival_order ? 0u : bit_width64(span);
     hdr->span_max = span;
     hdr->dbits = dbits;
     hdr->keybits = sbits + dbits;
@@ -856,43 +803,10 @@ __device__ __forceinline__ SegVal unpack_val(unsigned long long w) {
   return a;
 }
 
-/* floor(x / d) for 32-bit x, with M = floor(2^64 / d) + 1 (d >= 2): exact
- * whenever x * d < 2^64, i.e. for every 32-bit x and d */
-__device__ __forceinline__ uint32_t div_magic32(uint32_t x, unsigned long long M) {
-  unsigned long long p0 = (unsigned long long)x * (uint32_t)M;
-  unsigned long long p1 = (unsigned long long)x * (uint32_t)(M >> 32) + (p0 >> 32);
-  return (uint32_t)(p1 >> 32);
-}
-
-__device__ __forceinline__ uint32_t threshold_u(int64_t X, const PardSegConst& K) {
-  /* number of requests that may be admitted ahead of or at this one while it
-   * still completes by its deadline: 0 if even position 0 is late, else
-   * cap * (floor(X / d) + 1), saturated */
-  if (X < 0) return 0;
-  unsigned long long q;
-  if (((unsigned long long)X >> 32) == 0 && K.d_magic)
-    q = div_magic32((uint32_t)X, K.d_magic);
-  else
-    q = (unsigned long long)X / (unsigned long long)K.d;    /* d == 1 or operands beyond 32 bits */
-  if (q >= kUClamp) return kUClamp;
-  unsigned long long u = (q + 1) * K.cap;
-  return u > kUClamp ? kUClamp : (uint32_t)u;
-}
-
 /* X = deadline - A of a request from its deadline offset: offsets of a queue served high
  * budget first count down from the ctx's largest deadline, and A_rel is that deadline - A */
 __device__ __forceinline__ long long slack_of(unsigned long long off, const PardSegConst& K) {
   return (K.narrow & kSegHighFirst) ? K.A_rel - (long long)off : (long long)off - K.A_rel;
-}
-
-/* 32 bytes with one access; p is 32-byte aligned */
-__device__ __forceinline__ void load4(const unsigned long long* p, unsigned long long* v) {
-  asm volatile("ld.global.nc.v4.u64 {%0, %1, %2, %3}, [%4];"
-               : "=l"(v[0]), "=l"(v[1]), "=l"(v[2]), "=l"(v[3]) : "l"(p));
-}
-__device__ __forceinline__ void store4(void* p, unsigned long long a, unsigned long long b,
-                                       unsigned long long c, unsigned long long d) {
-  asm volatile("st.global.v4.u64 [%0], {%1, %2, %3, %4};" :: "l"(p), "l"(a), "l"(b), "l"(c), "l"(d) : "memory");
 }
 
 /* First half of the decision pass for one thread's kDecItems consecutive
@@ -942,7 +856,7 @@ __device__ __forceinline__ void tile_first_half(const TileCtx& T, uint64_t base,
       const uint32_t lo = (uint32_t)e[i], hi = (uint32_t)(e[i] >> 32);
       idx[i] = lo & T.imask;
       const uint32_t off = __funnelshift_r(lo, hi, T.ibits) & (uint32_t)T.dmask;
-      const int32_t X = high_first ? K.a_rel32 - (int32_t)off : (int32_t)off - K.a_rel32;
+      const int32_t X = high_first ? (int32_t)K.A_rel - (int32_t)off : (int32_t)off - (int32_t)K.A_rel;
       const unsigned long long uu = (unsigned long long)(div_magic32((uint32_t)X, K.d_magic) + 1u) * K.cap;
       u[i] = X < 0 ? 0u : (uu > kUClamp ? kUClamp : (uint32_t)uu);
       r[i] = r0 + i;
@@ -1279,7 +1193,7 @@ k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restric
         ahead = c;
       }
       const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;
-      est[i] = K.A + (long long)((unsigned long long)round * K.d32);
+      est[i] = K.A + (long long)((unsigned long long)round * (uint32_t)K.d);
       const uint32_t kept = c < u[i] ? 1u : 0u;
       keepbits |= kept << i;
       if (kept && kept_tmp) kept_tmp[sstart + ahead] = idx[i];
@@ -1415,7 +1329,8 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
           const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
           uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
           uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
-          uint32_t force_scan, const uint32_t* __restrict__ hist, uint32_t sbits, uint32_t local_candidate) {
+          uint32_t force_scan, const uint32_t* __restrict__ hist, uint32_t sbits, uint32_t local_candidate,
+          uint32_t tables) {
   pdl_wait();
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1462,7 +1377,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
     seg_off[s] = lo[0];
     if (out_seg_off) out_seg_off[s] = lo[0];
   }
-  if (s == n_seg) return;
+  if (s == n_seg || !tables) return;             /* the boundaries are all the sequential rules need */
   /* A queue served high budget first needs no window table: its thresholds fall along the
    * queue while the positions rise, so the kept requests are a prefix of it.  The prefix
    * length (first position r with r >= u_r) is found by a 32-ary search and handed to the
@@ -1527,7 +1442,7 @@ k_seg_win_many(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
                const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
                uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
                uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
-               uint32_t force_scan) {
+               uint32_t force_scan, uint32_t tables) {
   pdl_wait();
   const uint32_t warp_g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1553,6 +1468,7 @@ k_seg_win_many(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
     if (out_seg_off) out_seg_off[s] = lo;
   }
   const uint32_t end = __shfl_down_sync(0xffffffffu, lo, 1);
+  if (!tables) return;                           /* the boundaries are all the sequential rules need */
   const bool mine = lane < 31 && s < n_seg;
   uint32_t w = 0;
   bool high_first = false;
@@ -1762,7 +1678,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
       long long X;
       if (narrow) {
         const int32_t off = (int32_t)(__funnelshift_r((uint32_t)e[i], (uint32_t)(e[i] >> 32), T.ibits) & (uint32_t)T.dmask);
-        X = (HF && (K.narrow & kSegHighFirst)) ? K.a_rel32 - off : off - K.a_rel32;
+        X = (HF && (K.narrow & kSegHighFirst)) ? (int32_t)K.A_rel - off : off - (int32_t)K.A_rel;
       } else {
         const uint32_t sg = (uint32_t)(e[i] >> T.kshift);
         if (sg != cur_seg) {
@@ -1943,10 +1859,28 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
                          const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,
                          const pard_plan_out_t* out, void* d_workspace, uint64_t workspace_bytes,
                          void* cuda_stream) {
+  return pard_plan_policy(pipelines, n_pipelines, d_requests, nullptr, n, state, n_ctx, mode, out, d_workspace,
+                          workspace_bytes, cuda_stream);
+}
+
+extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
+                                const pard_request_t* d_requests, const pard_arrival_t* d_arrivals, uint64_t n,
+                                const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,
+                                const pard_plan_out_t* out, void* d_workspace, uint64_t workspace_bytes,
+                                void* cuda_stream) {
   /* ---- host-side checks, nothing launched before they pass ---- */
   if (!pipelines || n_pipelines < 1 || !out) return PARD_EINVAL;
   if (n_pipelines > kMaxPipelinesPerCall) return PARD_ERANGE;
-  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN | PARD_MODE_TEST_STALL)) return PARD_EINVAL;
+  constexpr uint32_t kRuleBits = PARD_MODE_PATH_MASK | PARD_MODE_FCFS | PARD_MODE_NEXUS | PARD_MODE_CLIPPER;
+  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN | PARD_MODE_TEST_STALL | kRuleBits)) return PARD_EINVAL;
+  /* the rules decided by a walk of every queue, and what they combine with */
+  const bool rule_walk = (mode & kRuleBits) != 0;
+  const bool arrival_order = (mode & (PARD_MODE_FCFS | PARD_MODE_NEXUS | PARD_MODE_CLIPPER)) != 0;
+  if (rule_walk && (mode & PARD_MODE_RAW)) return PARD_EINVAL;
+  if ((mode & PARD_MODE_NEXUS) && (mode & (PARD_MODE_CLIPPER | PARD_MODE_PATH_MASK))) return PARD_EINVAL;
+  if ((mode & PARD_MODE_CLIPPER) && (mode & PARD_MODE_PATH_MASK)) return PARD_EINVAL;
+  if ((mode & PARD_MODE_CLIPPER) && n > 0 && (!d_arrivals || ((uintptr_t)d_arrivals & 15))) return PARD_EINVAL;
+  if (arrival_order && state && state->d_priority) return PARD_EINVAL;
   int rc = check_state(state, n_ctx);
   if (rc != PARD_OK) return rc;
   if (n >= PARD_MAX_REQUESTS) return PARD_ERANGE;
@@ -2044,10 +1978,10 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   const bool fold_width = L.n_seg <= kFoldSegs;          /* few queues: k_seg_const's last block finds the key width */
   if (!fold_width) {
     if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
-    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr);
+    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr, arrival_order ? 1u : 0u);
   }
   launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
-             hdr, sbits, ibits, fold_width ? 1u : 0u);
+             hdr, sbits, ibits, fold_width ? 1u : 0u, arrival_order ? 1u : 0u);
   if (local_cand && !local_sure) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
   mark();
   if (local_cand)                                /* every ctx inside one tile: sorted block by block, straight from the requests */
@@ -2071,12 +2005,24 @@ extern "C" int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pip
   if (L.n_seg >= kManyQueues)
     launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
                seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-               (mode & PARD_MODE_SCAN) ? 1u : 0u);
+               (mode & PARD_MODE_SCAN) ? 1u : 0u, rule_walk ? 0u : 1u);
   else
     launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
                out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits, local_cand);
-  if (n > 0) {
+               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits, local_cand, rule_walk ? 0u : 1u);
+  if (n > 0 && rule_walk) {
+    /* a rule without rising thresholds: every queue is walked in order (pard_policy.cu) */
+    PolicyArgs pa = {};
+    pa.hdr = hdr; pa.buf_a = buf_a; pa.buf_b = buf_b;
+    pa.n = n32; pa.ibits = ibits; pa.n_seg = L.n_seg; pa.mode = mode;
+    pa.ktab = ktab; pa.seg_off = seg_off; pa.req = req4; pa.arrivals = d_arrivals;
+    pa.pipes = pipe_table; pa.n_pipelines = n_pipelines; pa.st = *state;
+    pa.out_keep = out->d_keep; pa.out_est = (long long*)out->d_est_us; pa.out_perm = out->d_perm;
+    pa.kept_tmp = out->d_kept_idx ? kept_tmp : nullptr; pa.seg_kept = seg_kept;
+    mark();
+    rc = launch_policy_decision(pa, sms, stream);
+    if (rc != PARD_OK) return rc;
+  } else if (n > 0) {
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
     long long* est = (long long*)out->d_est_us;
     const bool raw = mode & PARD_MODE_RAW;

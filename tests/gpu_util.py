@@ -7,7 +7,7 @@ from paper_2602_08747_b200 import binding as pb
 from paper_2602_08747_b200 import build as pbuild
 
 
-def run_library(wl, mode=0, check=True):
+def run_library(wl, mode=0, check=True, arrivals=None):
     import torch
     pbuild.build()
     assert torch.cuda.is_available()
@@ -20,7 +20,12 @@ def run_library(wl, mode=0, check=True):
     out = pb.alloc_out(wl.n, n_seg, dev)
     ws = pb.alloc_workspace(pb.pard_plan_workspace_bytes(wl.n, wl.n_ctx, S), dev)
     stream = torch.cuda.current_stream().cuda_stream
-    rc = pb.pard_plan(pipes, d_req, wl.n, d_state, wl.n_ctx, mode, out, ws, stream=stream, check=check)
+    if arrivals is not None or mode & (pb.PARD_MODE_PATH_MASK | pb.PARD_MODE_FCFS | pb.PARD_MODE_NEXUS | pb.PARD_MODE_CLIPPER):
+        d_arr = None if arrivals is None else pb.device_requests(arrivals, dev)      # 16-byte records as well
+        rc = pb.pard_plan_policy(pipes, d_req, d_arr, wl.n, d_state, wl.n_ctx, mode, out, ws, stream=stream,
+                                 check=check)
+    else:
+        rc = pb.pard_plan(pipes, d_req, wl.n, d_state, wl.n_ctx, mode, out, ws, stream=stream, check=check)
     if rc != pb.PARD_OK:
         return rc, None
     total = torch.empty(wl.n_ctx, dtype=torch.int64, device=dev)

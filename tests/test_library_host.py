@@ -151,7 +151,11 @@ def test_plan_argument_checks_happen_before_any_launch():
     cst, cout = st.c_struct(), out.c_struct()
     # null pipelines / bad mode / n_ctx = 0 / missing state arrays
     assert lib.pard_plan(None, 1, None, 0, C.byref(cst), 1, 0, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
-    assert lib.pard_plan(hs, 1, None, 0, C.byref(cst), 1, 16, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
+    assert lib.pard_plan(hs, 1, None, 0, C.byref(cst), 1, 1 << 20, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
+    # rules that exclude each other, and the split-budget rule without its arrival records
+    assert lib.pard_plan(hs, 1, None, 0, C.byref(cst), 1, 64 | 128, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
+    assert lib.pard_plan(hs, 1, None, 5, C.byref(cst), 1, 128, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
+    assert lib.pard_plan(hs, 1, None, 0, C.byref(cst), 1, 32 | 1, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
     assert lib.pard_plan(hs, 1, None, 0, C.byref(cst), 0, 0, C.byref(cout), None, 0, None) == pb.PARD_EINVAL
     bad = pb.QueueStateArrays(2, 1, None, dummy, dummy, dummy).c_struct()
     assert lib.pard_plan(hs, 1, None, 0, C.byref(bad), 1, 0, C.byref(cout), None, 0, None) == pb.PARD_EINVAL

@@ -152,7 +152,12 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    n = 1 << 22 if args.steps + args.warmup <= 100 else 1 << 20
+    # the full 2^24-request snapshot costs about 3 s per step on one core: the whole snapshot while
+    # steps + warm-up stay within about two and a half minutes, else the largest power-of-two
+    # sample of it that does
+    n = 1 << 24
+    while n > (1 << 16) and (args.steps + args.warmup) * (n / 5.5e6) > 150.0:
+        n >>= 1
     wl = inputs.make(WORKLOAD, n=n)
     from oracle import oracle
     for _ in range(args.warmup):
@@ -162,14 +167,16 @@ def run_reference(args):
         oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx)
     dt = time.perf_counter() - t0
     value = wl.n * args.steps / dt
-    sample = "%s workload drawn at n=%d requests per step" % (WORKLOAD, n)
+    sample = ("the full %s snapshot (%d requests) per step" % (WORKLOAD, n) if n == 1 << 24 else
+              "%s workload drawn at n=%d requests per step" % (WORKLOAD, n))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
         "data": "synthetic",
         "config": {"workload": WORKLOAD, "requests_per_step": n, "stages": 16, "paths": 12,
-                   "note": "CPU oracle (single thread) on a bounded sample"},
+                   "contexts": wl.n_ctx,
+                   "note": "CPU oracle (single thread)" + ("" if n == 1 << 24 else " on a bounded sample")},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                          "host_cores": os.cpu_count()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -275,6 +282,14 @@ def kernel_table(prof, n, keep_frac, peak, prof_coarse=None):
     other = ms["clear"] + ms["segments"] + sum(ms[s] for s in sort_names if s not in sort_active)
     rows["other"] = {"ms_per_step": other / k}
     return rows
+
+
+def pass_scalars(rows, suffix=""):
+    """The pass over the sorted queues (thresholds, positions, estimates, drop rule, compaction,
+    goodput counters; window tables included) as three plain numbers."""
+    r = rows["decision_pass"]
+    return {"pass_ms" + suffix: r["ms_per_launch"], "pass_bytes_per_request" + suffix: r["algorithmic_bytes_per_request"],
+            "pass_frac" + suffix: r["frac"]}
 
 
 def run_e2e(wl, dev, steps, dist, lanes=1):
@@ -512,14 +527,64 @@ def _paths(p):
     return out
 
 
+def run_sharded(dev, dist, world, rank):
+    """One job split over the ranks (fixed total work): the many-context workloads by ctx, the
+    single-ctx workload by stage.  No exchange on the data path; the per-ctx goodput counters are
+    gathered (by ctx) or summed (by stage) over NCCL after the timed region.  Time = max over ranks."""
+    import torch
+    from paper_2602_08747_b200 import sharding
+    out = {}
+    for name, how in (("C4", "ctx"), ("C5", "ctx"), (WORKLOAD, "stage")):
+        wl = inputs.make(name)
+        mine = sharding.shard_workload(wl, world, rank) if how == "ctx" else sharding.shard_by_stage(wl, world, rank)
+        plan = DevicePlan(mine, dev)
+        plan.step(nowait=False)
+        steps = 20
+        sec, _ = timed_steps(plan, steps, 5, dist)
+        if how == "ctx":
+            tot, kept = sharding.gather_counters(plan.total, plan.kept, wl.n_ctx)
+        else:
+            tot, kept = sharding.sum_counters(plan.total, plan.kept)
+        torch.cuda.synchronize()
+        out[name] = {"split": "by " + how, "ranks": world, "requests": wl.n, "requests_this_rank": mine.n,
+                     "us_per_step": 1e6 * sec / steps, "requests_per_s": wl.n * steps / sec, "scaling": "strong",
+                     "counted_requests": int(tot.sum().item()), "kept_requests": int(kept.sum().item())}
+        del plan, mine, wl
+    return out
+
+
+def _free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_entry(local_rank, world, port, target, args):
+    os.environ.update({"MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port), "WORLD_SIZE": str(world),
+                       "RANK": str(local_rank), "LOCAL_RANK": str(local_rank)})
+    target(*args)
+
+
+def spawn_ranks(world, target, args=()):
+    """One process per GPU of this node, with the rendezvous environment a launcher would set
+    (`python bench.py --gpus N` without torchrun)."""
+    import torch.multiprocessing as mp
+    mp.spawn(_rank_entry, args=(world, _free_port(), target, args), nprocs=world, join=True)
+
+
 def run_ours(args):
     import torch
     from paper_2602_08747_b200 import build as pbuild
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit("bench.py: --gpus %d but WORLD_SIZE=%d: launch one rank per GPU" % (args.gpus, world))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the planner has no CPU path")
+    if torch.cuda.device_count() <= local:
+        raise SystemExit("bench.py: rank %d has no GPU (%d visible)" % (local, torch.cuda.device_count()))
     pbuild.build()
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
@@ -578,7 +643,10 @@ def run_ours(args):
                     "unit": "GB/s", "frac": timed[top]["frac"], "traffic": traffic,
                     "peak_kind": "of " + peak_kind,
                     "algorithmic_bytes_per_launch": timed[top]["algorithmic_bytes_per_request"] * wl.n,
+                    "pass_note": "pass = everything after the sort, goodput counters included, timed as one "
+                                 "phase; bytes = 21 + 4 * keep fraction per request",
                     "kernels": kernels}
+        roofline.update(pass_scalars(kernels))
         # the balanced variant (about half of the requests kept) as a second data point
         variants = {}
         if not args.no_variants:
@@ -588,9 +656,11 @@ def run_ours(args):
             kf = float(pl2.out.n_kept.cpu()[0]) / wlb.n
             s2, prof2 = timed_steps(pl2, max(10, args.steps // 4), 5, None, profile_every=4)
             _, prof2c = timed_steps(pl2, 40, 0, None, profile_every=4 | pb.PARD_PROFILE_COARSE)
+            kernels_b = kernel_table(prof2, wlb.n, kf, peak, prof2c)
             variants[WORKLOAD + "b"] = {"value": wlb.n * max(10, args.steps // 4) / s2, "unit": UNIT,
-                                        "keep_fraction": kf,
-                                        "kernels": kernel_table(prof2, wlb.n, kf, peak, prof2c)}
+                                        "keep_fraction": kf, "kernels": kernels_b}
+            roofline.update(pass_scalars(kernels_b, "_c3b"))
+            roofline["keep_fraction_c3b"] = kf
             del pl2
         aux = {} if args.no_variants else run_aux(dev, peak)
         others = {}
@@ -609,6 +679,8 @@ def run_ours(args):
             others["C4"]["cpu_baseline_all_cores"] = oracle_all_cores("C4", {"n_epochs": 512, "per_epoch": 8192})
             others["C5"]["cpu_baseline_all_cores"] = oracle_all_cores("C5", {"n_inst": 64, "per_inst": 65536})
         t_cpu, _ = time_oracle(wl, 2)
+    sharded = run_sharded(dev, dist, world, rank) if (world > 1 and not args.no_variants) else {}
+    if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True,
@@ -621,6 +693,8 @@ def run_ours(args):
             "e2e": {"value": n_total * e2e_steps / e2e_sec, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "ms_per_step": 1e3 * e2e_sec / e2e_steps,
+                    "host_link_gbs": (h2d + d2h) * e2e_steps / e2e_sec / 1e9,
+                    "host_link_gbs_outside_device_time": (h2d + d2h) / max(1e-9, e2e_sec / e2e_steps - sec / args.steps) / 1e9,
                     "note": "one blocking pard_plan_host call after the other on one stream"},
             "e2e_two_streams": {"value": n_total * e2e_steps / e2e2_sec, "unit": UNIT, "steps": e2e_steps,
                                 "ms_per_step": 1e3 * e2e2_sec / e2e_steps,
@@ -635,6 +709,7 @@ def run_ours(args):
             "variants": variants,
             "state_planner_kernels": aux,
             "other_workloads": others,
+            "sharded_jobs": sharded,
         }
         print(json.dumps(line))
     if dist is not None:
@@ -661,6 +736,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args.gpus, run_ours, (args,))          # no launcher around us: start the ranks here
     else:
         run_ours(args)
 

@@ -478,7 +478,8 @@ int pard_update_priority(const pard_pipeline_t* const* pipelines, uint32_t n_pip
  * records CUDA events on its stream between its phases; the other calls are
  * untouched.  pard_profile_end waits for the sampled calls, adds up the
  * elapsed milliseconds per phase into ms_sum[PARD_N_PHASES] and returns the
- * number of sampled calls.  Process-wide state: do not call begin/end while
+ * number of sampled calls.  A pard_goodput call that follows a sampled pard_plan
+ * call counts into that call's last phase.  Process-wide state: do not call begin/end while
  * another thread is inside pard_plan.  The paper has no counterpart. */
 #define PARD_N_PHASES 15
 /* Or-ed into `every`: no events inside the decision pass (an event between two

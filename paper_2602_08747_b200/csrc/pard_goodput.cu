@@ -145,6 +145,7 @@ extern "C" int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets
   if (d_seg_kept) {
     launch_pdl(k_goodput_from_queues, (n_ctx + kThreads / 32 - 1) / (kThreads / 32), kThreads, 0, stream, d_seg_offsets,
                d_seg_kept, n_ctx, (uint32_t)stage_stride, (long long*)d_out_total, (long long*)d_out_kept);
+    pard_profile_extend_last(stream);
     PARD_CUDA_OK(cudaGetLastError());
     return PARD_OK;
   }
@@ -156,6 +157,7 @@ extern "C" int pard_goodput(const uint8_t* d_keep, const uint32_t* d_seg_offsets
                                                      (uint32_t)stage_stride,
                                                      (unsigned long long*)d_out_kept);
   }
+  pard_profile_extend_last(stream);
   PARD_CUDA_OK(cudaGetLastError());
   return PARD_OK;
 }

@@ -77,6 +77,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }
 #endif
 
+/* see pard_profile_begin: lets pard_goodput count as the end of the planner's last phase */
+void pard_profile_extend_last(cudaStream_t stream);
+
 #define PARD_CUDA_OK(expr)                    \
   do {                                        \
     cudaError_t e__ = (expr);                 \

@@ -1787,6 +1787,7 @@ constexpr int kEventsPerSample = PARD_N_PHASES + 1;
 static_assert(PARD_N_PHASES == 4 + kMaxPasses + 3, "phase list");
 struct Profiler {
   std::mutex mu;
+  cudaEvent_t* last = nullptr;       /* events of the most recent sampled call */
   std::atomic<bool> on{false};       /* read without the lock by every pard_plan call */
   bool coarse = false;
   uint32_t every = 1, max_samples = 0, calls = 0, n_samples = 0;
@@ -1803,8 +1804,10 @@ cudaEvent_t* profile_acquire(bool* coarse) {
   if (!g_prof.on.load(std::memory_order_relaxed)) return nullptr;
   *coarse = g_prof.coarse;
   uint32_t call = g_prof.calls++;
+  g_prof.last = nullptr;
   if (call % g_prof.every != 0 || g_prof.n_samples >= g_prof.max_samples) return nullptr;
-  return g_prof.ev.data() + (size_t)(g_prof.n_samples++) * kEventsPerSample;
+  g_prof.last = g_prof.ev.data() + (size_t)(g_prof.n_samples++) * kEventsPerSample;
+  return g_prof.last;
 }
 
 /* the sort pass needs more dynamic shared memory than the default limit: opt in once per device */
@@ -1843,6 +1846,15 @@ int check_state(const pard_queue_state_t* st, uint32_t n_ctx) {
 }
 
 }  // namespace
+
+/* pard_goodput follows pard_plan on the same stream and belongs to the same pass over the
+ * sorted queues: when the plan call just before it was a sampled one, the end of its last phase
+ * moves behind the goodput kernel. */
+void pard_profile_extend_last(cudaStream_t stream) {
+  if (!g_prof.on.load(std::memory_order_acquire)) return;
+  std::lock_guard<std::mutex> lock(g_prof.mu);
+  if (g_prof.on.load(std::memory_order_relaxed) && g_prof.last) cudaEventRecord(g_prof.last[PARD_N_PHASES], stream);
+}
 
 extern "C" int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                                          uint64_t* bytes) {
@@ -2112,6 +2124,7 @@ extern "C" int pard_profile_begin(uint32_t every, uint32_t max_samples) {
   g_prof.max_samples = max_samples;
   g_prof.calls = 0;
   g_prof.n_samples = 0;
+  g_prof.last = nullptr;
   g_prof.on.store(true, std::memory_order_release);
   return PARD_OK;
 }
@@ -2136,6 +2149,7 @@ extern "C" int pard_profile_end(float* ms_sum, uint32_t* n_samples) {
   if (n_samples) *n_samples = g_prof.n_samples;
   for (auto& e : g_prof.ev) cudaEventDestroy(e);
   g_prof.ev.clear();
+  g_prof.last = nullptr;
   g_prof.on.store(false, std::memory_order_release);
   return rc;
 }

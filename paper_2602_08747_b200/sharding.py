@@ -2,9 +2,12 @@
 
 Contexts are independent planning problems (one pipeline instance at one
 decision epoch), so a job shards by ctx with no exchange on the data path:
-every rank plans a contiguous block of contexts on its own GPU.  The only
-communication is the optional gathering of the per-ctx goodput counters for
-reporting.  Host logic only; the planning itself is `binding.pard_plan`.
+every rank plans a contiguous block of contexts on its own GPU.  A job with a
+single ctx shards by stage instead: the queues of one ctx are independent once
+every rank holds the ctx's (small) state rows, so every rank plans a contiguous
+block of stages.  The only communication is the combination of the per-ctx
+goodput counters: gathered (by ctx) or summed (by stage).  Host logic only; the
+planning itself is `binding.pard_plan`.
 """
 from __future__ import annotations
 
@@ -37,6 +40,34 @@ def shard_workload(wl: inputs.Workload, world: int, rank: int) -> inputs.Workloa
                               rows(st.pipeline_of_ctx), rows(st.priority))
     return inputs.Workload("%s[%d/%d]" % (wl.name, rank, world), wl.pipelines, req, state, hi - lo,
                            dict(wl.notes))
+
+
+def stage_range(n_stages: int, world: int, rank: int):
+    """Contiguous, balanced block of stages of `rank`."""
+    return ctx_range(n_stages, world, rank)
+
+
+def shard_by_stage(wl: inputs.Workload, world: int, rank: int) -> inputs.Workload:
+    """The requests queued at this rank's block of stages; contexts, stage ids and the whole
+    state are kept (L_sub of a stage reads the rows of the stages downstream of it), so segment
+    ids mean the same on every rank and the queues of the other ranks' stages are simply empty
+    here.  Service order is (ctx, stage)-major: with one ctx the ranks' outputs, in rank order,
+    concatenate to the whole job's; per-ctx counters add up over the ranks."""
+    lo, hi = stage_range(wl.state.stage_stride, world, rank)
+    sel = (wl.requests["stage"] >= lo) & (wl.requests["stage"] < hi)
+    req = np.ascontiguousarray(wl.requests[sel])
+    return inputs.Workload("%s[stages %d/%d]" % (wl.name, rank, world), wl.pipelines, req, wl.state, wl.n_ctx,
+                           dict(wl.notes))
+
+
+def sum_counters(total, kept, group=None):
+    """Per-ctx (total, kept) counters of a job sharded by stage: the sum over the ranks, on
+    every rank (one all-reduce of 2 * n_ctx int64 values)."""
+    import torch
+    import torch.distributed as dist
+    both = torch.stack([total, kept])
+    dist.all_reduce(both, op=dist.ReduceOp.SUM, group=group)
+    return both[0], both[1]
 
 
 def gather_counters(total, kept, n_ctx: int, group=None):

@@ -7,11 +7,14 @@ scratch array inside its own image and offers pard_plan_static, which takes no
 workspace.  This test drives it through the C ABI and requires the same bits as
 pard_plan (with a caller-allocated workspace) on two consecutive calls, so that
 whatever the first call leaves in the shared scratch is shown not to leak into
-the second.  Collected last on purpose: a failure here cannot hide other tests.
+the second; both are also held against the CPU oracle, and the device's free
+memory is read before and after a call to see that nothing was allocated.
+Collected last on purpose: a failure here cannot hide other tests.
 """
 import numpy as np
 import pytest
 
+from oracle import oracle
 from paper_2602_08747_b200 import binding as pb
 from paper_2602_08747_b200 import build as pbuild
 from paper_2602_08747_b200 import inputs
@@ -48,9 +51,14 @@ def _static(wl, mode):
     out = pb.alloc_out(wl.n, wl.n_ctx * S)      # outputs are still the caller's
     for t in (out.keep, out.est_us, out.perm, out.kept_idx, out.seg_kept, out.seg_offsets):
         t.fill_(-1 if t.dtype != torch.uint8 else 255)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
     pb.pard_plan_static(pipes, d_req, wl.n, d_state, wl.n_ctx, mode, out, stream=stream)
     torch.cuda.synchronize()
-    return pb.out_to_numpy(out, wl.n)
+    free_after, _ = torch.cuda.mem_get_info()
+    res = pb.out_to_numpy(out, wl.n)
+    res["free_bytes"] = (free_before, free_after)
+    return res
 
 
 def _same(got, want):
@@ -67,11 +75,21 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     second = inputs.make("C1b")
     want_first, want_second = _with_workspace(first, 0), _with_workspace(second, 0)
     _same(_static(first, 0), want_first)
-    _same(_static(second, 0), want_second)
+    got_second = _static(second, 0)
+    _same(got_second, want_second)
+    # the device had as much free memory after the call as before it (the very first call on a
+    # device may load the library's kernels, so the second call is the one looked at)
+    before, after = got_second["free_bytes"]
+    assert after >= before
     # and the same problem twice, in the other position mode
     want = _with_workspace(first, 1)
     _same(_static(first, 1), want)
-    _same(_static(first, 1), want)
+    again = _static(first, 1)
+    _same(again, want)
+    assert again["free_bytes"][1] >= again["free_bytes"][0]
+    # the reference results themselves are the oracle's
+    for wl, mode, got in ((first, 0, want_first), (second, 0, want_second), (first, 1, want)):
+        _same(got, oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, mode))
 
 
 def test_problem_larger_than_the_scratch_is_refused():

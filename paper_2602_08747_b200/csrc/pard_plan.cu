@@ -25,7 +25,7 @@ namespace {
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: cleared by k_clear (of the two
    * look-back arrays only the first: every sort pass clears the array of the pass after it) */
-  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, lookback, zero_end,
+  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, whist, lookback, zero_end,
       ctx_start, pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
@@ -60,6 +60,7 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.seg_kept = o;  o = al(o + 4ull * L.n_seg);
   L.win_done = o;  o = al(o + 4ull * L.n_seg);
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
+  L.whist = o;     o = al(o + (L.n_seg <= kHistSegs ? 4ull * kHistCap : 0ull));   /* window counts of calls with few queues */
   L.lookback = o;  L.zero_end = al(o + 4ull * kBins * (uint64_t)L.sort_tiles);
   o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);                    /* two arrays, used in turn */
   L.ctx_start = o; o = al(o + 4ull * ((uint64_t)n_ctx + 1));
@@ -70,6 +71,7 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.tile_agg = o;  o = al(o + 8ull * L.dec_tiles);
   L.tile_carry = o; o = al(o + 4ull * L.dec_tiles);
   L.win_capacity = (uint32_t)(n / 32 + 4ull * L.n_seg + 1024);
+  if (L.n_seg <= kHistSegs) L.win_capacity = std::max(L.win_capacity, kHistCap);   /* counted tables: see k_seg_const */
   L.win_off = o;   o = al(o + 4ull * (L.n_seg + 1));
   L.win_cnt = o;   o = al(o + 4ull * (L.n_seg + 1));
   L.win_own = o;   o = al(o + 4ull * L.win_capacity);
@@ -235,7 +237,8 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
             pard_queue_state_t st, uint32_t n_ctx,
             const unsigned long long* __restrict__ ctx_dmin_inv,
             const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
-            PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width, uint32_t arrival_order) {
+            PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width, uint32_t arrival_order,
+            uint32_t win_hist, uint32_t force_scan, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt) {
   pdl_wait();
   const uint32_t S = (uint32_t)st.stage_stride;
   const uint32_t lane = threadIdx.x & 31;
@@ -341,21 +344,75 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
       hdr->wide = 1;
       set_status(hdr, PARD_ERANGE);
     }
+    /* Few queues: their batch-window tables are COUNTED while the requests are packed (k_pack)
+     * instead of being searched for in the sorted elements afterwards.  That needs the tables'
+     * extents before any request has been looked at: a queue can have no window beyond that of
+     * its ctx's latest deadline.  Entry 0 of a queue counts its requests with deadline < A, entry
+     * b + 1 those of window b; every queue has at least entry 0, so that the counts also give
+     * the queues' lengths. */
+    if (win_hist) {
+      const uint32_t n_seg = n_ctx * S;
+      uint32_t total = 0;
+      bool scan = force_scan != 0;
+      for (uint32_t q = 0; q < n_seg; ++q) {
+        const PardSegConst K = ktab[q];
+        const uint32_t c = q / S;
+        uint32_t w = 1;
+        const unsigned long long lo = ~ctx_dmin_inv[c], hi = ctx_dmax[c];
+        if (!(K.narrow & kSegNoStage) && lo <= hi) {
+          const long long X = (long long)hi - K.A;
+          const unsigned long long nb = X < 0 ? 0ull : (unsigned long long)X / (unsigned long long)K.d + 1;
+          if (nb >= 4096) scan = true;                 /* kWinMaxPerSeg: too many windows for a table */
+          else w = (uint32_t)nb + 1;
+        }
+        if (total + w > kHistCap) { scan = true; w = 1; }
+        win_off[q] = total;
+        win_cnt[q] = w;
+        total += w;
+      }
+      hdr->win_total = total;
+      if (scan) hdr->use_scan = 1;
+    }
   }
 }
 
 /* request -> sort element; digit histograms of every pass */
+template <bool WIN>
 __global__ void __launch_bounds__(256)
 k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
        const unsigned long long* __restrict__ ctx_dmin_inv, const unsigned long long* __restrict__ ctx_dmax,
        const uint8_t* __restrict__ priority, uint32_t ibits,
        PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst,
-       uint32_t* __restrict__ hist, uint32_t local_candidate) {
+       uint32_t* __restrict__ hist, uint32_t local_candidate,
+       const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ win_off,
+       const uint32_t* __restrict__ win_cnt, uint32_t* __restrict__ whist) {
   pdl_wait();
   __shared__ uint32_t s_hist[kMaxPasses * kBins];
+  /* WIN: the batch-window tables are counted here (few queues); per-queue constants in shared memory */
+  constexpr uint32_t kWinWords = 2048;                      /* more would cost the kernel its occupancy */
+  __shared__ uint32_t s_win[WIN ? kWinWords : 1];
+  __shared__ long long s_A[WIN ? kHistSegs : 1], s_d[WIN ? kHistSegs : 1];
+  __shared__ unsigned long long s_magic[WIN ? kHistSegs : 1];
+  __shared__ uint2 s_wext[WIN ? kHistSegs : 1];            /* first entry and number of entries of the queue's table */
   if (hdr->wide || sort_is_local(hdr, local_candidate)) return;   /* sorted block by block: k_sort_local read the requests itself */
   const uint32_t npass = hdr->npass, dbits = hdr->dbits;
   for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
+  /* The counters are kept in as many copies as fit (a power of two, at most one per lane), lane l
+   * counting in copy l mod copies: requests of one warp that fall into the same entry -- the
+   * usual case when most of a queue is expired, or lies in few windows -- then hit different words. */
+  uint32_t win_total = 0, copies = 1, my_copy = 0;
+  bool win_shared = false;                                  /* tables beyond kWinWords entries are counted in global memory */
+  if (WIN) {
+    win_total = (uint32_t)hdr->win_total;
+    win_shared = win_total <= kWinWords;
+    while (copies < 32 && 2 * copies * win_total <= kWinWords) copies *= 2;
+    my_copy = (threadIdx.x & (copies - 1)) * win_total;
+    if (win_shared) for (uint32_t i = threadIdx.x; i < win_total * copies; i += blockDim.x) s_win[i] = 0;
+    for (uint32_t q = threadIdx.x; q < n_ctx * S; q += blockDim.x) {
+      const PardSegConst K = ktab[q];
+      s_A[q] = K.A; s_d[q] = K.d; s_magic[q] = K.d_magic; s_wext[q] = make_uint2(win_off[q], win_cnt[q]);
+    }
+  }
   __syncthreads();
   const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
@@ -382,8 +439,22 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
         const bool high_first = priority && __ldg(&priority[seg]) != 0;
         unsigned long long off = (high_first ? ctx_dmax[ctx] - D : D - ~ctx_dmin_inv[ctx]) & dmask;
         e = ((((unsigned long long)seg << dbits) | off) << ibits) | j;
+        if (WIN) {
+          const uint2 ext = s_wext[seg];
+          const long long X = (long long)D - s_A[seg];
+          uint32_t h = 0;
+          if (X >= 0) {
+            const unsigned long long M = s_magic[seg];
+            const unsigned long long b = (((unsigned long long)X >> 32) == 0 && M) ? div_magic32((uint32_t)X, M)
+                                                                                  : (unsigned long long)X / (unsigned long long)s_d[seg];
+            h = b + 1 < ext.y ? (uint32_t)b + 1 : ext.y - 1;   /* never beyond the queue's entries (a queue decided by scanning has one) */
+          }
+          if (win_shared) atomicAdd(&s_win[my_copy + ext.x + h], 1u);
+          else atomicAdd(&whist[ext.x + h], 1u);
+        }
       } else {
         e = j;                                  /* flagged by the prepass; keep indices in range */
+        if (WIN) atomicAdd(win_shared ? &s_win[my_copy] : &whist[0], 1u);   /* it sorts into queue 0: counted there, so that the counts stay the queues' lengths */
       }
       dst[j] = e;
       unsigned long long key = e >> ibits;
@@ -393,6 +464,12 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
   __syncthreads();
   for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x)
     if (s_hist[i]) atomicAdd(&hist[i], s_hist[i]);
+  if (WIN && win_shared)
+    for (uint32_t i = threadIdx.x; i < win_total; i += blockDim.x) {
+      uint32_t sum = 0;
+      for (uint32_t r = 0; r < copies; ++r) sum += s_win[r * win_total + i];
+      if (sum) atomicAdd(&whist[i], sum);
+    }
 }
 
 /* ------------------------------------------------------------------------ */
@@ -1634,6 +1711,50 @@ k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegCo
   win_prefix_warp(s, ktab, win_off, win_cnt, wtab, threadIdx.x & 31);
 }
 
+/* The window tables of a call with few queues, from the counts k_pack took: P is the running sum
+ * of a queue's counts, E and Kp follow as in the searched tables, and the queues' first positions
+ * are the running sum of their lengths.  One block; a warp per queue.  Runs before the sort: the
+ * counts do not depend on the order of the elements. */
+__global__ void __launch_bounds__(1024)
+k_win_from_counts(PlanHeader* hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
+                  const uint32_t* __restrict__ whist, const uint32_t* __restrict__ win_off,
+                  const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab,
+                  uint32_t* __restrict__ seg_off, uint32_t* __restrict__ out_seg_off) {
+  pdl_wait();
+  __shared__ uint32_t s_len[kHistSegs];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (uint32_t q = warp; q < n_seg; q += blockDim.x / 32) {
+    const uint32_t off = win_off[q], cnt = win_cnt[q];
+    uint32_t run = 0;
+    for (uint32_t b0 = 0; b0 < cnt; b0 += 32) {
+      const uint32_t b = b0 + lane;
+      uint32_t x = b < cnt ? whist[off + b] : 0u;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= (uint32_t)o) x += y;
+      }
+      if (b < cnt) wtab[off + b].P = run + x;        /* requests of the queue up to and including entry b's */
+      run += __shfl_sync(0xffffffffu, x, 31);
+    }
+    if (lane == 0) s_len[q] = run;
+    __threadfence_block();
+    __syncwarp();
+    /* P as the decision reads it: entry b = requests in windows below b, i.e. the sum up to entry b */
+    win_prefix_warp(q, ktab, win_off, win_cnt, wtab, lane);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t first = 0;
+    for (uint32_t q = 0; q < n_seg; ++q) {
+      seg_off[q] = first;
+      if (out_seg_off) out_seg_off[q] = first;
+      first += s_len[q];
+    }
+    seg_off[n_seg] = first;
+    if (out_seg_off) out_seg_off[n_seg] = first;
+  }
+}
+
 /* Decision pass from the window tables: every request on its own.  HF: some
  * queue may be served high budget first (the caller gave priorities). */
 template <bool RAW, bool HF>
@@ -1778,7 +1899,15 @@ k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ 
     const uint32_t count = min((uint32_t)kCompactChunk, seg_kept[s] - first);
     const uint32_t* src = kept_tmp + seg_off[s] + first;
     uint32_t* dst = out_kept_idx + kept_base[s] + first;
-    for (uint32_t i = lane; i < count; i += 32) dst[i] = src[i];
+    uint32_t i = lane;
+    for (; i + 224 < count; i += 256) {            /* eight loads in flight per lane */
+      uint32_t v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = src[i + 32 * k];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) dst[i + 32 * k] = v[k];
+    }
+    for (; i < count; i += 32) dst[i] = src[i];
   }
 }
 
@@ -1941,6 +2070,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   uint32_t* win_own = (uint32_t*)(ws + L.win_own);
   uint32_t* win_big = (uint32_t*)(ws + L.win_big);
   uint32_t* win_done = (uint32_t*)(ws + L.win_done);
+  uint32_t* whist = (uint32_t*)(ws + L.whist);
   unsigned long long* buf_a = (unsigned long long*)(ws + L.buf_a);
   unsigned long long* buf_b = (unsigned long long*)(ws + L.buf_b);
   const uint32_t n32 = (uint32_t)n;
@@ -1992,8 +2122,12 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
     launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr, arrival_order ? 1u : 0u);
   }
+  /* few queues, decided by the planner's own rule in budget order from the start of every queue:
+   * the window tables are counted while the requests are packed */
+  const bool win_hist = n > 0 && L.n_seg <= kHistSegs && !rule_walk && !state->d_priority && !local_cand;
   launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
-             hdr, sbits, ibits, fold_width ? 1u : 0u, arrival_order ? 1u : 0u);
+             hdr, sbits, ibits, fold_width ? 1u : 0u, arrival_order ? 1u : 0u, win_hist ? 1u : 0u,
+             (mode & PARD_MODE_SCAN) ? 1u : 0u, win_off, win_cnt);
   if (local_cand && !local_sure) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
   mark();
   if (local_cand)                                /* every ctx inside one tile: sorted block by block, straight from the requests */
@@ -2002,8 +2136,12 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
                ceil_log2(S), ibits);
   if (n > 0 && !local_sure) {                    /* returns at once when the blocks above did the work */
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
-    launch_pdl(k_pack, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, ibits, hdr, buf_a, hist,
-               local_cand);
+    launch_pdl(win_hist ? k_pack<true> : k_pack<false>, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax,
+               state->d_priority, ibits, hdr, buf_a, hist, local_cand, (const PardSegConst*)ktab, (const uint32_t*)win_off,
+               (const uint32_t*)win_cnt, whist);
+    if (win_hist)
+      launch_pdl(k_win_from_counts, 1, 1024, 0, stream, hdr, L.n_seg, (const PardSegConst*)ktab, (const uint32_t*)whist,
+                 (const uint32_t*)win_off, (const uint32_t*)win_cnt, wtab, seg_off, out->d_seg_offsets);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
@@ -2014,7 +2152,9 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
           n32, ibits, (p == 0 && (mode & PARD_MODE_TEST_STALL)) ? 1u : 0u, local_cand);
   }
   mark();
-  if (L.n_seg >= kManyQueues)
+  if (win_hist) {
+    /* boundaries and tables are there already */
+  } else if (L.n_seg >= kManyQueues)
     launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
                seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
                (mode & PARD_MODE_SCAN) ? 1u : 0u, rule_walk ? 0u : 1u);
@@ -2039,9 +2179,11 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     long long* est = (long long*)out->d_est_us;
     const bool raw = mode & PARD_MODE_RAW;
     /* window tables, and the decision from them */
-    launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream, 
-        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
-    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab);
+    if (!win_hist) {
+      launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream,
+          hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
+      launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab);
+    }
     mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
@@ -2093,16 +2235,20 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* clear, seg_const, seg_win and kept_scan always, key_width (and, when n > 0, ctx_span) with many
-   * queues; prepass, ctx_span, pack, the passes,
-   * win_bounds, win_prefix, decide_win, tile_agg, decide and kept_move (when the compacted indices
-   * are requested) when n > 0 */
-  const uint32_t width_kernels = (uint64_t)n_ctx * (uint64_t)stage_stride <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
+  /* For the planner's own rule without priorities.  Always: clear, seg_const, kept_scan, and the
+   * queue boundaries (seg_win; with few queues they come with the counted window tables instead).
+   * With many queues also key_width (and, when n > 0, ctx_span).  When n > 0: prepass, pack, the
+   * radix passes, the window tables (win_bounds and win_prefix, or win_from_counts for few
+   * queues), decide_win, the two scan kernels that return at once, and kept_move. */
+  const uint64_t n_seg = (uint64_t)n_ctx * (uint64_t)stage_stride;
+  const uint32_t width_kernels = n_seg <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
   const bool local_cand = local_sort_candidate(n, n_ctx), local_sure = local_cand && n_ctx == 1;
   const uint32_t local_kernels = local_sure ? 1 : local_cand ? 2 : 0;       /* sort_local (, ctx_ranges) */
   const uint32_t passes = local_sure ? 0 : make_layout(n, n_ctx, stage_stride).max_passes;
   const uint32_t pack = local_sure ? 0 : 1;
-  *launches = n > 0 ? 4 + width_kernels + 1 + pack + width_kernels + local_kernels + passes + 6 : 4 + width_kernels;
+  const bool counted = n > 0 && n_seg <= kHistSegs && !local_cand;
+  const uint32_t tables = counted ? 1 : 3;                     /* win_from_counts | seg_win, win_bounds, win_prefix */
+  *launches = n > 0 ? 3 + 2 * width_kernels + 1 + pack + local_kernels + passes + tables + 4 : 4 + width_kernels;
   return PARD_OK;
 }
 

@@ -15,6 +15,8 @@ constexpr uint32_t kSegNarrow = 1u;                /* bits of PardSegConst::narr
 constexpr uint32_t kSegNoStage = 2u;
 constexpr uint32_t kSegHighFirst = 4u;
 constexpr uint32_t kFoldSegs = 1024;              /* up to this many queues the key width is found inside k_seg_const */
+constexpr uint32_t kHistSegs = 64;                /* up to this many queues the batch-window tables are counted, not searched */
+constexpr uint32_t kHistCap = 8192;               /* window-table entries a counted table may have in all */
 constexpr uint32_t kSpinLimit = 1u << 18;          /* polling rounds (about a microsecond each) before giving up */
 
 constexpr int kSortThreads = 512;

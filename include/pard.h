@@ -179,6 +179,23 @@ typedef struct pard_plan_out {
                                    block by block (requests grouped by ctx, no ctx above
                                    8,192 requests) have no such wait and are unaffected */
 
+#define PARD_MODE_GROUPED 256u  /* the caller's word that d_requests is grouped by ascending
+                                   ctx and that no ctx holds more than 8,192 requests
+                                   (batched decision epochs, many small instances).  For
+                                   calls of up to a few hundred contexts one thread block
+                                   then plans each ctx from start to end in shared memory
+                                   -- constants, sort, positions, decisions -- in five
+                                   kernel launches instead of about twenty, two to three
+                                   times faster on small and medium calls; larger calls
+                                   take the general path (which finds the grouping by
+                                   itself).  Where the block-per-ctx path runs, the device
+                                   checks the claim and a call that breaks it returns
+                                   PARD_EDATA; a call that cannot keep it (n > 8,192 *
+                                   n_ctx) returns PARD_EINVAL.  A call with a single ctx of
+                                   at most 8,192 requests is always planned by one block
+                                   (one kernel launch).  Ignored by the rules below, which
+                                   take their own path.  Same results. */
+
 /* Other decision orders and rules on the same queues, for comparison with the
  * planner's own (which stays the default).  Their thresholds do not rise along
  * a queue, so each queue is walked in order by one warp (32 requests per step)
@@ -253,7 +270,9 @@ int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
  * Performance note: requests may come in any order.  When they come grouped by
  * ascending ctx and no ctx holds more than 8,192 of them (batched decision
  * epochs, one module's queue), every ctx is sorted by one thread block in
- * shared memory, which is markedly faster; the result is the same. */
+ * shared memory, which is markedly faster; the result is the same.  A caller
+ * who knows this of its requests says so with PARD_MODE_GROUPED and gets the
+ * whole plan of a ctx from one thread block. */
 int pard_plan(const pard_pipeline_t* const* pipelines, uint32_t n_pipelines,
               const pard_request_t* d_requests, uint64_t n,
               const pard_queue_state_t* state, uint32_t n_ctx, uint32_t mode,

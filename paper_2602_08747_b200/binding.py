@@ -24,6 +24,7 @@ PARD_STATIC_SCRATCH_BYTES = 8 << 20
 PARD_LOAD_HOST_ONLY = 1
 PARD_MODE_ADMITTED, PARD_MODE_RAW, PARD_MODE_NOWAIT, PARD_MODE_SCAN, PARD_MODE_TEST_STALL = 0, 1, 2, 4, 8
 PARD_MODE_PATH_MASK, PARD_MODE_FCFS, PARD_MODE_NEXUS, PARD_MODE_CLIPPER = 16, 32, 64, 128
+PARD_MODE_GROUPED = 256
 PARD_N_PHASES = 15
 PARD_PROFILE_COARSE = 0x80000000
 PARD_MAX_WAIT_SAMPLES = 1 << 15

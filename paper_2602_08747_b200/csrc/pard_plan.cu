@@ -229,22 +229,15 @@ __global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr, uin
   }
 }
 
-/* Per-segment constants; one warp per (ctx, stage), lanes over the stage's
- * downstream paths (the path table of the pipeline lists, for every stage,
- * each stage sequence from a successor to a sink). */
-__global__ void __launch_bounds__(128)
-k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
-            pard_queue_state_t st, uint32_t n_ctx,
-            const unsigned long long* __restrict__ ctx_dmin_inv,
-            const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
-            PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width, uint32_t arrival_order,
-            uint32_t win_hist, uint32_t force_scan, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt) {
-  pdl_wait();
+/* The constants of one queue (ctx c, stage k), by one whole warp: lanes over the stage's
+ * downstream paths (the path table of the pipeline lists, for every stage, each stage sequence
+ * from a successor to a sink).  dmin / dmax: smallest and largest deadline of the ctx, the
+ * origins of the queue's deadline offsets.  Every lane returns the same value; *bad is set in
+ * the lanes that met an input out of range. */
+__device__ PardSegConst seg_const_warp(const PipeTable& pipes, uint32_t n_pipelines, const pard_queue_state_t& st,
+                                       uint32_t c, uint32_t k, unsigned long long dmin, unsigned long long dmax,
+                                       uint32_t lane, bool* bad_out) {
   const uint32_t S = (uint32_t)st.stage_stride;
-  const uint32_t lane = threadIdx.x & 31;
-  const uint32_t seg = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (seg < n_ctx * S) {                                 /* whole warps take the same side */
-  const uint32_t c = seg / S, k = seg % S;
   PardSegConst out;
   out.A = 0; out.A_rel = 0; out.d = 1; out.cap = 1; out.d_magic = 0; out.cap_magic = 0;
   out.narrow = 0; out.lsub = 0; out.dsum = 1;
@@ -294,7 +287,7 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
         /* A against the origin of the queue's deadline offsets: offsets count up from the ctx's
          * smallest deadline, or, for a queue served high budget first, down from its largest */
         const bool high_first = st.d_priority && st.d_priority[(size_t)c * S + k] != 0;
-        out.A_rel = high_first ? (int64_t)ctx_dmax[c] - out.A : out.A - (int64_t)(~ctx_dmin_inv[c]);
+        out.A_rel = high_first ? (int64_t)dmax - out.A : out.A - (int64_t)dmin;
         out.d_magic = (d >= 2 && d < ((int64_t)1 << 32)) ? magic64((uint64_t)d) : 0;
         out.cap_magic = out.cap >= 2 ? magic64(out.cap) : 0;
         const int64_t lim = (int64_t)1 << 29;
@@ -313,8 +306,28 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
       }
     }
   }
-  if (bad) set_status(hdr, PARD_EDATA);
-  if (lane == 0) ktab[seg] = out;
+  *bad_out = bad;
+  return out;
+}
+
+/* Per-segment constants; one warp per (ctx, stage). */
+__global__ void __launch_bounds__(128)
+k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
+            pard_queue_state_t st, uint32_t n_ctx,
+            const unsigned long long* __restrict__ ctx_dmin_inv,
+            const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
+            PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width, uint32_t arrival_order,
+            uint32_t win_hist, uint32_t force_scan, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt) {
+  pdl_wait();
+  const uint32_t S = (uint32_t)st.stage_stride;
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t seg = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (seg < n_ctx * S) {                                 /* whole warps take the same side */
+    const uint32_t c = seg / S, k = seg % S;
+    bool bad = false;
+    const PardSegConst out = seg_const_warp(pipes, n_pipelines, st, c, k, ~ctx_dmin_inv[c], ctx_dmax[c], lane, &bad);
+    if (bad) set_status(hdr, PARD_EDATA);
+    if (lane == 0) ktab[seg] = out;
   }
   /* With few queues the block that finishes last also finds the widest deadline span and with
    * it the width of the sort key (the work of k_ctx_span and k_key_width, without their launches). */
@@ -530,9 +543,10 @@ __device__ __forceinline__ void sort_load_count(unsigned long long (&key)[kItems
 template <int ITEMS, int CAP>
 __device__ __forceinline__ void sort_rank_drop(const unsigned long long (&key)[CAP], uint32_t shift,
                                                uint32_t* slot_row, uint32_t* match_row, unsigned long long* keys,
-                                               uint32_t lanebit) {
+                                               uint32_t lanebit, int items = ITEMS) {
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
+    if (i >= items) break;                             /* the same for the whole block */
     const uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
     atomicOr(&match_row[d], lanebit);
     __syncwarp();
@@ -1911,6 +1925,458 @@ k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ 
   }
 }
 
+/* ------------------------------------------------------------------------ */
+/* one block plans one ctx from start to end                                 */
+/* ------------------------------------------------------------------------ */
+/* For calls whose requests come grouped by ascending ctx with no ctx above a sort tile -- one
+ * module's queue planned every few milliseconds, or many decision epochs in one call -- a block
+ * does the whole job for "its" ctx without leaving shared memory: it reads the ctx's requests
+ * once, finds the ctx's deadline range, computes the constants of the ctx's queues (Eq. 3),
+ * sorts (radix passes over the stage and deadline bits, as k_sort_local), finds every request's
+ * admitted position by a segmented scan over the sorted elements, and writes the outputs: 16
+ * bytes read and 13 + 4f written per request, no element ever stored to global memory, no window
+ * table, no search.  The scan runs twice over the elements, which stay in shared memory: once
+ * for the warps' aggregates, once for the positions.  With a single ctx the block also packs the
+ * survivors (the whole call is one launch); with several, k_kept_scan and k_kept_move follow. */
+struct LocalArgs {
+  const uint4* req;
+  const uint32_t* ctx_start;       /* NULL: the call has one ctx */
+  uint32_t n, n_ctx, ibits, raw;
+  PipeTable pipes;
+  uint32_t n_pipelines;
+  pard_queue_state_t st;
+  uint8_t* out_keep;
+  long long* out_est;
+  uint32_t* out_perm;
+  uint32_t* out_kept_idx;          /* used directly only with one ctx */
+  unsigned long long* out_n_kept;
+  uint32_t* out_seg_off;
+  uint32_t* out_seg_kept;
+  const PardSegConst* ktab;        /* several ctx: the queues' constants, from k_seg_const */
+  uint32_t* seg_off;               /* workspace copies, read by k_kept_scan / k_kept_move */
+  uint32_t* seg_kept;
+  uint32_t* kept_tmp;
+};
+
+struct LocalSmem {
+  SortSmem sort;
+  PardSegConst K[PARD_MAX_STAGES];
+  uint32_t stage_cnt[PARD_MAX_STAGES];
+  uint32_t stage_first[PARD_MAX_STAGES + 1];
+  uint32_t stage_kept[PARD_MAX_STAGES];
+  uint32_t kept_base[PARD_MAX_STAGES + 1];
+  uint32_t hb_kept[PARD_MAX_STAGES];       /* high budget first: length of the kept prefix */
+  unsigned long long red_min[kSortThreads / 32], red_max[kSortThreads / 32];
+  int32_t wm[kSortThreads / 32];
+  uint32_t wh[kSortThreads / 32];
+  uint32_t flag_foreign, flag_bad;
+};
+
+/* decoded view of one sorted element inside a block of k_plan_local */
+struct LocalElem {
+  uint32_t stage, idx, r, u;
+  bool high_first;
+};
+
+__device__ __forceinline__ LocalElem local_decode(unsigned long long e, uint32_t pos, const LocalSmem& Sm,
+                                                  uint32_t ibits, uint32_t dbits, unsigned long long dmask,
+                                                  uint32_t imask) {
+  LocalElem x;
+  x.stage = (uint32_t)(e >> (ibits + dbits));
+  x.idx = (uint32_t)e & imask;
+  const PardSegConst& K = Sm.K[x.stage];
+  x.high_first = K.narrow & kSegHighFirst;
+  x.r = pos - Sm.stage_first[x.stage];
+  const unsigned long long off = (e >> ibits) & dmask;
+  if ((K.narrow & kSegNarrow) && dbits <= 29) {
+    const int32_t X = x.high_first ? (int32_t)K.A_rel - (int32_t)off : (int32_t)off - (int32_t)K.A_rel;
+    const unsigned long long uu = (unsigned long long)(div_magic32((uint32_t)X, K.d_magic) + 1u) * K.cap;
+    x.u = X < 0 ? 0u : (uu > kUClamp ? kUClamp : (uint32_t)uu);
+  } else {
+    x.u = (K.narrow & kSegNoStage) ? 0u : threshold_u(slack_of(off, K), K);
+  }
+  return x;
+}
+
+template <bool RAW>
+__global__ void __launch_bounds__(kSortThreads, 2)
+k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
+  pdl_wait();
+  constexpr int WARPS = kSortThreads / 32;
+  constexpr int kItems = kSortTile / kSortThreads;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  LocalSmem& Sm = *reinterpret_cast<LocalSmem*>(smem_raw);
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lanebit = 1u << lane;
+  const uint32_t S = (uint32_t)a.st.stage_stride;
+  const uint32_t c = blockIdx.x;
+  const bool single = a.ctx_start == nullptr;
+  if (single) {                                          /* the only kernel of the call: the header starts here */
+    if (tid < sizeof(PlanHeader) / 4) reinterpret_cast<uint32_t*>(hdr)[tid] = 0;
+    __syncthreads();
+  } else if (hdr->unsorted || hdr->ctx_too_big) {      /* k_ctx_ranges found the promised grouping broken */
+    if (tid == 0 && c == 0) set_status(hdr, PARD_EDATA);
+    return;
+  }
+  const uint32_t first = single ? 0u : a.ctx_start[c];
+  const uint32_t cnt = single ? a.n : a.ctx_start[c + 1] - first;
+  /* every warp owns `items` rounds of 32 consecutive requests: as few as the ctx needs */
+  const int items = (int)((cnt + kSortThreads - 1) / kSortThreads);
+  const uint32_t wfirst = warp * (32 * (uint32_t)items);
+  uint16_t* stage16 = reinterpret_cast<uint16_t*>(&Sm.sort.slot[0][0]);     /* 16 KB: the stages until the elements are built */
+
+  /* 1. the ctx's requests: deadlines into the tile buffer, stages beside them; deadline range,
+   * queue lengths, input checks */
+  for (uint32_t i = tid; i < S; i += kSortThreads) { Sm.stage_cnt[i] = 0; Sm.stage_kept[i] = 0; }
+  if (tid == 0) { Sm.flag_foreign = 0; Sm.flag_bad = 0; }
+  __syncthreads();
+  unsigned long long lmin = ~0ull, lmax = 0;
+  bool foreign = false, bad = false;
+#pragma unroll 4
+  for (int i = 0; i < kItems; ++i) {
+    if (i >= items) break;
+    const uint32_t pos = wfirst + i * 32 + lane;
+    if (pos < cnt) {
+      const uint4 r = __ldg(&a.req[first + pos]);
+      const unsigned long long D = ((unsigned long long)r.y << 32) | r.x;
+      const uint32_t stage = r.w & 0xffffu;
+      foreign |= r.z != c;
+      const bool ok = r.z == c && stage < S && D < (unsigned long long)PARD_TIME_LIMIT_US;
+      bad |= !ok;
+      Sm.sort.keys[pos] = D;
+      stage16[pos] = ok ? (uint16_t)stage : (uint16_t)0xffffu;
+      if (ok) {
+        lmin = D < lmin ? D : lmin;
+        lmax = D > lmax ? D : lmax;
+        atomicAdd(&Sm.stage_cnt[stage], 1u);
+      }
+    }
+  }
+  for (int o = 16; o; o >>= 1) {
+    const unsigned long long x = __shfl_xor_sync(0xffffffffu, lmin, o), y = __shfl_xor_sync(0xffffffffu, lmax, o);
+    lmin = x < lmin ? x : lmin;
+    lmax = y > lmax ? y : lmax;
+  }
+  if (lane == 0) { Sm.red_min[warp] = lmin; Sm.red_max[warp] = lmax; }
+  if (foreign) Sm.flag_foreign = 1;
+  if (bad) Sm.flag_bad = 1;
+  __syncthreads();
+  if (Sm.flag_foreign) {                                 /* not grouped by ctx after all (or, with one ctx, a request of another) */
+    if (tid == 0) { hdr->unsorted = 1; set_status(hdr, PARD_EDATA); }
+    return;
+  }
+  unsigned long long dmin = ~0ull, dmax = 0;
+#pragma unroll
+  for (int w = 0; w < WARPS; ++w) {
+    dmin = Sm.red_min[w] < dmin ? Sm.red_min[w] : dmin;
+    dmax = Sm.red_max[w] > dmax ? Sm.red_max[w] : dmax;
+  }
+  const uint32_t dbits = dmin <= dmax ? bit_width64(dmax - dmin) : 0u;
+  /* stage field of the elements: requests that failed the checks carry the value S there, so
+   * that they sort behind the ctx's queues; they are reported, never decided */
+  const uint32_t sb = 32u - __clz(Sm.flag_bad ? S : S - 1);    /* bit width of the largest value; __clz(0) = 32 */
+  if (sb + dbits + a.ibits > 64) {                       /* the element does not fit 64 bits */
+    if (tid == 0) { hdr->wide = 1; set_status(hdr, PARD_ERANGE); }
+    return;
+  }
+  if (Sm.flag_bad && tid == 0) set_status(hdr, PARD_EDATA);
+
+  /* 2. constants of the ctx's queues: worked out here, a warp per stage, when the call is this
+   * one block; else taken from the table k_seg_const has filled for all queues at once (a chain
+   * of dependent loads that every block would otherwise wait for) and completed with what hangs
+   * on the ctx's deadline range */
+  if (single) {
+    for (uint32_t k = warp; k < S; k += WARPS) {
+      bool kbad = false;
+      const PardSegConst K = seg_const_warp(a.pipes, a.n_pipelines, a.st, c, k, dmin, dmax, lane, &kbad);
+      if (kbad) set_status(hdr, PARD_EDATA);
+      if (lane == 0) Sm.K[k] = K;
+    }
+  } else {
+    for (uint32_t k = tid; k < S; k += kSortThreads) {
+      PardSegConst K = a.ktab[(size_t)c * S + k];
+      const bool high_first = K.narrow & kSegHighFirst;
+      K.A_rel = high_first ? (int64_t)dmax - K.A : K.A - (int64_t)dmin;
+      const int64_t lim = (int64_t)1 << 29;
+      const bool fits32 = K.d_magic != 0 && K.d < ((int64_t)1 << 31) && K.A_rel > -lim && K.A_rel < lim;
+      K.narrow = (K.narrow & ~kSegNarrow) | (fits32 && !(K.narrow & kSegNoStage) ? kSegNarrow : 0u);
+      Sm.K[k] = K;
+    }
+  }
+  if (warp == 0) {                                       /* first position of every queue inside the ctx */
+    uint32_t run = 0;
+    for (uint32_t k0 = 0; k0 < S; k0 += 32) {
+      const uint32_t k = k0 + lane;
+      const uint32_t v = k < S ? Sm.stage_cnt[k] : 0u;
+      uint32_t x = v;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= (uint32_t)o) x += y;
+      }
+      if (k < S) Sm.stage_first[k] = run + x - v;
+      run += __shfl_sync(0xffffffffu, x, 31);
+    }
+    if (lane == 0) Sm.stage_first[S] = run;
+  }
+  __syncthreads();
+  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  const uint32_t imask = (1u << a.ibits) - 1;
+
+  /* 3. sort elements (stage | deadline offset | index), built from the tile buffer */
+  unsigned long long key[kItems];
+#pragma unroll
+  for (int i = 0; i < kItems; ++i) {
+    if (i >= items) break;
+    const uint32_t pos = wfirst + i * 32 + lane;
+    key[i] = ~0ull;                                      /* padding sorts last */
+    if (pos < cnt) {
+      const unsigned long long D = Sm.sort.keys[pos];
+      const uint32_t stage = stage16[pos];
+      const uint32_t j = first + pos;
+      if (stage != 0xffffu) {
+        const bool high_first = Sm.K[stage].narrow & kSegHighFirst;
+        const unsigned long long off = (high_first ? dmax - D : D - dmin) & dmask;
+        key[i] = ((((unsigned long long)stage << dbits) | off) << a.ibits) | j;
+      } else {
+        key[i] = (((unsigned long long)S << dbits) << a.ibits) | j;
+      }
+    }
+  }
+  __syncthreads();                                       /* the stages have been read: their room becomes the counters again */
+  const uint32_t local_bits = dbits + sb;
+  const uint32_t passes = (local_bits + 7) / 8;
+  for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) (&Sm.sort.match[0][0])[i] = 0;
+  for (uint32_t p = 0; p < passes; ++p) {
+    const uint32_t shift = a.ibits + 8 * p;
+    for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) (&Sm.sort.slot[0][0])[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kItems; ++i)
+      if (i < items) atomicAdd(&Sm.sort.slot[warp][(uint32_t)(key[i] >> shift) & 255u], 1u);
+    __syncthreads();
+    uint32_t count = 0, x = 0;
+    if (tid < kBins) {
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) {
+        const uint32_t t = Sm.sort.slot[w][tid];
+        Sm.sort.slot[w][tid] = count;
+        count += t;
+      }
+      x = count;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= (uint32_t)o) x += y;
+      }
+      if (lane == 31) Sm.sort.scan[0][warp] = x;
+    }
+    __syncthreads();
+    if (tid < kBins) {
+      uint32_t wx = 0;
+#pragma unroll
+      for (int w = 0; w < kBins / 32; ++w)
+        if (w < (int)warp) wx += Sm.sort.scan[0][w];
+      const uint32_t dstart = wx + x - count;
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) Sm.sort.slot[w][tid] += dstart;
+    }
+    __syncthreads();
+    sort_rank_drop<kItems, kItems>(key, shift, Sm.sort.slot[warp], Sm.sort.match[warp], Sm.sort.keys, lanebit, items);
+    __syncthreads();
+    if (p + 1 < passes) {
+#pragma unroll
+      for (int i = 0; i < kItems; ++i)
+        if (i < items) key[i] = Sm.sort.keys[wfirst + i * 32 + lane];
+      __syncthreads();
+    }
+  }
+  if (passes == 0) {
+#pragma unroll
+    for (int i = 0; i < kItems; ++i)
+      if (i < items) Sm.sort.keys[wfirst + i * 32 + lane] = key[i];
+    __syncthreads();
+  }
+
+  /* 4. queue boundaries of the ctx */
+  const uint32_t n_good = Sm.stage_first[S];             /* requests that passed the checks; the others follow them */
+  for (uint32_t k = tid; k < S; k += kSortThreads) {
+    const uint32_t v = first + Sm.stage_first[k];
+    a.seg_off[(size_t)c * S + k] = v;
+    if (a.out_seg_off) a.out_seg_off[(size_t)c * S + k] = v;
+    Sm.hb_kept[k] = Sm.stage_cnt[k];
+  }
+  if (c + 1 == a.n_ctx && tid == 0) {
+    a.seg_off[(size_t)a.n_ctx * S] = a.n;
+    if (a.out_seg_off) a.out_seg_off[(size_t)a.n_ctx * S] = a.n;
+  }
+  __syncthreads();
+  /* a queue served high budget first keeps a prefix: its length is the first position r with r >= u_r */
+  if (a.st.d_priority) {
+#pragma unroll 2
+    for (int i = 0; i < kItems; ++i) {
+      if (i >= items) break;
+      const uint32_t pos = wfirst + i * 32 + lane;
+      if (pos < n_good) {
+        const LocalElem x = local_decode(Sm.sort.keys[pos], pos, Sm, a.ibits, dbits, dmask, imask);
+        if (x.high_first && x.r >= x.u) atomicMin(&Sm.hb_kept[x.stage], x.r);
+      }
+    }
+    __syncthreads();
+  }
+
+  /* 5. segmented scan, first time: what every warp's elements add up to.  kGroup rounds are
+   * scanned side by side (their shuffles do not wait for each other), then chained. */
+  constexpr int kGroup = 4;
+  static_assert(kItems % kGroup == 0, "whole groups");
+  SegVal run = seg_identity<RAW>();
+  for (int i0 = 0; i0 < kItems; i0 += kGroup) {
+    if (i0 >= items) break;
+    SegVal v[kGroup];
+#pragma unroll
+    for (int g = 0; g < kGroup; ++g) {
+      const uint32_t pos = wfirst + (i0 + g) * 32 + lane;
+      v[g] = seg_identity<RAW>();
+      if (i0 + g < items && pos < n_good) {
+        const LocalElem x = local_decode(Sm.sort.keys[pos], pos, Sm, a.ibits, dbits, dmask, imask);
+        v[g].head = x.r == 0 ? 1u : 0u;
+        v[g].m = RAW ? (x.r < x.u ? 1 : 0) : (int32_t)x.u - (int32_t)x.r;
+      }
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+      for (int g = 0; g < kGroup; ++g) {
+        SegVal l;
+        l.m = __shfl_up_sync(0xffffffffu, v[g].m, o);
+        l.head = __shfl_up_sync(0xffffffffu, v[g].head, o);
+        if (lane >= (uint32_t)o) v[g] = seg_combine<RAW>(l, v[g]);
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < kGroup; ++g) {
+      SegVal all;
+      all.m = __shfl_sync(0xffffffffu, v[g].m, 31);
+      all.head = __shfl_sync(0xffffffffu, v[g].head, 31);
+      run = seg_combine<RAW>(run, all);
+    }
+  }
+  if (lane == 0) { Sm.wm[warp] = run.m; Sm.wh[warp] = run.head; }
+  __syncthreads();
+  SegVal carry = seg_identity<RAW>();
+#pragma unroll
+  for (int w = 0; w < WARPS; ++w) {
+    SegVal t; t.m = Sm.wm[w]; t.head = Sm.wh[w];
+    if (w < (int)warp) carry = seg_combine<RAW>(carry, t);
+  }
+
+  /* 6. second time: every request's position, estimate and decision; outputs */
+  for (int i0 = 0; i0 < kItems; i0 += kGroup) {
+    if (i0 >= items) break;
+    SegVal v[kGroup];
+    LocalElem x[kGroup];
+    unsigned long long e[kGroup];
+#pragma unroll
+    for (int g = 0; g < kGroup; ++g) {
+      const uint32_t pos = wfirst + (i0 + g) * 32 + lane;
+      v[g] = seg_identity<RAW>();
+      x[g].stage = 0; x[g].idx = 0; x[g].r = 0; x[g].u = 0; x[g].high_first = false;
+      e[g] = 0;
+      if (i0 + g < items && pos < cnt) e[g] = Sm.sort.keys[pos];
+      if (i0 + g < items && pos < n_good) {
+        x[g] = local_decode(e[g], pos, Sm, a.ibits, dbits, dmask, imask);
+        v[g].head = x[g].r == 0 ? 1u : 0u;
+        v[g].m = RAW ? (x[g].r < x[g].u ? 1 : 0) : (int32_t)x[g].u - (int32_t)x[g].r;
+      }
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+      for (int g = 0; g < kGroup; ++g) {
+        SegVal l;
+        l.m = __shfl_up_sync(0xffffffffu, v[g].m, o);
+        l.head = __shfl_up_sync(0xffffffffu, v[g].head, o);
+        if (lane >= (uint32_t)o) v[g] = seg_combine<RAW>(l, v[g]);
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < kGroup; ++g) {
+      const uint32_t pos = wfirst + (i0 + g) * 32 + lane;
+      const bool valid = i0 + g < items && pos < n_good;
+      SegVal exc;
+      exc.m = __shfl_up_sync(0xffffffffu, v[g].m, 1);
+      exc.head = __shfl_up_sync(0xffffffffu, v[g].head, 1);
+      if (lane == 0) exc = seg_identity<RAW>();
+      const SegVal pre = seg_combine<RAW>(carry, exc);   /* over the earlier requests of the same queue */
+      SegVal all;
+      all.m = __shfl_sync(0xffffffffu, v[g].m, 31);
+      all.head = __shfl_sync(0xffffffffu, v[g].head, 31);
+      carry = seg_combine<RAW>(carry, all);
+      if (i0 + g < items && pos < cnt) {
+        const uint32_t gpos = first + pos;
+        uint32_t keep = 0;
+        long long est = 0;
+        if (valid) {
+          const PardSegConst& K = Sm.K[x[g].stage];
+          uint32_t cpos, ahead;                          /* batch-slot position; kept requests ahead in the queue */
+          if (RAW) {
+            cpos = x[g].r;
+            ahead = x[g].r == 0 ? 0u : (uint32_t)pre.m;
+          } else {
+            if (x[g].r == 0) cpos = 0;
+            else {
+              const long long cc = (long long)x[g].r - 1 + pre.m;
+              cpos = cc < (long long)x[g].r ? (uint32_t)cc : x[g].r;
+            }
+            if (x[g].high_first) cpos = min(x[g].r, Sm.hb_kept[x[g].stage]);
+            ahead = cpos;
+          }
+          const uint32_t round = K.cap_magic ? div_magic32(cpos, K.cap_magic) : cpos;
+          est = K.A + (long long)round * K.d;
+          keep = (cpos < x[g].u && !(K.narrow & kSegNoStage)) ? 1u : 0u;
+          if (K.narrow & kSegNoStage) set_status(hdr, PARD_EDATA);
+          if (keep && a.kept_tmp) a.kept_tmp[first + Sm.stage_first[x[g].stage] + ahead] = x[g].idx;
+          if (x[g].r + 1 == Sm.stage_cnt[x[g].stage]) Sm.stage_kept[x[g].stage] = ahead + keep;   /* the queue's last request */
+        }
+        if (a.out_keep) a.out_keep[gpos] = (uint8_t)keep;
+        if (a.out_est) a.out_est[gpos] = est;
+        if (a.out_perm) a.out_perm[gpos] = (uint32_t)e[g] & imask;
+      }
+    }
+  }
+  __syncthreads();
+  for (uint32_t k = tid; k < S; k += kSortThreads) {
+    a.seg_kept[(size_t)c * S + k] = Sm.stage_kept[k];
+    if (single && a.out_seg_kept) a.out_seg_kept[k] = Sm.stage_kept[k];
+  }
+  if (!single) return;
+
+  /* 7. one ctx: pack the survivors here (queue after queue) and finish the call */
+  if (warp == 0) {
+    uint32_t run_k = 0;
+    for (uint32_t k0 = 0; k0 < S; k0 += 32) {
+      const uint32_t k = k0 + lane;
+      const uint32_t v = k < S ? Sm.stage_kept[k] : 0u;
+      uint32_t y = v;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t z = __shfl_up_sync(0xffffffffu, y, o);
+        if (lane >= (uint32_t)o) y += z;
+      }
+      if (k < S) Sm.kept_base[k] = run_k + y - v;
+      run_k += __shfl_sync(0xffffffffu, y, 31);
+    }
+    if (lane == 0) {
+      Sm.kept_base[S] = run_k;
+      if (a.out_n_kept) *a.out_n_kept = run_k;
+    }
+  }
+  __threadfence_block();
+  __syncthreads();
+  if (a.out_kept_idx && a.kept_tmp)
+    for (uint32_t k = 0; k < S; ++k) {
+      const uint32_t nk = Sm.stage_kept[k], from = Sm.stage_first[k], to = Sm.kept_base[k];
+      for (uint32_t i = tid; i < nk; i += kSortThreads) a.out_kept_idx[to + i] = a.kept_tmp[from + i];
+    }
+}
+
 /* ---- optional phase timing (process-wide) ---- */
 constexpr int kEventsPerSample = PARD_N_PHASES + 1;
 static_assert(PARD_N_PHASES == 4 + kMaxPasses + 3, "phase list");
@@ -1953,6 +2419,10 @@ int allow_sort_smem(int dev) {
                                       (int)sizeof(SortSmem)));
     PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_local, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_plan_local<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(LocalSmem)));
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_plan_local<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(LocalSmem)));
     done[dev].store(true, std::memory_order_release);
   }
   return PARD_OK;
@@ -2013,7 +2483,9 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   if (!pipelines || n_pipelines < 1 || !out) return PARD_EINVAL;
   if (n_pipelines > kMaxPipelinesPerCall) return PARD_ERANGE;
   constexpr uint32_t kRuleBits = PARD_MODE_PATH_MASK | PARD_MODE_FCFS | PARD_MODE_NEXUS | PARD_MODE_CLIPPER;
-  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN | PARD_MODE_TEST_STALL | kRuleBits)) return PARD_EINVAL;
+  if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN | PARD_MODE_TEST_STALL | PARD_MODE_GROUPED | kRuleBits))
+    return PARD_EINVAL;
+  if ((mode & PARD_MODE_GROUPED) && n > (uint64_t)n_ctx * (uint64_t)kSortTile) return PARD_EINVAL;   /* some ctx must exceed a tile */
   /* the rules decided by a walk of every queue, and what they combine with */
   const bool rule_walk = (mode & kRuleBits) != 0;
   const bool arrival_order = (mode & (PARD_MODE_FCFS | PARD_MODE_NEXUS | PARD_MODE_CLIPPER)) != 0;
@@ -2092,24 +2564,62 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     ++phase;
   };
   mark();
-  /* ---- clear the scratch that must start at zero: one contiguous region ---- */
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  {
-    const unsigned long long n16 = (n > 0 ? L.zero_end : L.lookback) / 16;   /* offsets are multiples of 256 */
-    launch_pdl(k_clear, (uint32_t)std::min<unsigned long long>((n16 + 255) / 256, (unsigned long long)sms * 4), 256, 0,
-               stream, (uint4*)(ws + L.hdr), n16);
-  }
   PipeTable pipe_table = {};
   pipe_table.many = d_pipes;
   if (n_pipelines <= (uint32_t)kFewPipelines)
     for (uint32_t i = 0; i < n_pipelines; ++i) pipe_table.few[i] = h_pipes[i];
   else
     PARD_CUDA_OK(cudaMemcpyAsync(d_pipes, h_pipes.data(), 8ull * n_pipelines, cudaMemcpyHostToDevice, stream));
-
   rc = allow_sort_smem(dev);
   if (rc != PARD_OK) return rc;
   const uint4* req4 = (const uint4*)d_requests;
+
+  /* ---- a block per ctx does everything (k_plan_local): a single ctx within one tile, or the
+   * caller's word that the requests come grouped by ctx with no ctx beyond a tile ---- */
+  const bool fused_single = n_ctx == 1 && n > 0 && n <= (uint64_t)kSortTile && !rule_walk;
+  /* worth it while the blocks fit a few waves: beyond that the streaming decision kernel of the
+   * general path (which finds the grouping by itself) does the positions cheaper than the blocks' scans */
+  const bool fused_grouped = (mode & PARD_MODE_GROUPED) && n_ctx > 1 && n > 0 && !rule_walk && n_ctx <= 4u * (uint32_t)sms;
+  if (fused_single || fused_grouped) {
+    LocalArgs la = {};
+    la.req = req4; la.ctx_start = fused_single ? nullptr : ctx_start;
+    la.n = n32; la.n_ctx = n_ctx; la.ibits = ibits; la.raw = (mode & PARD_MODE_RAW) ? 1u : 0u;
+    la.pipes = pipe_table; la.n_pipelines = n_pipelines; la.st = *state;
+    la.out_keep = out->d_keep; la.out_est = (long long*)out->d_est_us; la.out_perm = out->d_perm;
+    la.out_kept_idx = out->d_kept_idx; la.out_n_kept = (unsigned long long*)out->d_n_kept;
+    la.out_seg_off = out->d_seg_offsets; la.out_seg_kept = out->d_seg_kept;
+    la.ktab = ktab; la.seg_off = seg_off; la.seg_kept = seg_kept; la.kept_tmp = out->d_kept_idx ? kept_tmp : nullptr;
+    if (fused_grouped) {
+      launch_pdl(k_clear, 4, 256, 0, stream, (uint4*)(ws + L.hdr), (unsigned long long)(L.hist / 16));
+      launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
+      /* the queues' constants; what depends on a ctx's deadline range is added by the ctx's block */
+      launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax,
+                 ktab, hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
+    }
+    launch_pdl((mode & PARD_MODE_RAW) ? k_plan_local<true> : k_plan_local<false>, n_ctx, kSortThreads, sizeof(LocalSmem),
+               stream, hdr, la);
+    if (fused_grouped) {
+      launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+                 (unsigned long long*)out->d_n_kept);
+      if (out->d_kept_idx)
+        launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
+                                                   (uint32_t)sms * 8), 256, 0, stream,
+                   kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
+    }
+    while (phase <= PARD_N_PHASES) mark();             /* the phases are those of the other path: all of this counts as the first */
+    PARD_CUDA_OK(cudaGetLastError());
+    if (mode & PARD_MODE_NOWAIT) return PARD_OK;
+    return pard_plan_status(d_workspace, cuda_stream);
+  }
+
+  /* ---- clear the scratch that must start at zero: one contiguous region ---- */
+  {
+    const unsigned long long n16 = (n > 0 ? L.zero_end : L.lookback) / 16;   /* offsets are multiples of 256 */
+    launch_pdl(k_clear, (uint32_t)std::min<unsigned long long>((n16 + 255) / 256, (unsigned long long)sms * 4), 256, 0,
+               stream, (uint4*)(ws + L.hdr), n16);
+  }
 
   mark();
   if (n > 0) {

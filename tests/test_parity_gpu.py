@@ -142,9 +142,10 @@ def test_multiple_pipelines_and_padded_rows():
     both(inputs.Workload("edge", [pa, pbig], r, st, n_ctx))
 
 
-def test_device_detected_errors():
+@pytest.mark.parametrize("n", [3000, 9000])     # planned by one block / by the kernels of the general path
+def test_device_detected_errors(n):
     p = util.pipeline(inputs.chain_edges(2), 2, [5, 6])
-    good = util.requests(np.arange(3000) + 100)
+    good = util.requests(np.arange(n) + 100)
     st = util.state(1, 2, 1, 10, 1)
     for bad_field, bad_val in (("stage", 2), ("ctx", 1), ("deadline_us", -5), ("deadline_us", 1 << 60)):
         r = good.copy()
@@ -161,7 +162,7 @@ def test_device_detected_errors():
     rc, _ = run_library(inputs.Workload("bad", [p], r, util.state(1, 3, 1, 10, 1), 1), check=False)
     assert rc == pb.PARD_EDATA
     # the same with a deadline far from the queue's start: the request's batch window (offset 2,500
-    # with the default duration of 1) lies beyond every window table (1,133 entries here); it must be
+    # with the default duration of 1) lies beyond the queue's window table; it must be
     # reported, not looked up (the offset stays below n, i.e. inside the caller's workspace)
     r = good.copy()
     r["stage"][2500] = 2
@@ -284,20 +285,85 @@ def _grouped(n_epochs=40, seed=0, keep_lo=0.3):
     return wl, rng
 
 
+def grouped(wl, mode=0):
+    """The same through PARD_MODE_GROUPED: one thread block plans each ctx from start to end."""
+    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, mode & 1)
+    rc, got = run_library(wl, mode | pb.PARD_MODE_GROUPED)
+    assert rc == 0
+    assert_identical(got, want)
+
+
 @pytest.mark.parametrize("mode", [0, 1])
 def test_grouped_contexts_take_the_local_sort(mode):
     wl, rng = _grouped(seed=1)
     both(wl, mode)
+    grouped(wl, mode)
     # some contexts empty, one with a single request
     wl, rng = _grouped(seed=2, keep_lo=0.5)
     r = wl.requests
     drop = np.isin(r["ctx"], [3, 4, 17]) | ((r["ctx"] == 9) & (np.arange(wl.n) != np.flatnonzero(r["ctx"] == 9)[0]))
     wl.requests = np.ascontiguousarray(r[~drop])
     both(wl, mode)
+    grouped(wl, mode)
     # queues served high budget first among them
     wl, rng = _grouped(seed=3)
     wl.state.priority = rng.integers(0, 2, size=(wl.n_ctx, wl.state.stage_stride)).astype(np.uint8)
     both(wl, mode)
+    grouped(wl, mode)
+
+
+@pytest.mark.parametrize("name,kw", [("C4", {"n_epochs": 37, "per_epoch": 1000}), ("C4b", {"n_epochs": 64, "per_epoch": 8192}),
+                                     ("C5b", {"n_inst": 600, "per_inst": 301}), ("C5", {"n_inst": 9, "per_inst": 5001}),
+                                     ("C4b", {"n_epochs": 1100, "per_epoch": 200})])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_block_per_ctx_on_the_grouped_configs(name, kw, mode):
+    grouped(inputs.make(name, **kw), mode)
+
+
+def test_block_per_ctx_full_size():
+    grouped(inputs.make("C4"))
+
+
+def test_single_small_ctx_is_one_block():
+    """One ctx of at most a sort tile: the whole call is one kernel; sizes around the limit."""
+    for n in (1, 2, 31, 33, 4097, 8191, 8192, 8193):
+        both(inputs.make("C1b", n=n))
+        both(inputs.make("C1", n=n), mode=1)
+    # many stages, a DAG, priorities
+    wl = inputs.make("C3b", n=8000)
+    wl.state.priority = np.random.default_rng(4).integers(0, 2, size=(1, wl.state.stage_stride)).astype(np.uint8)
+    both(wl)
+    both(wl, mode=1)
+
+
+def test_broken_grouping_promise_is_reported():
+    wl, rng = _grouped(seed=4)
+    r = wl.requests.copy()
+    i, j = 5, wl.n - 7
+    r[[i, j]] = r[[j, i]]                                        # two requests far from their ctx's group
+    wl.requests = r
+    rc, _ = run_library(wl, pb.PARD_MODE_GROUPED, check=False)
+    assert rc == pb.PARD_EDATA
+    wl, rng = _grouped(seed=5, keep_lo=0.9)
+    r = wl.requests.copy()
+    r["ctx"][r["ctx"] == 21] = 20                                # ctx 20 now holds two epochs: more than a tile
+    wl.requests = r
+    rc, _ = run_library(wl, pb.PARD_MODE_GROUPED, check=False)
+    assert rc == pb.PARD_EDATA
+    # more requests than the contexts could hold: refused before anything is launched
+    big = inputs.make("C5b", n_inst=2, per_inst=9000)
+    rc, _ = run_library(big, pb.PARD_MODE_GROUPED, check=False)
+    assert rc == pb.PARD_EINVAL
+    # input errors inside a block-planned ctx
+    wl = inputs.make("C1b")
+    wl.requests["stage"][100] = 7
+    rc, _ = run_library(wl, 0, check=False)
+    assert rc == pb.PARD_EDATA
+    wl = inputs.make("C1b")
+    wl.requests["ctx"][100] = 3
+    rc, _ = run_library(wl, 0, check=False)
+    assert rc == pb.PARD_EDATA
+    both(inputs.make("C1b"))                                     # the context still works
 
 
 def test_grouped_contexts_fall_back_when_the_device_says_no():

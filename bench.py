@@ -189,15 +189,18 @@ def run_reference(args):
 class DevicePlan:
     """Device-resident workload, outputs and workspace for repeated planning."""
 
-    def __init__(self, wl, dev, mode=0):
+    def __init__(self, wl, dev, mode=0, arrivals=None):
         import torch
         self.mode = mode
+        self.d_arr = None
         from paper_2602_08747_b200 import binding as pb
         self.pb, self.torch, self.wl, self.dev = pb, torch, wl, dev
         self.S = wl.state.stage_stride
         self.n_seg = wl.n_ctx * self.S
         self.pipes = [pb.pard_load_pipeline(p) for p in wl.pipelines]
         self.d_req = pb.device_requests(wl.requests, dev)
+        if arrivals is not None:
+            self.d_arr = pb.device_requests(arrivals, dev)       # 16-byte records as well
         self.d_state = pb.device_state(wl.state, dev)
         self.out = pb.alloc_out(wl.n, self.n_seg, dev)
         self.ws = pb.alloc_workspace(pb.pard_plan_workspace_bytes(wl.n, wl.n_ctx, self.S), dev)
@@ -208,8 +211,13 @@ class DevicePlan:
 
     def step(self, nowait=True):
         pb, wl = self.pb, self.wl
-        pb.pard_plan(self.pipes, self.d_req, wl.n, self.d_state, wl.n_ctx,
-                     self.mode | (pb.PARD_MODE_NOWAIT if nowait else 0), self.out, self.ws, stream=self.stream)
+        rules = pb.PARD_MODE_PATH_MASK | pb.PARD_MODE_FCFS | pb.PARD_MODE_NEXUS | pb.PARD_MODE_CLIPPER
+        if self.mode & rules:
+            pb.pard_plan_policy(self.pipes, self.d_req, self.d_arr, wl.n, self.d_state, wl.n_ctx,
+                                self.mode | (pb.PARD_MODE_NOWAIT if nowait else 0), self.out, self.ws, stream=self.stream)
+        else:
+            pb.pard_plan(self.pipes, self.d_req, wl.n, self.d_state, wl.n_ctx,
+                         self.mode | (pb.PARD_MODE_NOWAIT if nowait else 0), self.out, self.ws, stream=self.stream)
         pb.pard_goodput(None, self.out.seg_offsets, self.out.seg_kept, wl.n, wl.n_ctx, self.S, self.total,
                         self.kept, stream=self.stream)
 
@@ -471,6 +479,26 @@ def run_aux(dev, peak, kernels_only=False):
     out["pard_plan_mixed_priority"] = {"workload": WORKLOAD + "b, priorities drawn per queue", "ms": 1e3 * sec / 40,
                                        "requests_per_s": wlh.n * 40 / sec}
     del plan
+
+    # the comparison rules and order variants on the balanced 2^24-request workload
+    rules = {}
+    wlr = inputs.make(WORKLOAD + "b", seed=2)
+    rr = np.random.default_rng(4)
+    arr = np.zeros(wlr.n, dtype=inputs.ARRIVAL_DTYPE)
+    arr["arrive_us"] = np.maximum(0, wlr.state.now_us[0] - rr.integers(0, 400_000, size=wlr.n))
+    arr["slo_us"] = rr.integers(100_000, 400_000, size=wlr.n)
+    masked = wlr.requests.copy()
+    masked["flags"] = rr.integers(0, 4, size=wlr.n)            # unknown, first, second, either of the first two paths
+    for label, mode, a, req in (("known_paths", pb.PARD_MODE_PATH_MASK, None, masked), ("arrival_order", pb.PARD_MODE_FCFS, None, None),
+                                ("nexus", pb.PARD_MODE_NEXUS, None, None), ("clipper_pp", pb.PARD_MODE_CLIPPER, arr, None)):
+        w2 = wlr if req is None else inputs.Workload(wlr.name, wlr.pipelines, req, wlr.state, wlr.n_ctx)
+        plan = DevicePlan(w2, dev, mode, a)
+        plan.step(nowait=False)
+        kf = float(plan.out.n_kept.cpu()[0]) / w2.n
+        sec, _ = timed_steps(plan, 10, 3, None)
+        rules[label] = {"ms": 1e3 * sec / 10, "requests_per_s": w2.n * 10 / sec, "keep_fraction": kf}
+        del plan
+    out["comparison_rules"] = {"workload": WORKLOAD + "b (16 queues of about 2^20 requests: one warp walks each queue)", **rules}
 
     # closed-loop replay: 16 instances, 64 epochs of 65,536 requests
     job_rng = np.random.default_rng(11)

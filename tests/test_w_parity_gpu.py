@@ -133,3 +133,22 @@ def test_estimate_feeds_the_planner():
     want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, 0)
     for k in ("keep", "est_us", "perm", "seg_kept"):
         assert np.array_equal(got[k], want[k]), k
+
+
+@pytest.mark.parametrize("name,kw", [("C1", {}), ("C1b", {}), ("C2b", {"n": 60_001}), ("C3b", {"n": 200_003}),
+                                     ("C4b", {"n_epochs": 12, "per_epoch": 4000}), ("C5b", {"n_inst": 7, "per_inst": 9001})])
+def test_configs_with_w_from_the_estimator(name, kw):
+    """The five workloads with their batch-wait estimates produced by the State Planner's own
+    estimator instead of being drawn: M = 10,000 recorded waits per stage, uniform on [0, d) (Sec. 3.2,
+    Fig. 3b), lambda = 0.1 (Sec. 4.2).  Each side estimates w itself and plans with its own w."""
+    wl = inputs.make(name, **kw)
+    samples = inputs.draw_wait_samples(np.random.default_rng(3), wl, 10_000)
+    rc, w = gpu_util.run_estimate_w(wl, samples, 1, 10, 7)
+    assert rc == pb.PARD_OK
+    w_or = oracle_w(wl, samples, 1, 10, 7)
+    wl.state.w_us = np.where(w < 0, 0, w)
+    rc, got = gpu_util.run_library(wl)
+    assert rc == 0
+    wl.state.w_us = np.where(w_or < 0, 0, w_or)
+    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, 0)
+    gpu_util.assert_identical(got, want)

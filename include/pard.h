@@ -266,6 +266,13 @@ int pard_plan_workspace_bytes(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
  * stream); the call then waits for the stream and reads back one status word,
  * so a PARD_EDATA / PARD_ETIMEOUT found on the device is returned here.  The
  * library allocates no device memory in this call.
+ * Keys wider than one sort element: when the bits of the segment id, of the
+ * widest per-ctx deadline span and of the request index add up to more than
+ * 64 (e.g. 2^14 requests in 64 queues with deadlines 2^59 us apart), the call
+ * finds that out on the device, then sorts the key in chunks and walks the
+ * queues (same results, several times slower).  That second stage needs the
+ * first one's report, so it only runs in the waiting form of the call; with
+ * PARD_MODE_NOWAIT such a call leaves PARD_ERANGE for pard_plan_status.
  * Host-detectable errors are returned before anything is launched.
  * Performance note: requests may come in any order.  When they come grouped by
  * ascending ctx and no ctx holds more than 8,192 of them (batched decision

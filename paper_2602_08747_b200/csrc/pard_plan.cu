@@ -2377,6 +2377,126 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
     }
 }
 
+/* ------------------------------------------------------------------------ */
+/* keys wider than one sort element                                          */
+/* ------------------------------------------------------------------------ */
+/* When segment, deadline and index bits together exceed 64 (deadline spans of years, millions
+ * of queues and requests at once) the key (segment | deadline offset, up to 84 bits) is sorted
+ * in chunks, least significant first, each chunk by the ordinary passes: a chunk's element is
+ * chunk << ibits | current position, so every super-pass is a stable sort of the current
+ * order by one more chunk, and the positions it yields are chased back to request indices.
+ * The last super-pass leaves the order of the requests; the elements are then rewritten as
+ * segment | index (no deadline bits) and the decision is taken by the queue walk, which looks
+ * the deadlines up in the request array.  A slow path for legal but extreme inputs. */
+__device__ __forceinline__ uint32_t wide_chunk_bits(const PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t super) {
+  const uint32_t kb = sbits + hdr->dbits, cw = 64 - ibits, lo = super * cw;
+  return lo < kb ? min(cw, kb - lo) : 0u;
+}
+
+__global__ void __launch_bounds__(256)
+k_wide_reset(PlanHeader* hdr, uint32_t* __restrict__ hist, uint32_t* __restrict__ lookback, unsigned long long lb_words,
+             uint32_t sbits, uint32_t ibits, uint32_t super) {
+  pdl_wait();
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    hdr->npass = (wide_chunk_bits(hdr, sbits, ibits, super) + 7) / 8;
+    for (int i = 0; i <= kMaxPasses; ++i) hdr->ticket[i] = 0;
+    if (super == 0) {
+      hdr->wide = 2;                                      /* the chunked sort is under way */
+      hdr->status = hdr->bad_input ? (uint32_t)(-PARD_EDATA) : 0u;   /* the width was not an error after all */
+    }
+  }
+  const unsigned long long step = (unsigned long long)gridDim.x * blockDim.x;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < lb_words + kMaxPasses * kBins; i += step) {
+    if (i < lb_words) lookback[i] = 0;
+    else hist[i - lb_words] = 0;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+k_wide_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
+            const unsigned long long* __restrict__ ctx_dmin_inv, const unsigned long long* __restrict__ ctx_dmax,
+            const uint8_t* __restrict__ priority, uint32_t sbits, uint32_t ibits, uint32_t super,
+            const PlanHeader* __restrict__ hdr, const uint32_t* __restrict__ order,
+            unsigned long long* __restrict__ dst, uint32_t* __restrict__ hist) {
+  pdl_wait();
+  __shared__ uint32_t s_hist[kMaxPasses * kBins];
+  const uint32_t bits = wide_chunk_bits(hdr, sbits, ibits, super), npass = (bits + 7) / 8;
+  const uint32_t dbits = hdr->dbits, lo = super * (64 - ibits);
+  for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
+  __syncthreads();
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t p = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += stride) {
+    const uint32_t orig = super == 0 ? (uint32_t)p : order[p];
+    const uint4 r = __ldg(&req[orig]);
+    const unsigned long long D = ((unsigned long long)r.y << 32) | r.x;
+    const uint32_t ctx = r.z, stage = r.w & 0xffffu;
+    unsigned long long chunk = 0;
+    if (ctx < n_ctx && stage < S && D < (unsigned long long)PARD_TIME_LIMIT_US && bits) {
+      const uint32_t seg = ctx * S + stage;
+      const bool high_first = priority && __ldg(&priority[seg]) != 0;
+      const unsigned long long off = high_first ? ctx_dmax[ctx] - D : D - ~ctx_dmin_inv[ctx];
+      const unsigned __int128 key = ((unsigned __int128)seg << dbits) | off;
+      chunk = (unsigned long long)(key >> lo) & (bits >= 64 ? ~0ull : ((1ull << bits) - 1));
+    }
+    dst[p] = (chunk << ibits) | p;                        /* flagged requests sort first, into queue 0 */
+    for (uint32_t q = 0; q < npass; ++q) atomicAdd(&s_hist[q * kBins + ((chunk >> (8 * q)) & 255u)], 1u);
+  }
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x)
+    if (s_hist[i]) atomicAdd(&hist[i], s_hist[i]);
+}
+
+/* positions of a super-pass -> request indices, into the buffer the sort has left free */
+__global__ void __launch_bounds__(256)
+k_wide_chase(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+             unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t super,
+             const uint32_t* __restrict__ order) {
+  pdl_wait();
+  const bool odd = hdr->npass & 1;
+  const unsigned long long* sorted = odd ? buf_b : buf_a;
+  uint32_t* tmp = reinterpret_cast<uint32_t*>(odd ? const_cast<unsigned long long*>(buf_a) : buf_b);
+  const uint32_t imask = (1u << ibits) - 1;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n; q += stride) {
+    const uint32_t pos = (uint32_t)sorted[q] & imask;
+    tmp[q] = super == 0 ? pos : order[pos];
+  }
+}
+
+__global__ void __launch_bounds__(256)
+k_wide_keep(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+            const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t* __restrict__ order) {
+  pdl_wait();
+  const uint32_t* tmp = reinterpret_cast<const uint32_t*>((hdr->npass & 1) ? buf_a : buf_b);
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n; q += stride) order[q] = tmp[q];
+}
+
+/* the sorted order as elements without deadline bits: segment | request index, in buf_a */
+__global__ void __launch_bounds__(256)
+k_wide_final(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S, uint32_t sbits, uint32_t ibits,
+             PlanHeader* hdr, const uint32_t* __restrict__ order, unsigned long long* __restrict__ buf_a) {
+  pdl_wait();
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; q < n; q += stride) {
+    const uint32_t orig = order[q];
+    const uint4 r = __ldg(&req[orig]);
+    const unsigned long long D = ((unsigned long long)r.y << 32) | r.x;
+    const uint32_t ctx = r.z, stage = r.w & 0xffffu;
+    const bool ok = ctx < n_ctx && stage < S && D < (unsigned long long)PARD_TIME_LIMIT_US;
+    buf_a[q] = ((unsigned long long)(ok ? ctx * S + stage : 0u) << ibits) | orig;
+  }
+}
+
+/* after k_wide_final: the header as the kernels behind the sort expect it */
+__global__ void k_wide_done(PlanHeader* hdr, uint32_t sbits) {
+  pdl_wait();
+  hdr->dbits = 0;
+  hdr->keybits = sbits;
+  hdr->npass = 0;
+  hdr->wide = 0;
+}
+
 /* ---- optional phase timing (process-wide) ---- */
 constexpr int kEventsPerSample = PARD_N_PHASES + 1;
 static_assert(PARD_N_PHASES == 4 + kMaxPasses + 3, "phase list");
@@ -2576,6 +2696,70 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   if (rc != PARD_OK) return rc;
   const uint4* req4 = (const uint4*)d_requests;
 
+  /* ---- keys wider than one sort element: see k_wide_reset.  Run only when a finished call has
+   * reported that width (the host cannot know the deadline span beforehand), hence not for
+   * PARD_MODE_NOWAIT, whose caller gets PARD_ERANGE from pard_plan_status as before. ---- */
+  auto plan_wide = [&]() -> int {
+    uint32_t h_wide = 0;
+    PARD_CUDA_OK(cudaMemcpyAsync(&h_wide, &hdr->wide, 4, cudaMemcpyDeviceToHost, stream));
+    PARD_CUDA_OK(cudaStreamSynchronize(stream));
+    if (!h_wide) return PARD_ERANGE;
+    const uint32_t grid_n = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
+    {
+      const unsigned long long n16 = L.zero_end / 16;
+      launch_pdl(k_clear, (uint32_t)std::min<unsigned long long>((n16 + 255) / 256, (unsigned long long)sms * 4), 256, 0,
+                 stream, (uint4*)(ws + L.hdr), n16);
+    }
+    launch_pdl(k_prepass, (uint32_t)std::min<uint64_t>((n + 2047) / 2048, (uint64_t)sms * 8), 256, 0, stream, req4, n32, n_ctx,
+               S, ctx_dmin, ctx_dmax, hdr);
+    launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
+    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr, 0u);
+    launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
+               hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
+    const uint32_t cw = 64 - ibits;                         /* key bits per super-pass */
+    const uint32_t supers = (sbits + 60 + cw - 1) / cw;     /* for the widest legal span; chunks beyond the key are empty */
+    const uint32_t chunk_passes = std::min<uint32_t>(kMaxPasses, (cw + 7) / 8);
+    uint32_t* order = kept_tmp;
+    for (uint32_t sp = 0; sp < supers; ++sp) {
+      launch_pdl(k_wide_reset, (uint32_t)std::min<uint64_t>((lb_words + kMaxPasses * kBins + 255) / 256, (uint64_t)sms * 4), 256,
+                 0, stream, hdr, hist, lookback, (unsigned long long)lb_words, sbits, ibits, sp);
+      launch_pdl(k_wide_pack, grid_n, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, sbits, ibits,
+                 sp, (const PlanHeader*)hdr, (const uint32_t*)order, buf_a, hist);
+      for (uint32_t p = 0; p < chunk_passes; ++p)
+        launch_pdl(k_sort_pass<false>, L.sort_tiles, kSortThreads, sizeof(SortSmem), stream, p, hdr, buf_a, buf_b, hist,
+                   lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words, n32, ibits, 0u, 0u);
+      launch_pdl(k_wide_chase, grid_n, 256, 0, stream, (const PlanHeader*)hdr, (const unsigned long long*)buf_a, buf_b, n32,
+                 ibits, sp, (const uint32_t*)order);
+      launch_pdl(k_wide_keep, grid_n, 256, 0, stream, (const PlanHeader*)hdr, (const unsigned long long*)buf_a,
+                 (const unsigned long long*)buf_b, n32, order);
+    }
+    launch_pdl(k_wide_final, grid_n, 256, 0, stream, req4, n32, n_ctx, S, sbits, ibits, hdr, (const uint32_t*)order, buf_a);
+    launch_pdl(k_wide_done, 1, 1, 0, stream, hdr, sbits);
+    if (L.n_seg >= kManyQueues)
+      launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
+                 seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity, 0u, 0u);
+    else
+      launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
+                 out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity, 0u, (const uint32_t*)hist, sbits, 0u, 0u);
+    PolicyArgs pa = {};
+    pa.hdr = hdr; pa.buf_a = buf_a; pa.buf_b = buf_b;
+    pa.n = n32; pa.ibits = ibits; pa.n_seg = L.n_seg; pa.mode = mode;
+    pa.ktab = ktab; pa.seg_off = seg_off; pa.req = req4; pa.arrivals = d_arrivals;
+    pa.pipes = pipe_table; pa.n_pipelines = n_pipelines; pa.st = *state;
+    pa.out_keep = out->d_keep; pa.out_est = (long long*)out->d_est_us; pa.out_perm = out->d_perm;
+    pa.kept_tmp = out->d_kept_idx ? kept_tmp : nullptr; pa.seg_kept = seg_kept;
+    int wrc = launch_policy_decision(pa, sms, stream);
+    if (wrc != PARD_OK) return wrc;
+    launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+               (unsigned long long*)out->d_n_kept);
+    if (out->d_kept_idx)
+      launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
+                                                 (uint32_t)sms * 8), 256, 0, stream,
+                 kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
+    PARD_CUDA_OK(cudaGetLastError());
+    return pard_plan_status(d_workspace, cuda_stream);
+  };
+
   /* ---- a block per ctx does everything (k_plan_local): a single ctx within one tile, or the
    * caller's word that the requests come grouped by ctx with no ctx beyond a tile ---- */
   const bool fused_single = n_ctx == 1 && n > 0 && n <= (uint64_t)kSortTile && !rule_walk;
@@ -2611,7 +2795,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     while (phase <= PARD_N_PHASES) mark();             /* the phases are those of the other path: all of this counts as the first */
     PARD_CUDA_OK(cudaGetLastError());
     if (mode & PARD_MODE_NOWAIT) return PARD_OK;
-    return pard_plan_status(d_workspace, cuda_stream);
+    rc = pard_plan_status(d_workspace, cuda_stream);
+    return rc == PARD_ERANGE ? plan_wide() : rc;
   }
 
   /* ---- clear the scratch that must start at zero: one contiguous region ---- */
@@ -2726,7 +2911,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   mark();
   PARD_CUDA_OK(cudaGetLastError());
   if (mode & PARD_MODE_NOWAIT) return PARD_OK;
-  return pard_plan_status(d_workspace, cuda_stream);
+  rc = pard_plan_status(d_workspace, cuda_stream);
+  return (rc == PARD_ERANGE && n > 0) ? plan_wide() : rc;
 }
 
 extern "C" int pard_plan_status(const void* d_workspace, void* cuda_stream) {

@@ -50,11 +50,13 @@ struct PlanHeader {
   uint32_t seg_done;          /* blocks of k_seg_const that have stored their constants */
   uint32_t unsorted;          /* 1: some request's ctx is smaller than its predecessor's */
   uint32_t ctx_too_big;       /* 1: some ctx holds more requests than one sort tile */
-  uint32_t pad[64 - 16 - (kMaxPasses + 1)];
+  uint32_t bad_input;         /* 1: PARD_EDATA was found (kept apart from `status`, which holds the first error only) */
+  uint32_t pad[64 - 17 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 
 __device__ __forceinline__ void set_status(PlanHeader* hdr, int status) {
+  if (status == PARD_EDATA) hdr->bad_input = 1;
   atomicCAS(&hdr->status, 0u, (uint32_t)(-status));
 }
 

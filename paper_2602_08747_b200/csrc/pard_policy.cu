@@ -187,9 +187,23 @@ k_policy_terms(const PolicyArgs a) {
 
 /* One warp per queue.  General rule: x <- x + [x < u_r]. */
 __device__ void walk_admit(const uint32_t* __restrict__ T, uint32_t* __restrict__ C, uint32_t lo, uint32_t hi,
-                           uint32_t lane, uint32_t* kept_out) {
+                           uint32_t lane, uint32_t* kept_out, bool raw) {
   const uint32_t below = (1u << lane) - 1;
   uint32_t x = 0;
+  if (raw) {
+    /* every queued request ahead takes a batch slot: a request is kept iff its own queue position
+     * is below its threshold, whatever happened before it; what is walked is only the count of
+     * kept requests ahead (the survivor's slot) */
+    for (uint32_t b0 = lo; b0 < hi; b0 += 32) {
+      const uint32_t j = b0 + lane;
+      const bool keep = j < hi && (j - lo) < T[j];
+      const uint32_t m = __ballot_sync(0xffffffffu, keep);
+      if (j < hi) C[j] = (x + __popc(m & below)) | (keep ? kKeepBit : 0u);
+      x += __popc(m);
+    }
+    *kept_out = x;
+    return;
+  }
   constexpr int kAhead = 4;                        /* steps whose thresholds are requested together */
   for (uint32_t b0 = lo; b0 < hi; b0 += 32 * kAhead) {
     uint32_t u[kAhead];
@@ -275,7 +289,7 @@ k_policy_walk(const PolicyArgs a) {
   uint32_t kept = 0;
   if (hi > lo) {
     if (a.mode & PARD_MODE_NEXUS) walk_nexus(v.T, v.C, lo, hi, a.ktab[s].cap, lane, &kept);
-    else walk_admit(v.T, v.C, lo, hi, lane, &kept);
+    else walk_admit(v.T, v.C, lo, hi, lane, &kept, (a.mode & PARD_MODE_RAW) != 0);
   }
   if (lane == 0) a.seg_kept[s] = kept;
 }
@@ -300,9 +314,11 @@ k_policy_emit(const PolicyArgs a) {
     if (!(K.narrow & kSegNoStage)) {
       const Terms t = request_terms(a, sp, seg, idx, K);
       const uint32_t w = v.C[j];
-      c = w & ~kKeepBit;
+      c = w & ~kKeepBit;                           /* kept requests ahead in the queue */
       keep = w >> 31;
-      const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;     /* floor(c / cap) */
+      /* the batch-slot position: the kept requests ahead, or, when every request ahead takes a slot, all of them */
+      const uint32_t slot = (a.mode & PARD_MODE_RAW) ? (uint32_t)j - a.seg_off[seg] : c;
+      const uint32_t round = K.cap_magic ? div_magic32(slot, K.cap_magic) : slot;     /* floor(slot / cap) */
       est = t.A + (long long)round * K.d;
     }
     if (a.out_keep) a.out_keep[j] = (uint8_t)keep;

@@ -182,15 +182,64 @@ def test_bounded_wait_runs_out_and_is_reported():
     both(wl)
 
 
-def test_key_wider_than_64_bits_is_reported():
-    # 2^59 span * 2^14 requests * 64 segments does not fit one 64-bit sort element
+def test_key_wider_than_64_bits_is_sorted_in_chunks():
+    """Segment, deadline and index bits beyond one 64-bit sort element: the key is sorted in
+    chunks and the queues are walked; same plan as the oracle's."""
+    # 2^59 span * 2^14 requests * 64 segments
     p = util.pipeline(inputs.chain_edges(2), 2, [5, 6])
     n = 10_000
-    dl = np.arange(n, dtype=np.int64)
+    rng = np.random.default_rng(12)
+    dl = rng.integers(0, 200, size=n).astype(np.int64)
     dl[-1] = (1 << 59)
+    dl[17] = (1 << 59) - 3
     st = util.state(32, 2, 1, 10, 1)
-    rc, _ = run_library(inputs.Workload("wide", [p], util.requests(dl), st, 32), check=False)
-    assert rc == pb.PARD_ERANGE
+    r = util.requests(dl, stage=rng.integers(0, 2, size=n), ctx=rng.integers(0, 32, size=n))
+    wl = inputs.Workload("wide", [p], r, st, 32)
+    for mode in (0, 1):
+        want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, mode)
+        rc, got = run_library(wl, mode)
+        assert rc == 0
+        assert_identical(got, want)
+    # deadlines spread over the whole span, several super-passes, some queues served high budget first
+    n = 60_001
+    dl = rng.integers(0, 1 << 59, size=n)
+    dl[:5000] = rng.integers(0, 400, size=5000)                  # and a cluster that the planner keeps part of
+    st = util.state(700, 2, 1, 10, 2)
+    st.priority = rng.integers(0, 2, size=(700, 2)).astype(np.uint8)
+    r = util.requests(dl, stage=rng.integers(0, 2, size=n), ctx=rng.integers(0, 700, size=n))
+    wl = inputs.Workload("wide", [p], r, st, 700)
+    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, 0)
+    rc, got = run_library(wl, 0)
+    assert rc == 0
+    assert_identical(got, want)
+    # one small ctx (the one-block path finds the width and hands over)
+    p1 = util.pipeline(inputs.chain_edges(40), 40, [3] * 40)
+    dl = rng.integers(0, 1 << 59, size=5000)
+    dl[:2000] = rng.integers(0, 300, size=2000)
+    wl = inputs.Workload("wide", [p1], util.requests(dl, stage=rng.integers(0, 40, size=5000)),
+                         util.state(1, 40, inputs.n_slots(p1), 10, 2), 1)
+    assert 6 + 59 + 13 > 64
+    want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, 0)
+    rc, got = run_library(wl, 0)
+    assert rc == 0
+    assert_identical(got, want)
+
+
+def test_wide_key_without_waiting_is_reported():
+    """With PARD_MODE_NOWAIT nothing is read back, so the chunked sort cannot be started: the
+    width is reported by pard_plan_status."""
+    import torch
+    p = util.pipeline(inputs.chain_edges(2), 2, [5, 6])
+    dl = np.arange(10_000, dtype=np.int64)
+    dl[-1] = 1 << 59
+    wl = inputs.Workload("wide", [p], util.requests(dl), util.state(32, 2, 1, 10, 1), 32)
+    pipes = [pb.pard_load_pipeline(q) for q in wl.pipelines]
+    ws = pb.alloc_workspace(pb.pard_plan_workspace_bytes(wl.n, 32, 2))
+    out = pb.alloc_out(wl.n, 64)
+    stream = torch.cuda.current_stream().cuda_stream
+    assert pb.pard_plan(pipes, pb.device_requests(wl.requests), wl.n, pb.device_state(wl.state), 32, pb.PARD_MODE_NOWAIT,
+                        out, ws, stream=stream, check=False) == pb.PARD_OK
+    assert pb.pard_plan_status(ws, stream, check=False) == pb.PARD_ERANGE
 
 
 def test_workspace_too_small_and_foreign_handle():

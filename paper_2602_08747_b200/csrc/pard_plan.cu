@@ -1079,44 +1079,39 @@ __device__ void tile_scan_block(const unsigned long long* tile_agg, uint32_t n_t
  * aggregates into the value carried into every tile, so that the decision
  * kernel never waits on another block. */
 template <bool RAW>
-__global__ void __launch_bounds__(kDecThreads)
-k_tile_agg(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
-           const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
-           const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
-           unsigned long long* __restrict__ tile_agg, int32_t* __restrict__ carry) {
-  pdl_wait();
+__device__ void tile_agg_tiles(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+                               const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
+                               const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+                               unsigned long long* __restrict__ tile_agg) {
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
   for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-  const uint64_t base = (uint64_t)tile * kDecTile + (uint64_t)tid * kDecItems;
-  unsigned long long e[kDecItems];
-  uint32_t idx[kDecItems], u[kDecItems], r[kDecItems], lheadbits, sstart, seg_first;
-  int32_t lv[kDecItems];
-  SegVal run;
-  PardSegConst K;
-  bool one_seg;
-  tile_first_half<RAW>(T, base, e, idx, u, r, lv, lheadbits, run, K, sstart, seg_first, one_seg);
-  const SegVal inc = warp_scan<RAW>(run, lane);
-  if (lane == 31) { s_wm[warp] = inc.m; s_wh[warp] = inc.head; }
-  __syncthreads();
-  if (tid == 0) {
-    SegVal agg = seg_identity<RAW>();
+    const uint64_t base = (uint64_t)tile * kDecTile + (uint64_t)tid * kDecItems;
+    unsigned long long e[kDecItems];
+    uint32_t idx[kDecItems], u[kDecItems], r[kDecItems], lheadbits, sstart, seg_first;
+    int32_t lv[kDecItems];
+    SegVal run;
+    PardSegConst K;
+    bool one_seg;
+    tile_first_half<RAW>(T, base, e, idx, u, r, lv, lheadbits, run, K, sstart, seg_first, one_seg);
+    const SegVal inc = warp_scan<RAW>(run, lane);
+    if (lane == 31) { s_wm[warp] = inc.m; s_wh[warp] = inc.head; }
+    __syncthreads();
+    if (tid == 0) {
+      SegVal agg = seg_identity<RAW>();
 #pragma unroll
-    for (int w = 0; w < WARPS; ++w) {
-      SegVal a; a.m = s_wm[w]; a.head = s_wh[w];
-      agg = seg_combine<RAW>(agg, a);
+      for (int w = 0; w < WARPS; ++w) {
+        SegVal a; a.m = s_wm[w]; a.head = s_wh[w];
+        agg = seg_combine<RAW>(agg, a);
+      }
+      tile_agg[tile] = pack_val(agg, 0);
     }
-    tile_agg[tile] = pack_val(agg, 0);
+    __syncthreads();
   }
-  __syncthreads();
-  }
-  /* the block that finishes last turns the aggregates into the value carried into every tile */
-  if (last_block_done(&const_cast<PlanHeader*>(hdr)->agg_done)) tile_scan_block<RAW, kDecThreads>(tile_agg, n_tiles, carry);
 }
 
 /* Kept requests per queue -> first output slot of every queue, the number of
@@ -1139,11 +1134,12 @@ __device__ void kept_scan_block(const uint32_t* seg_kept, uint32_t n_seg, uint32
     const uint32_t i0 = base + threadIdx.x * PER;
     uint32_t v[PER], c[PER], x = 0, y = 0;
     if (vec_in && i0 + PER <= n_seg) {
-      const uint4 a = *reinterpret_cast<const uint4*>(seg_kept + i0), b = *reinterpret_cast<const uint4*>(seg_kept + i0 + 4);
+      /* (L2 loads here and in kept_move_jobs: inside k_scan_path other blocks of the same kernel wrote these) */
+      const uint4 a = __ldcg(reinterpret_cast<const uint4*>(seg_kept + i0)), b = __ldcg(reinterpret_cast<const uint4*>(seg_kept + i0 + 4));
       v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
     } else {
 #pragma unroll
-      for (int k = 0; k < PER; ++k) v[k] = i0 + k < n_seg ? seg_kept[i0 + k] : 0;
+      for (int k = 0; k < PER; ++k) v[k] = i0 + k < n_seg ? __ldcg(&seg_kept[i0 + k]) : 0;
     }
     if (vec_user && i0 + PER <= n_seg) {
       *reinterpret_cast<uint4*>(out_seg_kept + i0) = make_uint4(v[0], v[1], v[2], v[3]);
@@ -1210,25 +1206,22 @@ __device__ void kept_scan_block(const uint32_t* seg_kept, uint32_t n_seg, uint32
  * a kept request's index goes to kept_tmp[first position of its queue + k_r]:
  * every queue's survivors end up contiguous, k_kept_move packs the queues. */
 template <bool RAW>
-__global__ void __launch_bounds__(kDecThreads, 3)
-k_decide(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
+__device__ void decide_tiles(const PlanHeader* __restrict__ hdr, const unsigned long long* __restrict__ buf_a,
          const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits,
          const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
          const uint32_t* __restrict__ win_off, const int32_t* __restrict__ carry,
          uint8_t* __restrict__ out_keep, long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
          uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept) {
-  pdl_wait();
   constexpr int WARPS = kDecThreads / 32;
   __shared__ int32_t s_wm[WARPS];
   __shared__ uint32_t s_wh[WARPS];
-  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
   const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
   for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
   const uint64_t base = (uint64_t)tile * kDecTile + (uint64_t)tid * kDecItems;
   const bool full = base + kDecItems <= n;
-  const int32_t tile_carry = carry[tile];
+  const int32_t tile_carry = __ldcg(&carry[tile]);       /* written by another block of this kernel */
 
   unsigned long long e[kDecItems];
   uint32_t idx[kDecItems], u[kDecItems], r[kDecItems], lheadbits, sstart, seg_first;
@@ -1733,9 +1726,11 @@ __global__ void __launch_bounds__(1024)
 k_win_from_counts(PlanHeader* hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
                   const uint32_t* __restrict__ whist, const uint32_t* __restrict__ win_off,
                   const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab,
-                  uint32_t* __restrict__ seg_off, uint32_t* __restrict__ out_seg_off) {
+                  uint32_t* __restrict__ seg_off, uint32_t* __restrict__ out_seg_off, uint32_t raw,
+                  uint32_t* __restrict__ seg_kept, uint32_t* __restrict__ out_seg_kept,
+                  uint32_t* __restrict__ kept_base, unsigned long long* __restrict__ out_n_kept) {
   pdl_wait();
-  __shared__ uint32_t s_len[kHistSegs];
+  __shared__ uint32_t s_len[kHistSegs], s_kept[kHistSegs];
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (uint32_t q = warp; q < n_seg; q += blockDim.x / 32) {
     const uint32_t off = win_off[q], cnt = win_cnt[q];
@@ -1755,17 +1750,34 @@ k_win_from_counts(PlanHeader* hdr, uint32_t n_seg, const PardSegConst* __restric
     __syncwarp();
     /* P as the decision reads it: entry b = requests in windows below b, i.e. the sum up to entry b */
     win_prefix_warp(q, ktab, win_off, win_cnt, wtab, lane);
+    /* With the tables complete the queue's number of kept requests is known before any request
+     * has been decided: the last entry closes the queue (P = its length), its Kp counts the kept
+     * requests under raw positions, and its E is the minimum of u_t - t over the whole queue, so
+     * that the admitted count after the last request is n - 1 + min(E, 1). */
+    if (lane == 0) {
+      __threadfence_block();
+      const WinEntry last = wtab[off + cnt - 1];
+      s_kept[q] = run == 0 ? 0u : (raw ? last.Kp : (uint32_t)((int32_t)run - 1 + min(last.E, 1)));
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    uint32_t first = 0;
+    const bool scan = hdr->use_scan != 0;                /* then the scan path counts and packs */
+    uint32_t first = 0, kept = 0;
     for (uint32_t q = 0; q < n_seg; ++q) {
       seg_off[q] = first;
       if (out_seg_off) out_seg_off[q] = first;
       first += s_len[q];
+      if (!scan) {
+        kept_base[q] = kept;
+        seg_kept[q] = s_kept[q];
+        if (out_seg_kept) out_seg_kept[q] = s_kept[q];
+        kept += s_kept[q];
+      }
     }
     seg_off[n_seg] = first;
     if (out_seg_off) out_seg_off[n_seg] = first;
+    if (!scan && out_n_kept) *out_n_kept = kept;
   }
 }
 
@@ -1779,8 +1791,12 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
              const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
              const WinEntry* __restrict__ wtab,
              uint8_t* __restrict__ out_keep, long long* __restrict__ out_est,
-             uint32_t* __restrict__ out_perm, uint32_t* __restrict__ kept_tmp,
+             uint32_t* __restrict__ out_perm, uint32_t* __restrict__ kept_dst, const uint32_t* __restrict__ kept_off,
              uint32_t* __restrict__ seg_kept) {
+  /* kept_dst / kept_off: where the survivors of a queue go.  Normally the queue's own range of a
+   * scratch array (kept_off = the queues' first positions), packed afterwards; with counted
+   * tables the queues' kept counts are known beforehand and the survivors go straight to their
+   * final place (kept_dst = the output, kept_off = the queues' output offsets, seg_kept = NULL). */
   pdl_wait();
   if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const TileCtx T = make_tile_ctx(hdr, buf_a, buf_b, n, ibits, ktab, seg_off);
@@ -1798,6 +1814,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
   uint32_t cur_seg = (uint32_t)(e[0] >> T.kshift);
   PardSegConst K = ktab[cur_seg];
   uint32_t sstart = seg_off[cur_seg], send = seg_off[cur_seg + 1], woff = win_off[cur_seg], wcnt = win_cnt[cur_seg];
+  uint32_t koff = kept_dst ? kept_off[cur_seg] : 0u;
   const bool narrow = T.narrow && (K.narrow & (kSegNarrow | kSegNoStage)) == kSegNarrow && full &&
                       cur_seg == (uint32_t)(e[kDecItems - 1] >> T.kshift);
 
@@ -1820,6 +1837,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
           cur_seg = sg;
           K = ktab[sg];
           sstart = seg_off[sg];
+          koff = kept_dst ? kept_off[sg] : 0u;
           send = seg_off[sg + 1];
           woff = win_off[sg];
           wcnt = win_cnt[sg];
@@ -1840,7 +1858,7 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
         if (b64 >= (unsigned long long)wcnt) {
           set_status(T.hdr, PARD_EDATA);
           est[i] = K.A;
-          if ((uint32_t)j + 1 == send) seg_kept[cur_seg] = 0;
+          if (seg_kept && (uint32_t)j + 1 == send) seg_kept[cur_seg] = 0;
           continue;
         }
         const uint32_t b = (uint32_t)b64;
@@ -1863,8 +1881,8 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
       kept = c < u ? 1u : 0u;
       const uint32_t round = K.cap_magic ? div_magic32(c, K.cap_magic) : c;
       est[i] = K.A + (long long)((unsigned long long)round * (unsigned long long)K.d);
-      if (kept && kept_tmp) kept_tmp[sstart + ahead] = idx[i];
-      if ((uint32_t)j + 1 == send) seg_kept[cur_seg] = ahead + kept;   /* the last request knows the queue's count */
+      if (kept && kept_dst) kept_dst[koff + ahead] = idx[i];
+      if (seg_kept && (uint32_t)j + 1 == send) seg_kept[cur_seg] = ahead + kept;   /* the last request knows the queue's count */
     }
     keepbits |= kept << i;
   }
@@ -1895,34 +1913,93 @@ k_decide_win(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
 
 /* Packs the queues' survivors: copy job j moves up to kCompactChunk indices of one queue; a
  * warp per job. */
+__device__ __forceinline__ void kept_move_jobs(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ seg_off,
+                                               const uint32_t* __restrict__ seg_kept, const uint32_t* __restrict__ kept_base,
+                                               const uint32_t* __restrict__ chunk_base, uint32_t n_seg,
+                                               uint32_t* __restrict__ out_kept_idx) {
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t jobs = __ldcg(&chunk_base[n_seg]), step = (gridDim.x * blockDim.x) >> 5;
+  for (uint32_t job = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; job < jobs; job += step) {
+    uint32_t lo = 0, hi = n_seg;                 /* last queue whose first job is <= job */
+    while (hi - lo > 1) {
+      const uint32_t mid = lo + (hi - lo) / 2;
+      if (__ldcg(&chunk_base[mid]) <= job) lo = mid; else hi = mid;
+    }
+    const uint32_t s = lo;
+    const uint32_t first = (job - __ldcg(&chunk_base[s])) * kCompactChunk;
+    const uint32_t count = min((uint32_t)kCompactChunk, __ldcg(&seg_kept[s]) - first);
+    const uint32_t* src = kept_tmp + seg_off[s] + first;
+    uint32_t* dst = out_kept_idx + __ldcg(&kept_base[s]) + first;
+    uint32_t i = lane;
+    for (; i + 224 < count; i += 256) {            /* eight loads in flight per lane */
+      uint32_t v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldcg(&src[i + 32 * k]);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) dst[i + 32 * k] = v[k];
+    }
+    for (; i < count; i += 32) dst[i] = __ldcg(&src[i]);
+  }
+}
+
 __global__ void __launch_bounds__(256)
 k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ seg_off,
             const uint32_t* __restrict__ seg_kept, const uint32_t* __restrict__ kept_base,
             const uint32_t* __restrict__ chunk_base, uint32_t n_seg, uint32_t* __restrict__ out_kept_idx) {
   pdl_wait();
-  const uint32_t lane = threadIdx.x & 31;
-  const uint32_t jobs = chunk_base[n_seg], step = (gridDim.x * blockDim.x) >> 5;
-  for (uint32_t job = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; job < jobs; job += step) {
-    uint32_t lo = 0, hi = n_seg;                 /* last queue whose first job is <= job */
-    while (hi - lo > 1) {
-      const uint32_t mid = lo + (hi - lo) / 2;
-      if (chunk_base[mid] <= job) lo = mid; else hi = mid;
+  kept_move_jobs(kept_tmp, seg_off, seg_kept, kept_base, chunk_base, n_seg, out_kept_idx);
+}
+
+/* The decision by scanning, from the sorted elements to the packed survivors, as ONE kernel: the
+ * fallback for calls whose queues have too many batch windows for the tables (and what
+ * PARD_MODE_SCAN asks for).  Launched on every call; returns at once when the tables did the
+ * work.  Its five steps -- tile aggregates, their scan (block 0), the decision, the queues' kept
+ * counts into output offsets (block 0), the packing of the survivors -- need the whole grid to
+ * have finished the step before: the grid is small enough to be resident as a whole (at most three
+ * blocks of 128 threads per multiprocessor), and its blocks meet at counters in the workspace
+ * header, each wait bounded like the sort's (PARD_ETIMEOUT, every block gives up, nothing hangs). */
+__device__ bool grid_barrier(PlanHeader* hdr, int k) {
+  __shared__ uint32_t s_ok;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(&hdr->bar[k], 1u);
+    uint32_t spins = 0;
+    bool ok = true;
+    while (ld_relaxed(&hdr->bar[k]) < gridDim.x) {
+      if (++spins > kSpinLimit || hdr->aborted) { ok = false; break; }
+      __nanosleep(200);
     }
-    const uint32_t s = lo;
-    const uint32_t first = (job - chunk_base[s]) * kCompactChunk;
-    const uint32_t count = min((uint32_t)kCompactChunk, seg_kept[s] - first);
-    const uint32_t* src = kept_tmp + seg_off[s] + first;
-    uint32_t* dst = out_kept_idx + kept_base[s] + first;
-    uint32_t i = lane;
-    for (; i + 224 < count; i += 256) {            /* eight loads in flight per lane */
-      uint32_t v[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = src[i + 32 * k];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) dst[i + 32 * k] = v[k];
-    }
-    for (; i < count; i += 32) dst[i] = src[i];
+    if (!ok) set_aborted(hdr);
+    __threadfence();
+    s_ok = ok ? 1u : 0u;
   }
+  __syncthreads();
+  return s_ok != 0;
+}
+
+template <bool RAW>
+__global__ void __launch_bounds__(kDecThreads, 3)
+k_scan_path(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
+            const unsigned long long* __restrict__ buf_b, uint32_t n, uint32_t ibits, uint32_t n_seg,
+            const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
+            const uint32_t* __restrict__ win_off, unsigned long long* __restrict__ tile_agg, int32_t* __restrict__ carry,
+            uint8_t* __restrict__ out_keep, long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
+            uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept, uint32_t* __restrict__ kept_base,
+            uint32_t* __restrict__ chunk_base, uint32_t* __restrict__ out_seg_kept,
+            unsigned long long* __restrict__ out_n_kept, uint32_t* __restrict__ out_kept_idx) {
+  pdl_wait();
+  if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
+  const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
+  tile_agg_tiles<RAW>(hdr, buf_a, buf_b, n, ibits, ktab, seg_off, tile_agg);
+  if (!grid_barrier(hdr, 0)) return;
+  if (blockIdx.x == 0) tile_scan_block<RAW, kDecThreads>(tile_agg, n_tiles, carry);
+  if (!grid_barrier(hdr, 1)) return;
+  decide_tiles<RAW>(hdr, buf_a, buf_b, n, ibits, ktab, seg_off, win_off, carry, out_keep, out_est, out_perm, kept_tmp, seg_kept);
+  if (!grid_barrier(hdr, 2)) return;
+  if (blockIdx.x == 0) kept_scan_block<kDecThreads>(seg_kept, n_seg, kept_base, chunk_base, out_seg_kept, out_n_kept);
+  if (!grid_barrier(hdr, 3)) return;
+  if (out_kept_idx) kept_move_jobs(kept_tmp, seg_off, seg_kept, kept_base, chunk_base, n_seg, out_kept_idx);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -2836,7 +2913,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
                (const uint32_t*)win_cnt, whist);
     if (win_hist)
       launch_pdl(k_win_from_counts, 1, 1024, 0, stream, hdr, L.n_seg, (const PardSegConst*)ktab, (const uint32_t*)whist,
-                 (const uint32_t*)win_off, (const uint32_t*)win_cnt, wtab, seg_off, out->d_seg_offsets);
+                 (const uint32_t*)win_off, (const uint32_t*)win_cnt, wtab, seg_off, out->d_seg_offsets,
+                 (mode & PARD_MODE_RAW) ? 1u : 0u, seg_kept, out->d_seg_kept, kept_base, (unsigned long long*)out->d_n_kept);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
@@ -2883,31 +2961,27 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
                           : (state->d_priority ? k_decide_win<false, true> : k_decide_win<false, false>);
+    /* counted tables: the queues' kept counts are known, the survivors go straight to the output */
     launch_pdl(decide_win, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, win_cnt, wtab,
-               out->d_keep, est, out->d_perm, tmp, seg_kept);
-    /* fallback when a queue has too many batch windows: the same decision by scanning (these two
-     * return at once otherwise) */
+               out->d_keep, est, out->d_perm, win_hist ? out->d_kept_idx : tmp,
+               win_hist ? (const uint32_t*)kept_base : (const uint32_t*)seg_off, win_hist ? (uint32_t*)nullptr : seg_kept);
+    /* fallback when a queue has too many batch windows: the same decision by scanning, one kernel
+     * that returns at once otherwise */
     const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3);
-    if (raw) {
-      launch_pdl(k_tile_agg<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg,
-                 tile_carry);
-      launch_pdl(k_decide<true>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
-                 tile_carry, out->d_keep, est, out->d_perm, tmp, seg_kept);
-    } else {
-      launch_pdl(k_tile_agg<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, tile_agg,
-                 tile_carry);
-      launch_pdl(k_decide<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off,
-                 tile_carry, out->d_keep, est, out->d_perm, tmp, seg_kept);
-    }
+    launch_pdl(raw ? k_scan_path<true> : k_scan_path<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits,
+               L.n_seg, ktab, seg_off, win_off, tile_agg, tile_carry, out->d_keep, est, out->d_perm, tmp, seg_kept, kept_base,
+               chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept, out->d_kept_idx);
   }
   if (n == 0) mark();
   mark();
-  launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
-             (unsigned long long*)out->d_n_kept);
-  if (n > 0 && out->d_kept_idx)
-    launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
-                                               (uint32_t)sms * 8), 256, 0, stream, 
-        kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
+  if (!win_hist) {                                 /* with counted tables this was known before the sort */
+    launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+               (unsigned long long*)out->d_n_kept);
+    if (n > 0 && out->d_kept_idx)
+      launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
+                                                 (uint32_t)sms * 8), 256, 0, stream,
+          kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
+  }
   mark();
   PARD_CUDA_OK(cudaGetLastError());
   if (mode & PARD_MODE_NOWAIT) return PARD_OK;
@@ -2931,20 +3005,21 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   if (!launches) return PARD_EINVAL;
   int rc = pard_plan_workspace_bytes(n, n_ctx, stage_stride, &bytes);
   if (rc != PARD_OK) return rc;
-  /* For the planner's own rule without priorities.  Always: clear, seg_const, kept_scan, and the
-   * queue boundaries (seg_win; with few queues they come with the counted window tables instead).
-   * With many queues also key_width (and, when n > 0, ctx_span).  When n > 0: prepass, pack, the
-   * radix passes, the window tables (win_bounds and win_prefix, or win_from_counts for few
-   * queues), decide_win, the two scan kernels that return at once, and kept_move. */
+  /* For the planner's own rule without priorities and without PARD_MODE_GROUPED.  One ctx of at
+   * most a sort tile: one kernel.  Else always clear and seg_const; with many queues also
+   * key_width (and, when n > 0, ctx_span); when n > 0: prepass, pack, the radix passes, decide_win
+   * and the scan path (one kernel that returns at once); with at most 64 queues the counted window
+   * tables (win_from_counts), else the queue boundaries and searched tables (seg_win, win_bounds,
+   * win_prefix) and the packing of the survivors (kept_scan, kept_move). */
   const uint64_t n_seg = (uint64_t)n_ctx * (uint64_t)stage_stride;
   const uint32_t width_kernels = n_seg <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
-  const bool local_cand = local_sort_candidate(n, n_ctx), local_sure = local_cand && n_ctx == 1;
-  const uint32_t local_kernels = local_sure ? 1 : local_cand ? 2 : 0;       /* sort_local (, ctx_ranges) */
-  const uint32_t passes = local_sure ? 0 : make_layout(n, n_ctx, stage_stride).max_passes;
-  const uint32_t pack = local_sure ? 0 : 1;
+  const bool local_cand = local_sort_candidate(n, n_ctx);
+  const uint32_t local_kernels = local_cand ? 2 : 0;            /* ctx_ranges, sort_local */
+  const uint32_t passes = make_layout(n, n_ctx, stage_stride).max_passes;
   const bool counted = n > 0 && n_seg <= kHistSegs && !local_cand;
-  const uint32_t tables = counted ? 1 : 3;                     /* win_from_counts | seg_win, win_bounds, win_prefix */
-  *launches = n > 0 ? 3 + 2 * width_kernels + 1 + pack + local_kernels + passes + tables + 4 : 4 + width_kernels;
+  if (n_ctx == 1 && n > 0 && n <= (uint64_t)kSortTile) *launches = 1;
+  else if (n == 0) *launches = 4 + width_kernels;               /* clear, (key_width,) seg_const, seg_win, kept_scan */
+  else *launches = 2 + 2 * width_kernels + 2 + local_kernels + passes + 2 + (counted ? 1 : 5);
   return PARD_OK;
 }
 

@@ -51,7 +51,8 @@ struct PlanHeader {
   uint32_t unsorted;          /* 1: some request's ctx is smaller than its predecessor's */
   uint32_t ctx_too_big;       /* 1: some ctx holds more requests than one sort tile */
   uint32_t bad_input;         /* 1: PARD_EDATA was found (kept apart from `status`, which holds the first error only) */
-  uint32_t pad[64 - 17 - (kMaxPasses + 1)];
+  uint32_t bar[4];            /* blocks of k_scan_path that have reached each of its grid-wide barriers */
+  uint32_t pad[64 - 21 - (kMaxPasses + 1)];
 };
 static_assert(sizeof(PlanHeader) == 256, "header is 256 bytes");
 

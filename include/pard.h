@@ -172,13 +172,14 @@ typedef struct pard_plan_out {
                                    of batch windows)                                  */
 #define PARD_MODE_TEST_STALL 8u /* testing aid for the bounded device-side waits: the
                                    first tile of the first sort pass withholds the word
-                                   later tiles wait for, so their waits run out (after
-                                   about a third of a second) and the call returns
+                                   later tiles wait for, and the first block of the scan
+                                   path (PARD_MODE_SCAN) never arrives at the first of its
+                                   grid-wide meeting points; the waits run out (after a
+                                   fraction of a second) and the call returns
                                    PARD_ETIMEOUT with unspecified outputs; the CUDA
                                    context stays usable.  Calls that the library sorts
                                    block by block (requests grouped by ctx, no ctx above
-                                   8,192 requests) have no such wait and are unaffected */
-
+                                   8,192 requests) have no wait in the sort */
 #define PARD_MODE_GROUPED 256u  /* the caller's word that d_requests is grouped by ascending
                                    ctx and that no ctx holds more than 8,192 requests
                                    (batched decision epochs, many small instances).  For

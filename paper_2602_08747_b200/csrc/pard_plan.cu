@@ -1958,12 +1958,12 @@ k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ 
  * have finished the step before: the grid is small enough to be resident as a whole (at most three
  * blocks of 128 threads per multiprocessor), and its blocks meet at counters in the workspace
  * header, each wait bounded like the sort's (PARD_ETIMEOUT, every block gives up, nothing hangs). */
-__device__ bool grid_barrier(PlanHeader* hdr, int k) {
+__device__ bool grid_barrier(PlanHeader* hdr, int k, bool withhold = false) {
   __shared__ uint32_t s_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
-    atomicAdd(&hdr->bar[k], 1u);
+    if (!withhold) atomicAdd(&hdr->bar[k], 1u);      /* (testing aid: a block that never arrives) */
     uint32_t spins = 0;
     bool ok = true;
     while (ld_relaxed(&hdr->bar[k]) < gridDim.x) {
@@ -1987,12 +1987,12 @@ k_scan_path(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
             uint8_t* __restrict__ out_keep, long long* __restrict__ out_est, uint32_t* __restrict__ out_perm,
             uint32_t* __restrict__ kept_tmp, uint32_t* __restrict__ seg_kept, uint32_t* __restrict__ kept_base,
             uint32_t* __restrict__ chunk_base, uint32_t* __restrict__ out_seg_kept,
-            unsigned long long* __restrict__ out_n_kept, uint32_t* __restrict__ out_kept_idx) {
+            unsigned long long* __restrict__ out_n_kept, uint32_t* __restrict__ out_kept_idx, uint32_t stall) {
   pdl_wait();
   if (hdr->wide || hdr->aborted || !hdr->use_scan) return;
   const uint32_t n_tiles = (n + kDecTile - 1) / kDecTile;
   tile_agg_tiles<RAW>(hdr, buf_a, buf_b, n, ibits, ktab, seg_off, tile_agg);
-  if (!grid_barrier(hdr, 0)) return;
+  if (!grid_barrier(hdr, 0, stall && blockIdx.x == 0)) return;
   if (blockIdx.x == 0) tile_scan_block<RAW, kDecThreads>(tile_agg, n_tiles, carry);
   if (!grid_barrier(hdr, 1)) return;
   decide_tiles<RAW>(hdr, buf_a, buf_b, n, ibits, ktab, seg_off, win_off, carry, out_keep, out_est, out_perm, kept_tmp, seg_kept);
@@ -2970,7 +2970,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3);
     launch_pdl(raw ? k_scan_path<true> : k_scan_path<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits,
                L.n_seg, ktab, seg_off, win_off, tile_agg, tile_carry, out->d_keep, est, out->d_perm, tmp, seg_kept, kept_base,
-               chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept, out->d_kept_idx);
+               chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept, out->d_kept_idx,
+               (mode & PARD_MODE_TEST_STALL) ? 1u : 0u);
   }
   if (n == 0) mark();
   mark();

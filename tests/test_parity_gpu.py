@@ -182,6 +182,16 @@ def test_bounded_wait_runs_out_and_is_reported():
     both(wl)
 
 
+def test_bounded_grid_barrier_runs_out_and_is_reported():
+    """The scan path's blocks meet at counters; a block that never arrives (stall aid) makes every
+    other block's bounded wait run out: PARD_ETIMEOUT, nothing hangs, the next call is correct.
+    The call is sorted block by block, so the sort itself has no wait to run out first."""
+    wl, _ = _grouped(n_epochs=40, seed=7)
+    rc, _ = run_library(wl, mode=pb.PARD_MODE_SCAN | pb.PARD_MODE_TEST_STALL, check=False)
+    assert rc == pb.PARD_ETIMEOUT
+    both(wl)
+
+
 def test_key_wider_than_64_bits_is_sorted_in_chunks():
     """Segment, deadline and index bits beyond one 64-bit sort element: the key is sorted in
     chunks and the queues are walked; same plan as the oracle's."""

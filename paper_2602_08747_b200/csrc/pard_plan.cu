@@ -406,7 +406,7 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
   __shared__ uint32_t s_win[WIN ? kWinWords : 1];
   __shared__ long long s_A[WIN ? kHistSegs : 1], s_d[WIN ? kHistSegs : 1];
   __shared__ unsigned long long s_magic[WIN ? kHistSegs : 1];
-  __shared__ uint2 s_wext[WIN ? kHistSegs : 1];            /* first entry and number of entries of the queue's table */
+  __shared__ uint4 s_wcon[WIN ? kHistSegs : 1];            /* per queue: A_rel, first table entry, entries, A_rel and d fit 32 bits */
   if (hdr->wide || sort_is_local(hdr, local_candidate)) return;   /* sorted block by block: k_sort_local read the requests itself */
   const uint32_t npass = hdr->npass, dbits = hdr->dbits;
   for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
@@ -415,63 +415,114 @@ k_pack(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t S,
    * usual case when most of a queue is expired, or lies in few windows -- then hit different words. */
   uint32_t win_total = 0, copies = 1, my_copy = 0;
   bool win_shared = false;                                  /* tables beyond kWinWords entries are counted in global memory */
+  bool win_derive = false;
   if (WIN) {
     win_total = (uint32_t)hdr->win_total;
     win_shared = win_total <= kWinWords;
     while (copies < 32 && 2 * copies * win_total <= kWinWords) copies *= 2;
     my_copy = (threadIdx.x & (copies - 1)) * win_total;
     if (win_shared) for (uint32_t i = threadIdx.x; i < win_total * copies; i += blockDim.x) s_win[i] = 0;
+    /* When the queue id lies inside the last pass's digit the queues' lengths can be read off that
+     * pass's digit counts (see k_seg_win), and entry 0 of a queue -- its requests with deadline < A,
+     * often most of an overloaded queue -- is its length minus its other entries: such requests
+     * are then not counted here at all. */
+    win_derive = npass > 0 && hdr->keybits - dbits <= hdr->keybits - 8 * (npass - 1);
     for (uint32_t q = threadIdx.x; q < n_ctx * S; q += blockDim.x) {
       const PardSegConst K = ktab[q];
-      s_A[q] = K.A; s_d[q] = K.d; s_magic[q] = K.d_magic; s_wext[q] = make_uint2(win_off[q], win_cnt[q]);
+      s_A[q] = K.A; s_d[q] = K.d; s_magic[q] = K.d_magic;
+      s_wcon[q] = make_uint4((uint32_t)(int32_t)K.A_rel, win_off[q], win_cnt[q], (K.narrow & (kSegNarrow | kSegNoStage)) == kSegNarrow ? 1u : 0u);
     }
   }
   __syncthreads();
   const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
-  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  /* n < 2^30: positions and strides in 32 bits (the grid has at most n threads) */
+  const uint32_t stride = gridDim.x * blockDim.x;
+  const bool key32 = hdr->keybits <= 32;       /* the key fits one word: its digits are peeled off that word */
+  const bool off32 = dbits <= 29;              /* deadline offsets fit signed 32-bit arithmetic */
+  uint32_t cur_ctx = 0xffffffffu;              /* the ctx whose deadline range is at hand (requests of a ctx mostly sit together) */
+  unsigned long long cmin = 0, cmax = 0;
   constexpr int kUn = 4;                       /* requests in flight per thread (measured against 1: 74 vs 78.5 us at 2^24) */
-  for (uint64_t j0 = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j0 < n; j0 += stride * kUn) {
+  for (uint32_t j0 = blockIdx.x * blockDim.x + threadIdx.x; j0 < n; j0 += stride * kUn) {
     uint4 rr[kUn];
 #pragma unroll
     for (int u = 0; u < kUn; ++u) {
-      const uint64_t j = j0 + (uint64_t)u * stride;
+      const uint32_t j = j0 + (uint32_t)u * stride;
       if (j < n) rr[u] = __ldg(&req[j]);
     }
 #pragma unroll
     for (int u = 0; u < kUn; ++u) {
-      const uint64_t j = j0 + (uint64_t)u * stride;
+      const uint32_t j = j0 + (uint32_t)u * stride;
       if (j >= n) break;
       const uint4 r = rr[u];
-      unsigned long long D = ((unsigned long long)r.y << 32) | r.x;
-      uint32_t ctx = r.z, stage = r.w & 0xffffu;
-      unsigned long long e;
-      if (ctx < n_ctx && stage < S) {
-        /* ascending offsets give the queue's decision order: deadlines counted up from the ctx's
-         * smallest, or down from its largest when the queue is served high budget first */
-        const uint32_t seg = ctx * S + stage;
-        const bool high_first = priority && __ldg(&priority[seg]) != 0;
-        unsigned long long off = (high_first ? ctx_dmax[ctx] - D : D - ~ctx_dmin_inv[ctx]) & dmask;
-        e = ((((unsigned long long)seg << dbits) | off) << ibits) | j;
-        if (WIN) {
-          const uint2 ext = s_wext[seg];
+      const uint32_t ctx = r.z, stage = r.w & 0xffffu;
+      const bool ok = ctx < n_ctx && stage < S;
+      const uint32_t seg = ok ? ctx * S + stage : 0u;
+      if (ok && ctx != cur_ctx) {
+        cur_ctx = ctx;
+        cmin = ~ctx_dmin_inv[ctx];
+        cmax = ctx_dmax[ctx];
+      }
+      /* ascending offsets give the queue's decision order: deadlines counted up from the ctx's
+       * smallest, or down from its largest when the queue is served high budget first */
+      const bool high_first = ok && priority && __ldg(&priority[seg]) != 0;
+      uint32_t h = 0;                            /* the request's entry in its queue's window table: 0 for deadline < A, else window + 1 */
+      bool count = false;
+      uint4 c = make_uint4(0u, 0u, 1u, 0u);      /* A - ctx's smallest deadline (if it fits 32 bits), first entry, entries, fits? */
+      if (key32 && off32) {
+        /* everything in single words: the offset is below 2^29, so the low words of the 64-bit
+         * difference are the difference */
+        const uint32_t off = ok ? ((high_first ? (uint32_t)cmax - r.x : r.x - (uint32_t)cmin) & (uint32_t)dmask) : 0u;
+        uint32_t key = (seg << dbits) | off;
+        if (WIN && ok) {
+          c = s_wcon[seg];
+          count = true;
+          if (c.w) {
+            const int32_t X = (int32_t)off - (int32_t)c.x;
+            if (X >= 0) {
+              const uint32_t b = div_magic32((uint32_t)X, s_magic[seg]);
+              h = b + 1 < c.z ? b + 1 : c.z - 1;   /* never beyond the queue's entries (a queue decided by scanning has one) */
+            }
+          } else {
+            const long long X = (long long)(((unsigned long long)r.y << 32) | r.x) - s_A[seg];
+            if (X >= 0) {
+              const unsigned long long M = s_magic[seg];
+              const unsigned long long b = (((unsigned long long)X >> 32) == 0 && M) ? div_magic32((uint32_t)X, M)
+                                                                                    : (unsigned long long)X / (unsigned long long)s_d[seg];
+              h = b + 1 < c.z ? (uint32_t)b + 1 : c.z - 1;
+            }
+          }
+        }
+        *reinterpret_cast<uint2*>(dst + j) = make_uint2((key << ibits) | j, __funnelshift_l(key, 0u, ibits));
+        uint32_t* hp = s_hist;
+        for (uint32_t p = 0; p < npass; ++p, hp += kBins, key >>= 8) atomicAdd(hp + (key & 255u), 1u);
+      } else {
+        const unsigned long long D = ((unsigned long long)r.y << 32) | r.x;
+        const unsigned long long off = ok ? ((high_first ? cmax - D : D - cmin) & dmask) : 0ull;
+        unsigned long long key = ((unsigned long long)seg << dbits) | off;
+        if (WIN && ok) {
+          c = s_wcon[seg];
+          count = true;
           const long long X = (long long)D - s_A[seg];
-          uint32_t h = 0;
           if (X >= 0) {
             const unsigned long long M = s_magic[seg];
             const unsigned long long b = (((unsigned long long)X >> 32) == 0 && M) ? div_magic32((uint32_t)X, M)
                                                                                   : (unsigned long long)X / (unsigned long long)s_d[seg];
-            h = b + 1 < ext.y ? (uint32_t)b + 1 : ext.y - 1;   /* never beyond the queue's entries (a queue decided by scanning has one) */
+            h = b + 1 < c.z ? (uint32_t)b + 1 : c.z - 1;
           }
-          if (win_shared) atomicAdd(&s_win[my_copy + ext.x + h], 1u);
-          else atomicAdd(&whist[ext.x + h], 1u);
         }
-      } else {
-        e = j;                                  /* flagged by the prepass; keep indices in range */
-        if (WIN) atomicAdd(win_shared ? &s_win[my_copy] : &whist[0], 1u);   /* it sorts into queue 0: counted there, so that the counts stay the queues' lengths */
+        dst[j] = (key << ibits) | j;
+        uint32_t* hp = s_hist;
+        for (uint32_t p = 0; p < npass; ++p, hp += kBins, key >>= 8) atomicAdd(hp + ((uint32_t)key & 255u), 1u);
       }
-      dst[j] = e;
-      unsigned long long key = e >> ibits;
-      for (uint32_t p = 0; p < npass; ++p) atomicAdd(&s_hist[p * kBins + ((key >> (8 * p)) & 255u)], 1u);
+      if (WIN) {
+        /* a request flagged by the prepass (its element is its index alone) sorts into queue 0 and is
+         * counted there, entry 0: the counts stay the queues' lengths */
+        if (!ok) { c.y = 0; h = 0; count = true; }
+        if (count && (h != 0 || !win_derive)) {
+          if (win_shared) atomicAdd(&s_win[my_copy + c.y + h], 1u);
+          else atomicAdd(&whist[c.y + h], 1u);
+        }
+      }
     }
   }
   __syncthreads();
@@ -1728,16 +1779,36 @@ k_win_from_counts(PlanHeader* hdr, uint32_t n_seg, const PardSegConst* __restric
                   const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab,
                   uint32_t* __restrict__ seg_off, uint32_t* __restrict__ out_seg_off, uint32_t raw,
                   uint32_t* __restrict__ seg_kept, uint32_t* __restrict__ out_seg_kept,
-                  uint32_t* __restrict__ kept_base, unsigned long long* __restrict__ out_n_kept) {
+                  uint32_t* __restrict__ kept_base, unsigned long long* __restrict__ out_n_kept,
+                  const uint32_t* __restrict__ hist, uint32_t sbits) {
   pdl_wait();
   __shared__ uint32_t s_len[kHistSegs], s_kept[kHistSegs];
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  /* entry 0 left uncounted by k_pack (same condition there): the queue's length, from the last
+   * pass's digit counts, minus its other entries */
+  const uint32_t npass = hdr->npass;
+  const uint32_t top_bits = npass ? hdr->keybits - 8 * (npass - 1) : 0;
+  const bool derive = npass > 0 && sbits <= top_bits;
   for (uint32_t q = warp; q < n_seg; q += blockDim.x / 32) {
     const uint32_t off = win_off[q], cnt = win_cnt[q];
+    uint32_t entry0 = 0;
+    if (derive) {
+      const uint32_t* h = hist + (npass - 1) * kBins;
+      const uint32_t d0 = min(q << (top_bits - sbits), (uint32_t)kBins), d1 = min((q + 1) << (top_bits - sbits), (uint32_t)kBins);
+      uint32_t len = 0, others = 0;
+      for (uint32_t d = d0 + lane; d < d1; d += 32) len += h[d];
+      for (uint32_t b = 1 + lane; b < cnt; b += 32) others += whist[off + b];
+      for (int o = 16; o; o >>= 1) {
+        len += __shfl_xor_sync(0xffffffffu, len, o);
+        others += __shfl_xor_sync(0xffffffffu, others, o);
+      }
+      entry0 = len - others;
+    }
     uint32_t run = 0;
     for (uint32_t b0 = 0; b0 < cnt; b0 += 32) {
       const uint32_t b = b0 + lane;
       uint32_t x = b < cnt ? whist[off + b] : 0u;
+      if (derive && b == 0) x = entry0;
       for (int o = 1; o < 32; o <<= 1) {
         const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
         if (lane >= (uint32_t)o) x += y;
@@ -2914,7 +2985,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     if (win_hist)
       launch_pdl(k_win_from_counts, 1, 1024, 0, stream, hdr, L.n_seg, (const PardSegConst*)ktab, (const uint32_t*)whist,
                  (const uint32_t*)win_off, (const uint32_t*)win_cnt, wtab, seg_off, out->d_seg_offsets,
-                 (mode & PARD_MODE_RAW) ? 1u : 0u, seg_kept, out->d_seg_kept, kept_base, (unsigned long long*)out->d_n_kept);
+                 (mode & PARD_MODE_RAW) ? 1u : 0u, seg_kept, out->d_seg_kept, kept_base, (unsigned long long*)out->d_n_kept,
+                 (const uint32_t*)hist, sbits);
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();

@@ -357,27 +357,38 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
       hdr->wide = 1;
       set_status(hdr, PARD_ERANGE);
     }
-    /* Few queues: their batch-window tables are COUNTED while the requests are packed (k_pack)
-     * instead of being searched for in the sorted elements afterwards.  That needs the tables'
-     * extents before any request has been looked at: a queue can have no window beyond that of
-     * its ctx's latest deadline.  Entry 0 of a queue counts its requests with deadline < A, entry
-     * b + 1 those of window b; every queue has at least entry 0, so that the counts also give
-     * the queues' lengths. */
-    if (win_hist) {
-      const uint32_t n_seg = n_ctx * S;
+  }
+  /* Few queues: their batch-window tables are COUNTED while the requests are packed (k_pack)
+   * instead of being searched for in the sorted elements afterwards.  That needs the tables'
+   * extents before any request has been looked at: a queue can have no window beyond that of its
+   * ctx's latest deadline.  Entry 0 of a queue counts its requests with deadline < A, entry b + 1
+   * those of window b; every queue has at least entry 0, so that the counts also give the queues'
+   * lengths. */
+  if (win_hist) {                                        /* still the last block, all its threads */
+    __shared__ uint32_t s_w[kHistSegs];
+    __shared__ uint32_t s_scan;
+    const uint32_t n_seg = n_ctx * S;
+    if (threadIdx.x == 0) s_scan = force_scan;
+    __syncthreads();
+    for (uint32_t q = threadIdx.x; q < n_seg; q += blockDim.x) {   /* every queue's number of entries, side by side */
+      const PardSegConst K = ktab[q];
+      const uint32_t c = q / S;
+      uint32_t w = 1;
+      const unsigned long long lo = ~ctx_dmin_inv[c], hi = ctx_dmax[c];
+      if (!(K.narrow & kSegNoStage) && lo <= hi) {
+        const long long X = (long long)hi - K.A;
+        const unsigned long long nb = X < 0 ? 0ull : (unsigned long long)X / (unsigned long long)K.d + 1;
+        if (nb >= 4096) s_scan = 1;                      /* kWinMaxPerSeg: too many windows for a table */
+        else w = (uint32_t)nb + 1;
+      }
+      s_w[q] = w;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
       uint32_t total = 0;
-      bool scan = force_scan != 0;
+      bool scan = s_scan != 0;
       for (uint32_t q = 0; q < n_seg; ++q) {
-        const PardSegConst K = ktab[q];
-        const uint32_t c = q / S;
-        uint32_t w = 1;
-        const unsigned long long lo = ~ctx_dmin_inv[c], hi = ctx_dmax[c];
-        if (!(K.narrow & kSegNoStage) && lo <= hi) {
-          const long long X = (long long)hi - K.A;
-          const unsigned long long nb = X < 0 ? 0ull : (unsigned long long)X / (unsigned long long)K.d + 1;
-          if (nb >= 4096) scan = true;                 /* kWinMaxPerSeg: too many windows for a table */
-          else w = (uint32_t)nb + 1;
-        }
+        uint32_t w = s_w[q];
         if (total + w > kHistCap) { scan = true; w = 1; }
         win_off[q] = total;
         win_cnt[q] = w;

@@ -57,11 +57,13 @@ def ncu_traffic(kernel):
 
 
 class ClockSampler(threading.Thread):
-    """Polls SM clock and throttle reasons through NVML while the timed region runs."""
+    """Polls SM clock and throttle reasons through NVML.  The thread is started ahead of time (NVML's
+    start-up takes a while); only the samples taken between begin() and result() count."""
 
-    def __init__(self, index, period_s=0.01):
+    def __init__(self, index, period_s=0.002):
         super().__init__(daemon=True)
         self.index, self.period, self.stop_flag = index, period_s, threading.Event()
+        self.ready, self.active = threading.Event(), threading.Event()
         self.sm, self.reasons, self.max_mhz, self.err = [], set(), None, None
 
     def run(self):
@@ -78,17 +80,25 @@ class ClockSampler(threading.Thread):
             }
             get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            self.ready.set()
             while not self.stop_flag.is_set():
-                self.sm.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
-                bits = get(h)
-                for bit, name in names.items():
-                    if bits & bit:
-                        self.reasons.add(name)
+                if self.active.is_set():
+                    self.sm.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                    bits = get(h)
+                    for bit, name in names.items():
+                        if bits & bit:
+                            self.reasons.add(name)
                 time.sleep(self.period)
         except Exception as e:  # NVML missing: report it, do not fail the bench
             self.err = repr(e)
+            self.ready.set()
+
+    def begin(self):
+        self.ready.wait(timeout=20)
+        self.active.set()
 
     def result(self):
+        self.active.clear()
         self.stop_flag.set()
         self.join(timeout=2)
         out = {"sm_mhz": statistics.median(self.sm) if self.sm else None,
@@ -488,7 +498,7 @@ def run_aux(dev, peak, kernels_only=False):
     arr["arrive_us"] = np.maximum(0, wlr.state.now_us[0] - rr.integers(0, 400_000, size=wlr.n))
     arr["slo_us"] = rr.integers(100_000, 400_000, size=wlr.n)
     masked = wlr.requests.copy()
-    masked["flags"] = rr.integers(0, 4, size=wlr.n)            # unknown, first, second, either of the first two paths
+    masked["flags"] = rr.choice(np.array([0, 1, 3], dtype=np.uint16), size=wlr.n)   # path unknown, the first, one of the first two
     for label, mode, a, req in (("known_paths", pb.PARD_MODE_PATH_MASK, None, masked), ("arrival_order", pb.PARD_MODE_FCFS, None, None),
                                 ("nexus", pb.PARD_MODE_NEXUS, None, None), ("clipper_pp", pb.PARD_MODE_CLIPPER, arr, None)):
         w2 = wlr if req is None else inputs.Workload(wlr.name, wlr.pipelines, req, wlr.state, wlr.n_ctx)
@@ -645,17 +655,23 @@ def run_ours(args):
     keep_frac = float(plan.out.n_kept.cpu()[0]) / wl.n
 
     sampler = ClockSampler(physical_gpu_index(local))
-    # warm-up first so that the sampler only sees the timed region
+    sampler.start()
+    # warm-up first so that the sampler only sees work under load
     for _ in range(args.warmup):
         plan.step()
     plan.status()
-    sampler.start()
-    sec, prof = timed_steps(plan, args.steps, 0, dist, profile_every=8)
-    clocks = sampler.result()
-    # the decision pass as one phase, in a run of its own
+    sampler.begin()
+    sec, _ = timed_steps(plan, args.steps, 0, dist)         # the timed region: K steps, nothing else on the stream
+    # per-kernel durations from the library's own phase events, in a second run of the same steps
+    # (an event between two kernels keeps the second from being scheduled while the first drains,
+    # so a run with events is a little slower than the timed one)
+    _, prof = timed_steps(plan, max(args.steps, 16), 0, dist, profile_every=4)
+    # the decision pass as one phase, in a run of its own (same work, same load: the clock samples
+    # run on through it, the timed region alone may last only a few milliseconds)
     from paper_2602_08747_b200 import binding as pb
     _, prof_coarse = timed_steps(plan, max(40, args.steps // 4), 0, dist,
                                  profile_every=4 | pb.PARD_PROFILE_COARSE)
+    clocks = sampler.result()
 
     peak, peak_kind = measured_peaks()
     n_total = wl.n * world

@@ -166,10 +166,14 @@ typedef struct pard_plan_out {
 #define PARD_MODE_NOWAIT   2u   /* pard_plan returns once its work is enqueued and
                                    reads no status back; the status word stays in the
                                    workspace until pard_plan_status fetches it        */
-#define PARD_MODE_SCAN     4u   /* take the decision by the scan kernels even when the
+#define PARD_MODE_SCAN     4u   /* take the decision by the scan path even when the
                                    batch-window tables would do (same results; the scan
                                    is otherwise the fallback for queues with thousands
-                                   of batch windows)                                  */
+                                   of batch windows).  The scan path is one kernel whose
+                                   blocks (two per multiprocessor) wait for each other
+                                   between its steps, each wait bounded at about half a
+                                   second: a GPU that other streams keep completely full
+                                   for that long makes the call return PARD_ETIMEOUT   */
 #define PARD_MODE_TEST_STALL 8u /* testing aid for the bounded device-side waits: the
                                    first tile of the first sort pass withholds the word
                                    later tiles wait for, and the first block of the scan

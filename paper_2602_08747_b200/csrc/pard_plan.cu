@@ -2037,9 +2037,10 @@ k_kept_move(const uint32_t* __restrict__ kept_tmp, const uint32_t* __restrict__ 
  * PARD_MODE_SCAN asks for).  Launched on every call; returns at once when the tables did the
  * work.  Its five steps -- tile aggregates, their scan (block 0), the decision, the queues' kept
  * counts into output offsets (block 0), the packing of the survivors -- need the whole grid to
- * have finished the step before: the grid is small enough to be resident as a whole (at most three
+ * have finished the step before: the grid is small enough to be resident as a whole (at most two
  * blocks of 128 threads per multiprocessor), and its blocks meet at counters in the workspace
- * header, each wait bounded like the sort's (PARD_ETIMEOUT, every block gives up, nothing hangs). */
+ * header, each wait bounded like the sort's (PARD_ETIMEOUT, every block gives up, nothing hangs;
+ * the bound only bites when other streams keep the multiprocessors full for that long). */
 __device__ bool grid_barrier(PlanHeader* hdr, int k, bool withhold = false) {
   __shared__ uint32_t s_ok;
   __syncthreads();
@@ -2048,8 +2049,8 @@ __device__ bool grid_barrier(PlanHeader* hdr, int k, bool withhold = false) {
     if (!withhold) atomicAdd(&hdr->bar[k], 1u);      /* (testing aid: a block that never arrives) */
     uint32_t spins = 0;
     bool ok = true;
-    while (ld_relaxed(&hdr->bar[k]) < gridDim.x) {
-      if (++spins > kSpinLimit || hdr->aborted) { ok = false; break; }
+    while (ld_relaxed(&hdr->bar[k]) < gridDim.x) {     /* up to about half a second: other work may hold multiprocessors for a while */
+      if (++spins > 8 * kSpinLimit || hdr->aborted) { ok = false; break; }
       __nanosleep(200);
     }
     if (!ok) set_aborted(hdr);
@@ -3050,7 +3051,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
                win_hist ? (const uint32_t*)kept_base : (const uint32_t*)seg_off, win_hist ? (uint32_t*)nullptr : seg_kept);
     /* fallback when a queue has too many batch windows: the same decision by scanning, one kernel
      * that returns at once otherwise */
-    const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 3);
+    const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 2);
     launch_pdl(raw ? k_scan_path<true> : k_scan_path<false>, scan_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits,
                L.n_seg, ktab, seg_off, win_off, tile_agg, tile_carry, out->d_keep, est, out->d_perm, tmp, seg_kept, kept_base,
                chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept, out->d_kept_idx,

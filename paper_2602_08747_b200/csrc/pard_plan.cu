@@ -2118,17 +2118,21 @@ struct LocalArgs {
   uint32_t* kept_tmp;
 };
 
+template <int THREADS>
 struct LocalSmem {
-  SortSmem sort;
+  unsigned long long keys[kSortTile];
+  uint32_t slot[THREADS / 32][kBins];      /* counts, then next free slot per (warp, digit) */
+  uint32_t match[THREADS / 32][kBins];     /* lanes currently holding the digit */
+  uint32_t scan[THREADS / 32];
   PardSegConst K[PARD_MAX_STAGES];
   uint32_t stage_cnt[PARD_MAX_STAGES];
   uint32_t stage_first[PARD_MAX_STAGES + 1];
   uint32_t stage_kept[PARD_MAX_STAGES];
   uint32_t kept_base[PARD_MAX_STAGES + 1];
   uint32_t hb_kept[PARD_MAX_STAGES];       /* high budget first: length of the kept prefix */
-  unsigned long long red_min[kSortThreads / 32], red_max[kSortThreads / 32];
-  int32_t wm[kSortThreads / 32];
-  uint32_t wh[kSortThreads / 32];
+  unsigned long long red_min[THREADS / 32], red_max[THREADS / 32];
+  int32_t wm[THREADS / 32];
+  uint32_t wh[THREADS / 32];
   uint32_t flag_foreign, flag_bad;
 };
 
@@ -2138,7 +2142,8 @@ struct LocalElem {
   bool high_first;
 };
 
-__device__ __forceinline__ LocalElem local_decode(unsigned long long e, uint32_t pos, const LocalSmem& Sm,
+template <class SMEM>
+__device__ __forceinline__ LocalElem local_decode(unsigned long long e, uint32_t pos, const SMEM& Sm,
                                                   uint32_t ibits, uint32_t dbits, unsigned long long dmask,
                                                   uint32_t imask) {
   LocalElem x;
@@ -2158,14 +2163,17 @@ __device__ __forceinline__ LocalElem local_decode(unsigned long long e, uint32_t
   return x;
 }
 
-template <bool RAW>
-__global__ void __launch_bounds__(kSortThreads, 2)
+/* THREADS: 512, two blocks per multiprocessor.  (1,024 threads for a call that is this one block --
+ * half as many ranking rounds per warp, twice the warps -- measured the same 28 us at 4,096
+ * requests: the time is the chain of barriers and dependent shared-memory steps, not the warps.) */
+template <bool RAW, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 512 ? 2 : 1)
 k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
   pdl_wait();
-  constexpr int WARPS = kSortThreads / 32;
-  constexpr int kItems = kSortTile / kSortThreads;
+  constexpr int WARPS = THREADS / 32;
+  constexpr int kItems = kSortTile / THREADS;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  LocalSmem& Sm = *reinterpret_cast<LocalSmem*>(smem_raw);
+  LocalSmem<THREADS>& Sm = *reinterpret_cast<LocalSmem<THREADS>*>(smem_raw);
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lanebit = 1u << lane;
   const uint32_t S = (uint32_t)a.st.stage_stride;
@@ -2181,13 +2189,13 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
   const uint32_t first = single ? 0u : a.ctx_start[c];
   const uint32_t cnt = single ? a.n : a.ctx_start[c + 1] - first;
   /* every warp owns `items` rounds of 32 consecutive requests: as few as the ctx needs */
-  const int items = (int)((cnt + kSortThreads - 1) / kSortThreads);
+  const int items = (int)((cnt + THREADS - 1) / THREADS);
   const uint32_t wfirst = warp * (32 * (uint32_t)items);
-  uint16_t* stage16 = reinterpret_cast<uint16_t*>(&Sm.sort.slot[0][0]);     /* 16 KB: the stages until the elements are built */
+  uint16_t* stage16 = reinterpret_cast<uint16_t*>(&Sm.slot[0][0]);     /* 16 KB: the stages until the elements are built */
 
   /* 1. the ctx's requests: deadlines into the tile buffer, stages beside them; deadline range,
    * queue lengths, input checks */
-  for (uint32_t i = tid; i < S; i += kSortThreads) { Sm.stage_cnt[i] = 0; Sm.stage_kept[i] = 0; }
+  for (uint32_t i = tid; i < S; i += THREADS) { Sm.stage_cnt[i] = 0; Sm.stage_kept[i] = 0; }
   if (tid == 0) { Sm.flag_foreign = 0; Sm.flag_bad = 0; }
   __syncthreads();
   unsigned long long lmin = ~0ull, lmax = 0;
@@ -2203,7 +2211,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
       foreign |= r.z != c;
       const bool ok = r.z == c && stage < S && D < (unsigned long long)PARD_TIME_LIMIT_US;
       bad |= !ok;
-      Sm.sort.keys[pos] = D;
+      Sm.keys[pos] = D;
       stage16[pos] = ok ? (uint16_t)stage : (uint16_t)0xffffu;
       if (ok) {
         lmin = D < lmin ? D : lmin;
@@ -2253,7 +2261,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
       if (lane == 0) Sm.K[k] = K;
     }
   } else {
-    for (uint32_t k = tid; k < S; k += kSortThreads) {
+    for (uint32_t k = tid; k < S; k += THREADS) {
       PardSegConst K = a.ktab[(size_t)c * S + k];
       const bool high_first = K.narrow & kSegHighFirst;
       K.A_rel = high_first ? (int64_t)dmax - K.A : K.A - (int64_t)dmin;
@@ -2290,7 +2298,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
     const uint32_t pos = wfirst + i * 32 + lane;
     key[i] = ~0ull;                                      /* padding sorts last */
     if (pos < cnt) {
-      const unsigned long long D = Sm.sort.keys[pos];
+      const unsigned long long D = Sm.keys[pos];
       const uint32_t stage = stage16[pos];
       const uint32_t j = first + pos;
       if (stage != 0xffffu) {
@@ -2305,21 +2313,21 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
   __syncthreads();                                       /* the stages have been read: their room becomes the counters again */
   const uint32_t local_bits = dbits + sb;
   const uint32_t passes = (local_bits + 7) / 8;
-  for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) (&Sm.sort.match[0][0])[i] = 0;
+  for (uint32_t i = tid; i < WARPS * kBins; i += THREADS) (&Sm.match[0][0])[i] = 0;
   for (uint32_t p = 0; p < passes; ++p) {
     const uint32_t shift = a.ibits + 8 * p;
-    for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) (&Sm.sort.slot[0][0])[i] = 0;
+    for (uint32_t i = tid; i < WARPS * kBins; i += THREADS) (&Sm.slot[0][0])[i] = 0;
     __syncthreads();
 #pragma unroll
     for (int i = 0; i < kItems; ++i)
-      if (i < items) atomicAdd(&Sm.sort.slot[warp][(uint32_t)(key[i] >> shift) & 255u], 1u);
+      if (i < items) atomicAdd(&Sm.slot[warp][(uint32_t)(key[i] >> shift) & 255u], 1u);
     __syncthreads();
     uint32_t count = 0, x = 0;
     if (tid < kBins) {
 #pragma unroll
       for (int w = 0; w < WARPS; ++w) {
-        const uint32_t t = Sm.sort.slot[w][tid];
-        Sm.sort.slot[w][tid] = count;
+        const uint32_t t = Sm.slot[w][tid];
+        Sm.slot[w][tid] = count;
         count += t;
       }
       x = count;
@@ -2327,38 +2335,38 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
         const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
         if (lane >= (uint32_t)o) x += y;
       }
-      if (lane == 31) Sm.sort.scan[0][warp] = x;
+      if (lane == 31) Sm.scan[warp] = x;
     }
     __syncthreads();
     if (tid < kBins) {
       uint32_t wx = 0;
 #pragma unroll
       for (int w = 0; w < kBins / 32; ++w)
-        if (w < (int)warp) wx += Sm.sort.scan[0][w];
+        if (w < (int)warp) wx += Sm.scan[w];
       const uint32_t dstart = wx + x - count;
 #pragma unroll
-      for (int w = 0; w < WARPS; ++w) Sm.sort.slot[w][tid] += dstart;
+      for (int w = 0; w < WARPS; ++w) Sm.slot[w][tid] += dstart;
     }
     __syncthreads();
-    sort_rank_drop<kItems, kItems>(key, shift, Sm.sort.slot[warp], Sm.sort.match[warp], Sm.sort.keys, lanebit, items);
+    sort_rank_drop<kItems, kItems>(key, shift, Sm.slot[warp], Sm.match[warp], Sm.keys, lanebit, items);
     __syncthreads();
     if (p + 1 < passes) {
 #pragma unroll
       for (int i = 0; i < kItems; ++i)
-        if (i < items) key[i] = Sm.sort.keys[wfirst + i * 32 + lane];
+        if (i < items) key[i] = Sm.keys[wfirst + i * 32 + lane];
       __syncthreads();
     }
   }
   if (passes == 0) {
 #pragma unroll
     for (int i = 0; i < kItems; ++i)
-      if (i < items) Sm.sort.keys[wfirst + i * 32 + lane] = key[i];
+      if (i < items) Sm.keys[wfirst + i * 32 + lane] = key[i];
     __syncthreads();
   }
 
   /* 4. queue boundaries of the ctx */
   const uint32_t n_good = Sm.stage_first[S];             /* requests that passed the checks; the others follow them */
-  for (uint32_t k = tid; k < S; k += kSortThreads) {
+  for (uint32_t k = tid; k < S; k += THREADS) {
     const uint32_t v = first + Sm.stage_first[k];
     a.seg_off[(size_t)c * S + k] = v;
     if (a.out_seg_off) a.out_seg_off[(size_t)c * S + k] = v;
@@ -2376,7 +2384,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
       if (i >= items) break;
       const uint32_t pos = wfirst + i * 32 + lane;
       if (pos < n_good) {
-        const LocalElem x = local_decode(Sm.sort.keys[pos], pos, Sm, a.ibits, dbits, dmask, imask);
+        const LocalElem x = local_decode(Sm.keys[pos], pos, Sm, a.ibits, dbits, dmask, imask);
         if (x.high_first && x.r >= x.u) atomicMin(&Sm.hb_kept[x.stage], x.r);
       }
     }
@@ -2396,7 +2404,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
       const uint32_t pos = wfirst + (i0 + g) * 32 + lane;
       v[g] = seg_identity<RAW>();
       if (i0 + g < items && pos < n_good) {
-        const LocalElem x = local_decode(Sm.sort.keys[pos], pos, Sm, a.ibits, dbits, dmask, imask);
+        const LocalElem x = local_decode(Sm.keys[pos], pos, Sm, a.ibits, dbits, dmask, imask);
         v[g].head = x.r == 0 ? 1u : 0u;
         v[g].m = RAW ? (x.r < x.u ? 1 : 0) : (int32_t)x.u - (int32_t)x.r;
       }
@@ -2440,7 +2448,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
       v[g] = seg_identity<RAW>();
       x[g].stage = 0; x[g].idx = 0; x[g].r = 0; x[g].u = 0; x[g].high_first = false;
       e[g] = 0;
-      if (i0 + g < items && pos < cnt) e[g] = Sm.sort.keys[pos];
+      if (i0 + g < items && pos < cnt) e[g] = Sm.keys[pos];
       if (i0 + g < items && pos < n_good) {
         x[g] = local_decode(e[g], pos, Sm, a.ibits, dbits, dmask, imask);
         v[g].head = x[g].r == 0 ? 1u : 0u;
@@ -2503,7 +2511,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
     }
   }
   __syncthreads();
-  for (uint32_t k = tid; k < S; k += kSortThreads) {
+  for (uint32_t k = tid; k < S; k += THREADS) {
     a.seg_kept[(size_t)c * S + k] = Sm.stage_kept[k];
     if (single && a.out_seg_kept) a.out_seg_kept[k] = Sm.stage_kept[k];
   }
@@ -2533,7 +2541,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
   if (a.out_kept_idx && a.kept_tmp)
     for (uint32_t k = 0; k < S; ++k) {
       const uint32_t nk = Sm.stage_kept[k], from = Sm.stage_first[k], to = Sm.kept_base[k];
-      for (uint32_t i = tid; i < nk; i += kSortThreads) a.out_kept_idx[to + i] = a.kept_tmp[from + i];
+      for (uint32_t i = tid; i < nk; i += THREADS) a.out_kept_idx[to + i] = a.kept_tmp[from + i];
     }
 }
 
@@ -2699,10 +2707,10 @@ int allow_sort_smem(int dev) {
                                       (int)sizeof(SortSmem)));
     PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_local, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
-    PARD_CUDA_OK(cudaFuncSetAttribute(k_plan_local<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)sizeof(LocalSmem)));
-    PARD_CUDA_OK(cudaFuncSetAttribute(k_plan_local<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)sizeof(LocalSmem)));
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_plan_local<false, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(LocalSmem<512>)));
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_plan_local<true, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(LocalSmem<512>)));
     done[dev].store(true, std::memory_order_release);
   }
   return PARD_OK;
@@ -2942,8 +2950,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
       launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax,
                  ktab, hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
     }
-    launch_pdl((mode & PARD_MODE_RAW) ? k_plan_local<true> : k_plan_local<false>, n_ctx, kSortThreads, sizeof(LocalSmem),
-               stream, hdr, la);
+    launch_pdl((mode & PARD_MODE_RAW) ? k_plan_local<true, 512> : k_plan_local<false, 512>, n_ctx, 512,
+               sizeof(LocalSmem<512>), stream, hdr, la);
     if (fused_grouped) {
       launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
                  (unsigned long long*)out->d_n_kept);

@@ -2379,7 +2379,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
   __syncthreads();
   /* a queue served high budget first keeps a prefix: its length is the first position r with r >= u_r */
   if (a.st.d_priority) {
-#pragma unroll 2
+#pragma unroll 1
     for (int i = 0; i < kItems; ++i) {
       if (i >= items) break;
       const uint32_t pos = wfirst + i * 32 + lane;
@@ -2396,6 +2396,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
   constexpr int kGroup = 4;
   static_assert(kItems % kGroup == 0, "whole groups");
   SegVal run = seg_identity<RAW>();
+#pragma unroll 1                                         /* (see 6.) */
   for (int i0 = 0; i0 < kItems; i0 += kGroup) {
     if (i0 >= items) break;
     SegVal v[kGroup];
@@ -2436,7 +2437,11 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
     if (w < (int)warp) carry = seg_combine<RAW>(carry, t);
   }
 
-  /* 6. second time: every request's position, estimate and decision; outputs */
+  /* 6. second time: every request's position, estimate and decision; outputs.  The loop is kept a
+   * loop: a block that is alone on the device (one small ctx) waits for its instructions more than
+   * for anything else (ncu: "no instruction" is its first stall reason), so code that runs once
+   * per group is not unrolled over the groups. */
+#pragma unroll 1
   for (int i0 = 0; i0 < kItems; i0 += kGroup) {
     if (i0 >= items) break;
     SegVal v[kGroup];

@@ -625,6 +625,77 @@ __device__ __forceinline__ void sort_rank_drop(const unsigned long long (&key)[C
   }
 }
 
+/* The same two steps for a pass whose digit has one or two bits (the top pass of a key of 8k + 1
+ * or 8k + 2 bits): the lanes that hold the same digit find each other by one ballot per digit
+ * bit, lane j keeps the warp's running count of digit j in a register, and neither the counting
+ * nor the ranking touches shared memory apart from the key's own store.  Measured at 2^24
+ * elements: a 1-bit pass 89 us against 120 us through the generic code (where 32 lanes hammer two
+ * counters); with four ballots (a 4-bit digit) the instructions outweigh the saved shared-memory
+ * traffic (16.2 us against 14.5 us at 2^20 elements), so wider digits stay on the generic code.
+ * The 89 us are what a pass costs with ranking almost free: tile load, write-out, scans and
+ * barriers.  Full tiles only (no padding keys). */
+template <int BITS>
+__device__ __forceinline__ uint32_t digit_peers(uint32_t d, const uint32_t (&bal)[BITS]) {
+  uint32_t m = 0xffffffffu;
+#pragma unroll
+  for (int k = 0; k < BITS; ++k) m &= ((d >> k) & 1u) ? bal[k] : ~bal[k];
+  return m;
+}
+
+template <int ITEMS, int BITS>
+__device__ __forceinline__ void sort_load_count_few(unsigned long long (&key)[kItemsHi], const unsigned long long* src,
+                                                    uint64_t first, uint32_t shift, uint32_t* slot_row, uint32_t lane) {
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) key[i] = src[first + i * 32 + lane];
+  uint32_t mine = 0;                                     /* lane j: keys of this warp with digit j */
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const uint32_t d = (uint32_t)(key[i] >> shift);
+    uint32_t bal[BITS];
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) bal[k] = __ballot_sync(0xffffffffu, (d >> k) & 1u);
+    mine += __popc(digit_peers<BITS>(lane, bal));
+  }
+  if (lane < (1u << BITS)) slot_row[lane] = mine;
+}
+
+template <int ITEMS, int CAP, int BITS>
+__device__ __forceinline__ void sort_rank_drop_few(const unsigned long long (&key)[CAP], uint32_t shift,
+                                                   const uint32_t* slot_row, unsigned long long* keys, uint32_t lane) {
+  uint32_t next = lane < (1u << BITS) ? slot_row[lane] : 0u;   /* lane j: next free slot of digit j for this warp */
+  const uint32_t below = (1u << lane) - 1;
+#pragma unroll
+  for (int i = 0; i < ITEMS; ++i) {
+    const uint32_t d = (uint32_t)(key[i] >> shift) & ((1u << BITS) - 1);
+    uint32_t bal[BITS];
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) bal[k] = __ballot_sync(0xffffffffu, (d >> k) & 1u);
+    const uint32_t grp = digit_peers<BITS>(d, bal);
+    const uint32_t first = __shfl_sync(0xffffffffu, next, d);
+    keys[first + __popc(grp & below)] = key[i];
+    next += __popc(digit_peers<BITS>(lane, bal));
+  }
+}
+
+/* digit width known at run time only: one instantiation per width */
+template <int ITEMS>
+__device__ __forceinline__ void sort_load_count_few_n(unsigned long long (&key)[kItemsHi], const unsigned long long* src,
+                                                      uint64_t first, uint32_t shift, uint32_t bits, uint32_t* slot_row,
+                                                      uint32_t lane) {
+  switch (bits) {
+    case 1: sort_load_count_few<ITEMS, 1>(key, src, first, shift, slot_row, lane); break;
+    default: sort_load_count_few<ITEMS, 2>(key, src, first, shift, slot_row, lane); break;
+  }
+}
+template <int ITEMS, int CAP>
+__device__ __forceinline__ void sort_rank_drop_few_n(const unsigned long long (&key)[CAP], uint32_t shift, uint32_t bits,
+                                                     const uint32_t* slot_row, unsigned long long* keys, uint32_t lane) {
+  switch (bits) {
+    case 1: sort_rank_drop_few<ITEMS, CAP, 1>(key, shift, slot_row, keys, lane); break;
+    default: sort_rank_drop_few<ITEMS, CAP, 2>(key, shift, slot_row, keys, lane); break;
+  }
+}
+
 template <bool PERSIST>
 __global__ void __launch_bounds__(kSortThreads, 2)
 k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf_a,
@@ -670,7 +741,13 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   const bool lo_warp = warp < kLoWarps;
   const uint32_t wfirst = lo_warp ? warp * (32 * kItemsLo)
                                   : kLoWarps * 32 * kItemsLo + (warp - kLoWarps) * (32 * kItemsHi);
-  if (lo_warp) sort_load_count<kItemsLo>(key, src, base + wfirst, n, shift, S.slot[warp], lane);
+  /* a digit of one or two bits on a full tile: counted and ranked by ballots */
+  const uint32_t dig_bits = min(8u, hdr->keybits - 8 * pass);
+  const bool few = dig_bits <= 2 && base + kSortTile <= (uint64_t)n;
+  if (few) {
+    if (lo_warp) sort_load_count_few_n<kItemsLo>(key, src, base + wfirst, shift, dig_bits, S.slot[warp], lane);
+    else sort_load_count_few_n<kItemsHi>(key, src, base + wfirst, shift, dig_bits, S.slot[warp], lane);
+  } else if (lo_warp) sort_load_count<kItemsLo>(key, src, base + wfirst, n, shift, S.slot[warp], lane);
   else sort_load_count<kItemsHi>(key, src, base + wfirst, n, shift, S.slot[warp], lane);
   __syncthreads();
 
@@ -741,7 +818,10 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   }
 
   /* 4. rank and drop into the tile buffer */
-  if (lo_warp) sort_rank_drop<kItemsLo, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
+  if (few) {
+    if (lo_warp) sort_rank_drop_few_n<kItemsLo, kItemsHi>(key, shift, dig_bits, S.slot[warp], S.keys, lane);
+    else sort_rank_drop_few_n<kItemsHi, kItemsHi>(key, shift, dig_bits, S.slot[warp], S.keys, lane);
+  } else if (lo_warp) sort_rank_drop<kItemsLo, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
   else sort_rank_drop<kItemsHi, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
   __syncthreads();
   if (S.abort) {
@@ -2572,6 +2652,7 @@ k_wide_reset(PlanHeader* hdr, uint32_t* __restrict__ hist, uint32_t* __restrict_
   pdl_wait();
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     hdr->npass = (wide_chunk_bits(hdr, sbits, ibits, super) + 7) / 8;
+    hdr->keybits = wide_chunk_bits(hdr, sbits, ibits, super);   /* what the passes of this super-pass sort */
     for (int i = 0; i <= kMaxPasses; ++i) hdr->ticket[i] = 0;
     if (super == 0) {
       hdr->wide = 2;                                      /* the chunked sort is under way */

@@ -125,6 +125,17 @@ def test_wide_deadline_span():
     both(_one_stage(20_000, dl, d=1 << 30, B=4, now=0))
 
 
+def test_top_digit_of_one_and_two_bits():
+    """Keys of 8k + 1 and 8k + 2 bits: the top radix pass ranks by ballots instead of through
+    shared memory (full tiles) and by the generic code (the ragged last tile)."""
+    rng = np.random.default_rng(14)
+    for span_bits in (9, 10, 17, 18):
+        n = 50_001
+        dl = rng.integers(0, 1 << span_bits, size=n)
+        dl[0], dl[1] = 0, (1 << span_bits) - 1              # the span is exactly span_bits wide
+        both(_one_stage(n, dl, d=3, B=2))
+
+
 def test_multiple_pipelines_and_padded_rows():
     rng = np.random.default_rng(9)
     pa = util.pipeline(inputs.chain_edges(2), 2, [30, 40])

@@ -130,6 +130,18 @@ def test_known_paths_with_queues_served_high_budget_first():
     check(wl, MASK)
 
 
+def test_grouped_promise_does_not_change_the_rules():
+    """PARD_MODE_GROUPED is a performance promise for the planner's own rule; the comparison rules
+    take their own path with or without it."""
+    wl = inputs.make("C4b", n_epochs=20, per_epoch=3000)
+    draw_masks(wl, np.random.default_rng(26))
+    for mode in (MASK, FCFS, NEXUS):
+        want = oracle.plan(wl.pipelines, wl.requests, wl.state, wl.n_ctx, mode)
+        rc, got = run_library(wl, mode | pb.PARD_MODE_GROUPED)
+        assert rc == 0
+        assert_identical(got, want)
+
+
 def test_mask_of_zero_is_the_default_plan():
     wl = inputs.make("C2b", n=50_001)
     rc, plain = run_library(wl, 0)

@@ -191,15 +191,19 @@ typedef struct pard_plan_out {
                                    then plans each ctx from start to end in shared memory
                                    -- constants, sort, positions, decisions -- in five
                                    kernel launches instead of about twenty, two to three
-                                   times faster on small and medium calls; larger calls
-                                   take the general path (which finds the grouping by
-                                   itself).  Where the block-per-ctx path runs, the device
-                                   checks the claim and a call that breaks it returns
-                                   PARD_EDATA; a call that cannot keep it (n > 8,192 *
-                                   n_ctx) returns PARD_EINVAL.  A call with a single ctx of
-                                   at most 8,192 requests is always planned by one block
-                                   (one kernel launch).  Ignored by the rules below, which
-                                   take their own path.  Same results. */
+                                   times faster on small and medium calls.  For larger
+                                   calls a block per ctx reads, checks and sorts its ctx
+                                   and the rest is the general path: without the promise
+                                   the library finds such grouping by itself, but has to
+                                   read all requests once more beforehand and to launch
+                                   the kernels of the ungrouped case in reserve.  The
+                                   device checks the claim: a call that breaks it returns
+                                   PARD_EDATA (as does any request out of range) with
+                                   unspecified outputs; a call that cannot keep it
+                                   (n > 8,192 * n_ctx) returns PARD_EINVAL.  A call with a
+                                   single ctx of at most 8,192 requests is always planned
+                                   by one block (one kernel launch).  Ignored by the rules
+                                   below, which take their own path.  Same results. */
 
 /* Other decision orders and rules on the same queues, for comparison with the
  * planner's own (which stays the default).  Their thresholds do not rise along

@@ -860,11 +860,16 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
  * all requests, which is checked here. */
 __global__ void __launch_bounds__(256)
 k_ctx_ranges(const uint4* __restrict__ req, uint32_t n, uint32_t n_ctx, uint32_t* __restrict__ ctx_start,
-             PlanHeader* hdr) {
+             PlanHeader* hdr, uint32_t fmt_dbits, uint32_t sbits) {
   pdl_wait();
   const uint32_t c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
   if (c > n_ctx) return;                         /* whole warps leave together */
+  if (c == 0 && lane == 0 && fmt_dbits) {        /* the element format is fixed by the host: no key-width step */
+    hdr->dbits = fmt_dbits;
+    hdr->keybits = sbits + fmt_dbits;
+    hdr->npass = 0;                              /* the sorted elements are in the first buffer */
+  }
   uint32_t lo[2] = {0, 0}, hi[2] = {n, n};       /* first request whose ctx is >= c, >= c + 1 */
   while (lo[0] < hi[0] || lo[1] < hi[1]) {
 #pragma unroll
@@ -2196,6 +2201,13 @@ struct LocalArgs {
   uint32_t* seg_off;               /* workspace copies, read by k_kept_scan / k_kept_move */
   uint32_t* seg_kept;
   uint32_t* kept_tmp;
+  /* sort only (large grouped calls): the block stops behind the sort, hands the elements over in
+   * the call's format -- fmt_dbits deadline bits, whatever the ctx's own span -- and publishes the
+   * ctx's deadline range; the kernels of the general path take it from there */
+  uint32_t sort_only, fmt_dbits;
+  unsigned long long* dst;
+  unsigned long long* ctx_dmin_inv;
+  unsigned long long* ctx_dmax;
 };
 
 template <int THREADS>
@@ -2263,7 +2275,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
     if (tid < sizeof(PlanHeader) / 4) reinterpret_cast<uint32_t*>(hdr)[tid] = 0;
     __syncthreads();
   } else if (hdr->unsorted || hdr->ctx_too_big) {      /* k_ctx_ranges found the promised grouping broken */
-    if (tid == 0 && c == 0) set_status(hdr, PARD_EDATA);
+    if (tid == 0 && c == 0) { set_status(hdr, PARD_EDATA); hdr->aborted = 1; }   /* nothing is sorted: later kernels return */
     return;
   }
   const uint32_t first = single ? 0u : a.ctx_start[c];
@@ -2310,7 +2322,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
   if (bad) Sm.flag_bad = 1;
   __syncthreads();
   if (Sm.flag_foreign) {                                 /* not grouped by ctx after all (or, with one ctx, a request of another) */
-    if (tid == 0) { hdr->unsorted = 1; set_status(hdr, PARD_EDATA); }
+    if (tid == 0) { hdr->unsorted = 1; set_status(hdr, PARD_EDATA); hdr->aborted = 1; }
     return;
   }
   unsigned long long dmin = ~0ull, dmax = 0;
@@ -2333,7 +2345,9 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
    * one block; else taken from the table k_seg_const has filled for all queues at once (a chain
    * of dependent loads that every block would otherwise wait for) and completed with what hangs
    * on the ctx's deadline range */
-  if (single) {
+  if (a.sort_only) {
+    /* the constants come later, from k_seg_const, once every ctx's range is known */
+  } else if (single) {
     for (uint32_t k = warp; k < S; k += WARPS) {
       bool kbad = false;
       const PardSegConst K = seg_const_warp(a.pipes, a.n_pipelines, a.st, c, k, dmin, dmax, lane, &kbad);
@@ -2382,7 +2396,7 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
       const uint32_t stage = stage16[pos];
       const uint32_t j = first + pos;
       if (stage != 0xffffu) {
-        const bool high_first = Sm.K[stage].narrow & kSegHighFirst;
+        const bool high_first = a.st.d_priority && a.st.d_priority[(size_t)c * S + stage] != 0;
         const unsigned long long off = (high_first ? dmax - D : D - dmin) & dmask;
         key[i] = ((((unsigned long long)stage << dbits) | off) << a.ibits) | j;
       } else {
@@ -2442,6 +2456,29 @@ k_plan_local(PlanHeader* __restrict__ hdr, const LocalArgs a) {
     for (int i = 0; i < kItems; ++i)
       if (i < items) Sm.keys[wfirst + i * 32 + lane] = key[i];
     __syncthreads();
+  }
+
+  if (a.sort_only) {
+    if (Sm.flag_bad) {                                   /* a flagged request has no place in the general path's order */
+      if (tid == 0) hdr->aborted = 1;
+      return;
+    }
+    if (dbits > a.fmt_dbits) {                           /* this ctx's span does not fit the call's element */
+      if (tid == 0) { hdr->wide = 1; set_status(hdr, PARD_ERANGE); }
+      return;
+    }
+    if (tid == 0 && dmin <= dmax) {
+      a.ctx_dmin_inv[c] = ~dmin;
+      a.ctx_dmax[c] = dmax;
+      atomicMax(&hdr->span_max, dmax - dmin);
+    }
+    const uint32_t kshift = a.ibits + dbits;
+    for (uint32_t pos = tid; pos < cnt; pos += THREADS) {
+      const unsigned long long e = Sm.keys[pos];
+      const unsigned long long seg = (unsigned long long)c * S + (uint32_t)(e >> kshift);
+      a.dst[first + pos] = ((seg << a.fmt_dbits | ((e >> a.ibits) & dmask)) << a.ibits) | (e & imask);
+    }
+    return;
   }
 
   /* 4. queue boundaries of the ctx */
@@ -3031,7 +3068,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     la.ktab = ktab; la.seg_off = seg_off; la.seg_kept = seg_kept; la.kept_tmp = out->d_kept_idx ? kept_tmp : nullptr;
     if (fused_grouped) {
       launch_pdl(k_clear, 4, 256, 0, stream, (uint4*)(ws + L.hdr), (unsigned long long)(L.hist / 16));
-      launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
+      launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr, 0u, 0u);
       /* the queues' constants; what depends on a ctx's deadline range is added by the ctx's block */
       launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax,
                  ktab, hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
@@ -3047,6 +3084,59 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
                    kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
     }
     while (phase <= PARD_N_PHASES) mark();             /* the phases are those of the other path: all of this counts as the first */
+    PARD_CUDA_OK(cudaGetLastError());
+    if (mode & PARD_MODE_NOWAIT) return PARD_OK;
+    rc = pard_plan_status(d_workspace, cuda_stream);
+    return rc == PARD_ERANGE ? plan_wide() : rc;
+  }
+
+  /* ---- the same promise for more contexts than that: a block per ctx still reads, checks and
+   * sorts its ctx (k_plan_local, stopping behind the sort) and publishes the ctx's deadline range,
+   * so that neither the prepass over all requests nor the packing and radix kernels (launched
+   * otherwise in case the device finds the requests not grouped) are needed; the element format
+   * is fixed here (all bits the queue id and the index leave), tables and decision as in the
+   * general path ---- */
+  if ((mode & PARD_MODE_GROUPED) && n_ctx > 1 && n > 0 && !rule_walk) {
+    const uint32_t fmt_dbits = std::min(60u, 64u - ibits - sbits);
+    LocalArgs la = {};
+    la.req = req4; la.ctx_start = ctx_start;
+    la.n = n32; la.n_ctx = n_ctx; la.ibits = ibits;
+    la.pipes = pipe_table; la.n_pipelines = n_pipelines; la.st = *state;
+    la.sort_only = 1; la.fmt_dbits = fmt_dbits; la.dst = buf_a; la.ctx_dmin_inv = ctx_dmin; la.ctx_dmax = ctx_dmax;
+    launch_pdl(k_clear, 8, 256, 0, stream, (uint4*)(ws + L.hdr), (unsigned long long)(L.hist / 16));
+    launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr, fmt_dbits, sbits);
+    launch_pdl(k_plan_local<false, 512>, n_ctx, 512, sizeof(LocalSmem<512>), stream, hdr, la);
+    launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
+               hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
+    if (L.n_seg >= kManyQueues)
+      launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
+                 seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
+                 (mode & PARD_MODE_SCAN) ? 1u : 0u, 1u);
+    else
+      launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
+                 out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
+                 (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits, 1u, 1u);
+    uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
+    long long* est = (long long*)out->d_est_us;
+    const bool raw = mode & PARD_MODE_RAW;
+    launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream,
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
+    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab);
+    auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
+                          : (state->d_priority ? k_decide_win<false, true> : k_decide_win<false, false>);
+    launch_pdl(decide_win, (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile), kDecThreads, 0, stream, hdr, buf_a, buf_b, n32,
+               ibits, ktab, seg_off, win_off, win_cnt, wtab, out->d_keep, est, out->d_perm, tmp, (const uint32_t*)seg_off, seg_kept);
+    launch_pdl(raw ? k_scan_path<true> : k_scan_path<false>, std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 2), kDecThreads, 0,
+               stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off, win_off, tile_agg, tile_carry, out->d_keep, est,
+               out->d_perm, tmp, seg_kept, kept_base, chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept,
+               out->d_kept_idx, 0u);
+    launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+               (unsigned long long*)out->d_n_kept);
+    if (out->d_kept_idx)
+      launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
+                                                 (uint32_t)sms * 8), 256, 0, stream,
+                 kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
+    while (phase <= PARD_N_PHASES) mark();
     PARD_CUDA_OK(cudaGetLastError());
     if (mode & PARD_MODE_NOWAIT) return PARD_OK;
     rc = pard_plan_status(d_workspace, cuda_stream);
@@ -3077,7 +3167,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
              hdr, sbits, ibits, fold_width ? 1u : 0u, arrival_order ? 1u : 0u, win_hist ? 1u : 0u,
              (mode & PARD_MODE_SCAN) ? 1u : 0u, win_off, win_cnt);
-  if (local_cand && !local_sure) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr);
+  if (local_cand && !local_sure) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr, 0u, 0u);
   mark();
   if (local_cand)                                /* every ctx inside one tile: sorted block by block, straight from the requests */
     launch_pdl(k_sort_local, n_ctx, kSortThreads, sizeof(SortSmem), stream, hdr, local_cand, req4, ctx_dmin, ctx_dmax,

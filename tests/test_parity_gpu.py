@@ -420,6 +420,19 @@ def test_broken_grouping_promise_is_reported():
     wl.requests = r
     rc, _ = run_library(wl, pb.PARD_MODE_GROUPED, check=False)
     assert rc == pb.PARD_EDATA
+    # the same two breaches in a call of more contexts than the block-per-ctx planner takes on
+    # (there a block per ctx only sorts): reported as well, nothing behind the sort runs
+    for breach in ("order", "size"):
+        wl = inputs.make("C4b", n_epochs=700, per_epoch=600)
+        r = wl.requests.copy()
+        if breach == "order":
+            r[[5, wl.n - 7]] = r[[wl.n - 7, 5]]
+        else:
+            r["ctx"][(r["ctx"] >= 100) & (r["ctx"] < 120)] = 100      # 20 epochs in one ctx: 12,000 requests
+        wl.requests = r
+        rc, _ = run_library(wl, pb.PARD_MODE_GROUPED, check=False)
+        assert rc == pb.PARD_EDATA, breach
+    grouped(inputs.make("C4b", n_epochs=700, per_epoch=600))
     # more requests than the contexts could hold: refused before anything is launched
     big = inputs.make("C5b", n_inst=2, per_inst=9000)
     rc, _ = run_library(big, pb.PARD_MODE_GROUPED, check=False)

@@ -48,7 +48,8 @@ typedef enum pard_status {
   PARD_OK          =  0,
   PARD_EINVAL      = -1,  /* null pointer, bad count, malformed CSR, bad flag        */
   PARD_ECYCLE      = -2,  /* the stage graph has a cycle                             */
-  PARD_ERANGE      = -3,  /* a host-visible value is outside the limits above        */
+  PARD_ERANGE      = -3,  /* a host-visible value is outside the limits above; with
+                             PARD_MODE_NOWAIT also: the sort key exceeds 64 bits     */
   PARD_ENOMEM      = -4,  /* host or device allocation failed (load time only)       */
   PARD_EWORKSPACE  = -5,  /* caller's workspace is smaller than required             */
   PARD_ETIMEOUT    = -6,  /* a bounded device-side wait ran out; outputs unspecified */
@@ -310,9 +311,11 @@ int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_t n_pipelin
  * reused for anything else in between. */
 int pard_plan_status(const void* d_workspace, void* cuda_stream);
 
-/* Number of kernels one pard_plan call enqueues for these sizes (memsets and
+/* Number of kernels one pard_plan call enqueues for these sizes under the
+ * default rule, without priorities and without PARD_MODE_GROUPED (memsets and
  * copies not counted).  Radix passes beyond the key width found on the device
- * are launched and return at once; they are included. */
+ * and the scan path are launched and return at once; they are included.  A
+ * key wider than 64 bits adds the kernels of its second stage. */
 int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t stage_stride,
                               uint32_t* launches);
 

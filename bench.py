@@ -577,7 +577,7 @@ def run_sharded(dev, dist, world, rank):
         wl = inputs.make(name)
         mine = sharding.shard_workload(wl, world, rank) if how == "ctx" else sharding.shard_by_stage(wl, world, rank)
         from paper_2602_08747_b200 import binding as pb
-        plan = DevicePlan(mine, dev, pb.PARD_MODE_GROUPED if name == "C4" else 0)
+        plan = DevicePlan(mine, dev, pb.PARD_MODE_GROUPED if name in ("C4", "C5") else 0)
         plan.step(nowait=False)
         steps = 20
         sec, _ = timed_steps(plan, steps, 5, dist)
@@ -714,14 +714,14 @@ def run_ours(args):
             # the other configurations of the workload list, device-resident, for the record
             for name in ("C1", "C2", "C4", "C5"):
                 wlo = inputs.make(name)
-                # C4's epochs arrive as one array grouped by epoch (= ctx), 8,192 requests each: the caller says so
-                plo = DevicePlan(wlo, dev, pb.PARD_MODE_GROUPED if name == "C4" else 0)
+                # C4's epochs and C5's instances arrive as one array grouped by epoch / instance (= ctx): the caller says so
+                plo = DevicePlan(wlo, dev, pb.PARD_MODE_GROUPED if name in ("C4", "C5") else 0)
                 plo.step(nowait=False)
                 kfo = float(plo.out.n_kept.cpu()[0]) / wlo.n
                 so, _ = timed_steps(plo, 50, 5, None)
                 others[name] = {"requests": wlo.n, "contexts": wlo.n_ctx, "us_per_step": 1e6 * so / 50,
                                 "requests_per_s": wlo.n * 50 / so, "keep_fraction": kfo,
-                                "mode": "PARD_MODE_GROUPED" if name == "C4" else "default"}
+                                "mode": "PARD_MODE_GROUPED" if name in ("C4", "C5") else "default"}
                 del plo, wlo
             # the many-context workloads also against the oracle on all host cores (bounded samples)
             others["C4"]["cpu_baseline_all_cores"] = oracle_all_cores("C4", {"n_epochs": 512, "per_epoch": 8192})

@@ -186,25 +186,31 @@ typedef struct pard_plan_out {
                                    block by block (requests grouped by ctx, no ctx above
                                    8,192 requests) have no wait in the sort */
 #define PARD_MODE_GROUPED 256u  /* the caller's word that d_requests is grouped by ascending
-                                   ctx and that no ctx holds more than 8,192 requests
-                                   (batched decision epochs, many small instances).  For
-                                   calls of up to a few hundred contexts one thread block
-                                   then plans each ctx from start to end in shared memory
-                                   -- constants, sort, positions, decisions -- in five
-                                   kernel launches instead of about twenty, two to three
-                                   times faster on small and medium calls.  For larger
-                                   calls a block per ctx reads, checks and sorts its ctx
-                                   and the rest is the general path: without the promise
-                                   the library finds such grouping by itself, but has to
-                                   read all requests once more beforehand and to launch
-                                   the kernels of the ungrouped case in reserve.  The
-                                   device checks the claim: a call that breaks it returns
-                                   PARD_EDATA (as does any request out of range) with
-                                   unspecified outputs; a call that cannot keep it
-                                   (n > 8,192 * n_ctx) returns PARD_EINVAL.  A call with a
-                                   single ctx of at most 8,192 requests is always planned
-                                   by one block (one kernel launch).  Ignored by the rules
-                                   below, which take their own path.  Same results. */
+                                   ctx (batched decision epochs, many instances in one
+                                   call).  What the library makes of it depends on the
+                                   sizes:
+                                   - contexts of at most 8,192 requests on average: the
+                                     promise then includes that NO ctx holds more than
+                                     8,192.  Up to a few hundred contexts one thread block
+                                     plans each ctx from start to end in shared memory --
+                                     constants, sort, positions, decisions -- in five
+                                     kernel launches instead of about twenty, two to three
+                                     times faster on small and medium calls; beyond that a
+                                     block per ctx reads, checks and sorts its ctx and the
+                                     rest is the general path, minus its pass over all
+                                     requests for the deadline ranges and minus the
+                                     kernels it launches in reserve for ungrouped input;
+                                   - larger contexts (and stage_stride a power of two):
+                                     the radix passes stay inside every ctx's range and
+                                     sort the stage and deadline bits only -- one pass
+                                     fewer whenever the ctx bits of the key cost one.
+                                   The device checks the claim: a call that breaks it
+                                   returns PARD_EDATA (as does, in the block-per-ctx
+                                   forms, any request out of range) with unspecified
+                                   outputs.  A call with a single ctx of at most 8,192
+                                   requests is always planned by one block (one kernel
+                                   launch).  Ignored by the rules below, which take their
+                                   own path.  Same results. */
 
 /* Other decision orders and rules on the same queues, for comparison with the
  * planner's own (which stays the default).  Their thresholds do not rise along

@@ -25,10 +25,12 @@ namespace {
 struct Layout {
   /* [hdr, zero_end) must be zero when the first kernel starts: cleared by k_clear (of the two
    * look-back arrays only the first: every sort pass clears the array of the pass after it) */
-  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, whist, lookback, zero_end,
+  uint64_t hdr, ctx_dmin, ctx_dmax, seg_off, seg_kept, win_done, hist, whist, hist_ctx, lookback, zero_end, tile_first,
       ctx_start, pipes, ktab, kept_base, chunk_base, tile_agg, tile_carry, win_off, win_cnt, win_own, win_big, wtab, kept_tmp,
       buf_a, buf_b, total;
   uint32_t n_seg, sort_tiles, dec_tiles, max_passes, win_capacity;
+  uint32_t lb_tiles;          /* tiles the look-back arrays are sized for */
+  uint32_t ctx_passes;        /* 1: the call may sort inside the contexts' ranges (contexts of more than a tile on average) */
 };
 
 __host__ __device__ inline uint32_t bit_width64(unsigned long long x) {
@@ -61,8 +63,14 @@ Layout make_layout(uint64_t n, uint32_t n_ctx, int32_t stage_stride) {
   L.win_done = o;  o = al(o + 4ull * L.n_seg);
   L.hist = o;      o = al(o + 4ull * kMaxPasses * kBins);
   L.whist = o;     o = al(o + (L.n_seg <= kHistSegs ? 4ull * kHistCap : 0ull));   /* window counts of calls with few queues */
-  L.lookback = o;  L.zero_end = al(o + 4ull * kBins * (uint64_t)L.sort_tiles);
-  o = al(o + 2 * 4ull * kBins * (uint64_t)L.sort_tiles);                    /* two arrays, used in turn */
+  /* passes kept inside the contexts' ranges cut the tiles at ctx boundaries: at most one more
+   * tile per ctx; they keep digit counts per ctx */
+  L.ctx_passes = (n_ctx > 1 && (uint64_t)n_ctx * kSortTile < n) ? 1u : 0u;
+  L.lb_tiles = L.sort_tiles + (L.ctx_passes ? n_ctx : 0u);
+  L.hist_ctx = o;  o = al(o + (L.ctx_passes ? 4ull * kMaxPasses * kBins * (uint64_t)n_ctx : 0ull));
+  L.lookback = o;  L.zero_end = al(o + 4ull * kBins * (uint64_t)L.lb_tiles);
+  o = al(o + 2 * 4ull * kBins * (uint64_t)L.lb_tiles);                      /* two arrays, used in turn */
+  L.tile_first = o; o = al(o + (L.ctx_passes ? 4ull * ((uint64_t)n_ctx + 1) : 0ull));
   L.ctx_start = o; o = al(o + 4ull * ((uint64_t)n_ctx + 1));
   L.pipes = o;     o = al(o + 8ull * kMaxPipelinesPerCall);
   L.ktab = o;      o = al(o + sizeof(PardSegConst) * (uint64_t)L.n_seg);
@@ -215,13 +223,15 @@ __global__ void k_ctx_span(const unsigned long long* __restrict__ ctx_dmin_inv,
 }
 
 /* Width of the sort key, once the widest deadline span is known. */
-__global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr, uint32_t arrival_order) {
+/* key_sbits: the queue-id bits that the passes have to sort (all of them, or the stage bits only
+ * when the passes stay inside the contexts' ranges) */
+__global__ void k_key_width(uint32_t sbits, uint32_t ibits, PlanHeader* hdr, uint32_t arrival_order, uint32_t key_sbits) {
   pdl_wait();
   /* in arrival order the deadline takes no part in the key: the index alone orders a queue */
   const uint32_t dbits = arrival_order ? 0u : bit_width64(hdr->span_max);
   hdr->dbits = dbits;
-  hdr->keybits = sbits + dbits;
-  hdr->npass = (sbits + dbits + 7) / 8;
+  hdr->keybits = key_sbits + dbits;
+  hdr->npass = (key_sbits + dbits + 7) / 8;
   if (sbits + dbits + ibits > 64) {
     hdr->npass = 0;
     hdr->wide = 1;
@@ -317,7 +327,8 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
             const unsigned long long* __restrict__ ctx_dmin_inv,
             const unsigned long long* __restrict__ ctx_dmax, PardSegConst* __restrict__ ktab,
             PlanHeader* hdr, uint32_t sbits, uint32_t ibits, uint32_t with_key_width, uint32_t arrival_order,
-            uint32_t win_hist, uint32_t force_scan, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt) {
+            uint32_t win_hist, uint32_t force_scan, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
+            uint32_t key_sbits) {
   pdl_wait();
   const uint32_t S = (uint32_t)st.stage_stride;
   const uint32_t lane = threadIdx.x & 31;
@@ -350,8 +361,8 @@ k_seg_const(const PipeTable pipes, uint32_t n_pipelines,
     const uint32_t dbits = arrival_order ? 0u : bit_width64(span);
     hdr->span_max = span;
     hdr->dbits = dbits;
-    hdr->keybits = sbits + dbits;
-    hdr->npass = (sbits + dbits + 7) / 8;
+    hdr->keybits = key_sbits + dbits;
+    hdr->npass = (key_sbits + dbits + 7) / 8;
     if (sbits + dbits + ibits > 64) {
       hdr->npass = 0;
       hdr->wide = 1;
@@ -585,31 +596,32 @@ struct SortSmem {
   uint32_t scan[2][kSortThreads / 32];
   uint32_t tile;
   uint32_t abort;
+  uint32_t ctx, lo_tile, base, limit, first;   /* the tile's ctx and range when passes stay inside the contexts */
 };
 
 /* one warp's share of step 1: ITEMS rounds of 32 consecutive elements */
 template <int ITEMS>
 __device__ __forceinline__ void sort_load_count(unsigned long long (&key)[kItemsHi], const unsigned long long* src,
                                                 uint64_t first, uint32_t n, uint32_t shift, uint32_t* slot_row,
-                                                uint32_t lane) {
+                                                uint32_t lane, uint32_t dig_mask = 255u) {
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
     const uint64_t j = first + i * 32 + lane;
     key[i] = j < n ? src[j] : ~0ull;
   }
 #pragma unroll
-  for (int i = 0; i < ITEMS; ++i) atomicAdd(&slot_row[(uint32_t)(key[i] >> shift) & 255u], 1u);
+  for (int i = 0; i < ITEMS; ++i) atomicAdd(&slot_row[(uint32_t)(key[i] >> shift) & dig_mask], 1u);
 }
 
 /* one warp's share of step 4 */
 template <int ITEMS, int CAP>
 __device__ __forceinline__ void sort_rank_drop(const unsigned long long (&key)[CAP], uint32_t shift,
                                                uint32_t* slot_row, uint32_t* match_row, unsigned long long* keys,
-                                               uint32_t lanebit, int items = ITEMS) {
+                                               uint32_t lanebit, int items = ITEMS, uint32_t dig_mask = 255u) {
 #pragma unroll
   for (int i = 0; i < ITEMS; ++i) {
     if (i >= items) break;                             /* the same for the whole block */
-    const uint32_t d = (uint32_t)(key[i] >> shift) & 255u;
+    const uint32_t d = (uint32_t)(key[i] >> shift) & dig_mask;
     atomicOr(&match_row[d], lanebit);
     __syncwarp();
     const uint32_t grp = match_row[d];
@@ -696,12 +708,23 @@ __device__ __forceinline__ void sort_rank_drop_few_n(const unsigned long long (&
   }
 }
 
-template <bool PERSIST>
+/* CTX: the pass stays inside every ctx's range of the array (requests grouped by ctx, contexts of
+ * more than a tile): tiles are cut at ctx boundaries (tile_first[c] = first tile of ctx c), the
+ * digit counts are per ctx, a digit's range starts at the ctx's first position, and the look-back
+ * stops at the ctx's first tile -- so the ctx bits of the key need no pass at all. */
+struct CtxTiles {
+  const uint32_t* ctx_start;     /* [n_ctx + 1] */
+  const uint32_t* tile_first;    /* [n_ctx + 1] */
+  const uint32_t* hist;          /* [n_ctx][kMaxPasses][kBins] */
+  uint32_t n_ctx;
+};
+
+template <bool PERSIST, bool CTX>
 __global__ void __launch_bounds__(kSortThreads, 2)
 k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf_a,
             unsigned long long* __restrict__ buf_b, const uint32_t* __restrict__ hist,
             uint32_t* __restrict__ lookback, uint32_t* __restrict__ lookback_next, uint32_t n,
-            uint32_t ibits, uint32_t stall, uint32_t local_candidate) {
+            uint32_t ibits, uint32_t stall, uint32_t local_candidate, const CtxTiles ct) {
   pdl_wait();
   constexpr int WARPS = kSortThreads / 32;
   static_assert(kLoWarps * 32 == kBins, "one look-back thread per digit");
@@ -720,18 +743,35 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
    * otherwise one tile per block */
   for (;;) {
   if (tid == 0) {
-    S.tile = atomicAdd(&hdr->ticket[pass], 1u);
+    const uint32_t t = atomicAdd(&hdr->ticket[pass], 1u);
+    S.tile = t;
     S.abort = 0;
+    if (CTX) {                                           /* the ctx of the tile: last c with tile_first[c] <= t */
+      uint32_t lo = 0, hi = ct.n_ctx;
+      while (hi - lo > 1) {
+        const uint32_t mid = lo + (hi - lo) / 2;
+        if (ct.tile_first[mid] <= t) lo = mid; else hi = mid;
+      }
+      S.ctx = t < ct.tile_first[ct.n_ctx] ? lo : 0xffffffffu;     /* the grid may hold more blocks than there are tiles */
+      S.lo_tile = ct.tile_first[lo];
+      S.base = ct.ctx_start[lo] + (t - ct.tile_first[lo]) * (uint32_t)kSortTile;
+      S.limit = ct.ctx_start[lo + 1];
+      S.first = ct.ctx_start[lo];
+    }
   }
   for (uint32_t i = tid; i < WARPS * kBins; i += kSortThreads) {
     (&S.slot[0][0])[i] = 0;
     (&S.match[0][0])[i] = 0;
   }
-  const uint32_t gh = tid < kBins ? hist[tid] : 0;     /* global count of digit tid, needed in step 2 */
+  uint32_t gh = (!CTX && tid < kBins) ? hist[tid] : 0; /* count of digit tid in the whole array (in the ctx), needed in step 2 */
   __syncthreads();
   const uint32_t tile = S.tile;
   if (PERSIST && tile >= n_tiles) return;
-  const uint64_t base = (uint64_t)tile * kSortTile;
+  if (CTX && S.ctx == 0xffffffffu) return;
+  if (CTX && tid < kBins) gh = ct.hist[((size_t)S.ctx * kMaxPasses + pass) * kBins + tid];
+  const uint64_t base = CTX ? (uint64_t)S.base : (uint64_t)tile * kSortTile;
+  const uint32_t limit = CTX ? S.limit : n;            /* end of the range the tile belongs to */
+  const int64_t lo_tile = CTX ? (int64_t)S.lo_tile : 0;
   const uint32_t shift = ibits + 8 * pass;
 
   /* 1. load and count.  The warps that will do the look-back own fewer
@@ -743,12 +783,15 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
                                   : kLoWarps * 32 * kItemsLo + (warp - kLoWarps) * (32 * kItemsHi);
   /* a digit of one or two bits on a full tile: counted and ranked by ballots */
   const uint32_t dig_bits = min(8u, hdr->keybits - 8 * pass);
-  const bool few = dig_bits <= 2 && base + kSortTile <= (uint64_t)n;
+  /* inside a ctx the bits above the key (the ctx's part of the queue id) are the same everywhere
+   * and take no part in the digit */
+  const uint32_t dig_mask = CTX ? (1u << dig_bits) - 1 : 255u;
+  const bool few = dig_bits <= 2 && base + kSortTile <= (uint64_t)limit;
   if (few) {
     if (lo_warp) sort_load_count_few_n<kItemsLo>(key, src, base + wfirst, shift, dig_bits, S.slot[warp], lane);
     else sort_load_count_few_n<kItemsHi>(key, src, base + wfirst, shift, dig_bits, S.slot[warp], lane);
-  } else if (lo_warp) sort_load_count<kItemsLo>(key, src, base + wfirst, n, shift, S.slot[warp], lane);
-  else sort_load_count<kItemsHi>(key, src, base + wfirst, n, shift, S.slot[warp], lane);
+  } else if (lo_warp) sort_load_count<kItemsLo>(key, src, base + wfirst, limit, shift, S.slot[warp], lane, dig_mask);
+  else sort_load_count<kItemsHi>(key, src, base + wfirst, limit, shift, S.slot[warp], lane, dig_mask);
   __syncthreads();
 
   /* 2. thread d owns digit d */
@@ -780,7 +823,7 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
     for (int w = 0; w < kBins / 32; ++w)
       if (w < (int)warp) { wx += S.scan[0][w]; wg += S.scan[1][w]; }
     dstart = wx + x - cnt;                             /* first tile-local slot of digit tid  */
-    gstart = wg + g - gh;                              /* first global position of digit tid  */
+    gstart = wg + g - gh + (CTX ? S.first : 0u);       /* first global position of digit tid  */
     S.dstart[tid] = dstart;
 #pragma unroll
     for (int w = 0; w < WARPS; ++w) S.slot[w][tid] += dstart;
@@ -792,12 +835,12 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
     const uint32_t* lb = lookback;
     uint32_t excl = 0, spins = 0;
     int64_t t = (int64_t)tile - 1;
-    bool done = t < 0;
+    bool done = t < lo_tile;
     while (!done) {
       uint32_t v[kLookBatch];
 #pragma unroll
       for (int k = 0; k < kLookBatch; ++k)
-        v[k] = (t - k >= 0) ? ld_relaxed(lb + (size_t)(t - k) * kBins + tid) : +kLbIncl;   /* before tile 0: nothing */
+        v[k] = (t - k >= lo_tile) ? ld_relaxed(lb + (size_t)(t - k) * kBins + tid) : +kLbIncl;   /* before the first tile: nothing */
       int used = 0;
 #pragma unroll
       for (int k = 0; k < kLookBatch; ++k) {
@@ -821,8 +864,8 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   if (few) {
     if (lo_warp) sort_rank_drop_few_n<kItemsLo, kItemsHi>(key, shift, dig_bits, S.slot[warp], S.keys, lane);
     else sort_rank_drop_few_n<kItemsHi, kItemsHi>(key, shift, dig_bits, S.slot[warp], S.keys, lane);
-  } else if (lo_warp) sort_rank_drop<kItemsLo, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
-  else sort_rank_drop<kItemsHi, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit);
+  } else if (lo_warp) sort_rank_drop<kItemsLo, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit, kItemsLo, dig_mask);
+  else sort_rank_drop<kItemsHi, kItemsHi>(key, shift, S.slot[warp], S.match[warp], S.keys, lanebit, kItemsHi, dig_mask);
   __syncthreads();
   if (S.abort) {
     if (tid == 0) set_aborted(hdr);
@@ -830,16 +873,115 @@ k_sort_pass(uint32_t pass, PlanHeader* hdr, unsigned long long* __restrict__ buf
   }
 
   /* 5. write out */
-  const uint32_t nvalid = (uint32_t)min((uint64_t)kSortTile, (uint64_t)n - base);
+  const uint32_t nvalid = (uint32_t)min((uint64_t)kSortTile, (uint64_t)limit - base);
 #pragma unroll 4
   for (uint32_t pos = tid; pos < nvalid; pos += kSortThreads) {
     const unsigned long long k = S.keys[pos];
-    const uint32_t d = (uint32_t)(k >> shift) & 255u;
+    const uint32_t d = (uint32_t)(k >> shift) & dig_mask;
     dst[S.gofs[d] + pos] = k;
   }
   if (!PERSIST) return;
   __syncthreads();                                     /* the tile buffer and the tables are reused */
   }
+}
+
+/* First tile of every ctx when the tiles are cut at ctx boundaries: the running sum of
+ * ceil(requests of the ctx / kSortTile).  One block. */
+__global__ void __launch_bounds__(1024)
+k_tile_table(const uint32_t* __restrict__ ctx_start, uint32_t n_ctx, uint32_t* __restrict__ tile_first) {
+  pdl_wait();
+  __shared__ uint32_t s_w[32];
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t per = (n_ctx + 1023) / 1024;          /* contexts per thread, consecutive */
+  const uint32_t c0 = tid * per, c1 = min(n_ctx, c0 + per);
+  uint32_t sum = 0;
+  for (uint32_t c = c0; c < c1; ++c) sum += (ctx_start[c + 1] - ctx_start[c] + kSortTile - 1) / kSortTile;
+  uint32_t incl = sum;
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= (uint32_t)o) incl += y;
+  }
+  if (lane == 31) s_w[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const uint32_t w = s_w[lane];
+    uint32_t x = w;
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= (uint32_t)o) x += y;
+    }
+    s_w[lane] = x - w;
+  }
+  __syncthreads();
+  uint32_t run = s_w[warp] + incl - sum;
+  for (uint32_t c = c0; c < c1; ++c) {
+    tile_first[c] = run;
+    run += (ctx_start[c + 1] - ctx_start[c] + kSortTile - 1) / kSortTile;
+  }
+  if (c1 == n_ctx && c0 < n_ctx) tile_first[n_ctx] = run;
+  if (n_ctx == 0 && tid == 0) tile_first[0] = 0;
+}
+
+/* k_pack for passes that stay inside the contexts: a block packs one tile (all of one ctx) and
+ * adds its digit counts to the ctx's.  The digits cover the stage and deadline bits only; a
+ * request of another ctx inside the tile breaks the caller's promise. */
+__global__ void __launch_bounds__(256)
+k_pack_ctx(const uint4* __restrict__ req, uint32_t S, const unsigned long long* __restrict__ ctx_dmin_inv,
+           const unsigned long long* __restrict__ ctx_dmax, const uint8_t* __restrict__ priority, uint32_t ibits,
+           PlanHeader* __restrict__ hdr, unsigned long long* __restrict__ dst, uint32_t* __restrict__ hist_ctx,
+           const CtxTiles ct) {
+  pdl_wait();
+  __shared__ uint32_t s_hist[kMaxPasses * kBins];
+  __shared__ uint32_t s_c, s_base, s_limit;
+  if (hdr->unsorted) {                                   /* k_ctx_ranges found the requests out of ctx order */
+    if (blockIdx.x == 0 && threadIdx.x == 0) { hdr->aborted = 1; set_status(hdr, PARD_EDATA); }
+    return;
+  }
+  if (hdr->wide || hdr->aborted) return;
+  const uint32_t tile = blockIdx.x;
+  if (threadIdx.x == 0) {
+    uint32_t lo = 0, hi = ct.n_ctx;
+    while (hi - lo > 1) {
+      const uint32_t mid = lo + (hi - lo) / 2;
+      if (ct.tile_first[mid] <= tile) lo = mid; else hi = mid;
+    }
+    s_c = tile < ct.tile_first[ct.n_ctx] ? lo : 0xffffffffu;
+    s_base = ct.ctx_start[lo] + (tile - ct.tile_first[lo]) * (uint32_t)kSortTile;
+    s_limit = ct.ctx_start[lo + 1];
+  }
+  const uint32_t npass = hdr->npass, dbits = hdr->dbits;
+  for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x) s_hist[i] = 0;
+  __syncthreads();
+  const uint32_t c = s_c;
+  if (c == 0xffffffffu) return;
+  const uint32_t end = min(s_limit, s_base + (uint32_t)kSortTile);
+  const unsigned long long dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
+  const unsigned long long cmin = ~ctx_dmin_inv[c], cmax = ctx_dmax[c];
+  const unsigned long long keymask = hdr->keybits >= 64 ? ~0ull : ((1ull << hdr->keybits) - 1);
+  bool foreign = false;
+  for (uint32_t j = s_base + threadIdx.x; j < end; j += blockDim.x) {
+    const uint4 r = __ldg(&req[j]);
+    const unsigned long long D = ((unsigned long long)r.y << 32) | r.x;
+    const uint32_t stage = r.w & 0xffffu;
+    unsigned long long key = 0;
+    if (r.z != c) foreign = true;
+    else if (stage < S) {
+      const uint32_t seg = c * S + stage;
+      const bool high_first = priority && __ldg(&priority[seg]) != 0;
+      key = ((unsigned long long)seg << dbits) | ((high_first ? cmax - D : D - cmin) & dmask);
+    }
+    dst[j] = (key << ibits) | j;                         /* a flagged request keeps its index alone, as in k_pack */
+    key &= keymask;                                      /* the ctx's part of the queue id takes no part in the digits */
+    uint32_t* hp = s_hist;
+    for (uint32_t p = 0; p < npass; ++p, hp += kBins, key >>= 8) atomicAdd(hp + ((uint32_t)key & 255u), 1u);
+  }
+  if (__syncthreads_or(foreign)) {
+    if (threadIdx.x == 0) { hdr->unsorted = 1; hdr->aborted = 1; set_status(hdr, PARD_EDATA); }
+    return;
+  }
+  uint32_t* h = hist_ctx + (size_t)c * kMaxPasses * kBins;
+  for (uint32_t i = threadIdx.x; i < npass * kBins; i += blockDim.x)
+    if (s_hist[i]) atomicAdd(&h[i], s_hist[i]);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -2824,9 +2966,11 @@ int allow_sort_smem(int dev) {
   if (done[dev].load(std::memory_order_acquire)) return PARD_OK;    /* every call but the first on a device */
   std::lock_guard<std::mutex> lock(mu);
   if (!done[dev].load(std::memory_order_relaxed)) {
-    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
-    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)sizeof(SortSmem)));
+    PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_pass<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
     PARD_CUDA_OK(cudaFuncSetAttribute(k_sort_local, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)sizeof(SortSmem)));
@@ -2896,7 +3040,6 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   constexpr uint32_t kRuleBits = PARD_MODE_PATH_MASK | PARD_MODE_FCFS | PARD_MODE_NEXUS | PARD_MODE_CLIPPER;
   if (mode & ~(PARD_MODE_RAW | PARD_MODE_NOWAIT | PARD_MODE_SCAN | PARD_MODE_TEST_STALL | PARD_MODE_GROUPED | kRuleBits))
     return PARD_EINVAL;
-  if ((mode & PARD_MODE_GROUPED) && n > (uint64_t)n_ctx * (uint64_t)kSortTile) return PARD_EINVAL;   /* some ctx must exceed a tile */
   /* the rules decided by a walk of every queue, and what they combine with */
   const bool rule_walk = (mode & kRuleBits) != 0;
   const bool arrival_order = (mode & (PARD_MODE_FCFS | PARD_MODE_NEXUS | PARD_MODE_CLIPPER)) != 0;
@@ -2940,7 +3083,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   PardSegConst* ktab = (PardSegConst*)(ws + L.ktab);
   uint32_t* hist = (uint32_t*)(ws + L.hist);
   uint32_t* lookback = (uint32_t*)(ws + L.lookback);
-  const size_t lb_words = (size_t)L.sort_tiles * kBins;
+  const size_t lb_words = (size_t)L.lb_tiles * kBins;
   unsigned long long* tile_agg = (unsigned long long*)(ws + L.tile_agg);
   int32_t* tile_carry = (int32_t*)(ws + L.tile_carry);
   uint32_t* seg_kept = (uint32_t*)(ws + L.seg_kept);
@@ -3004,9 +3147,9 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     launch_pdl(k_prepass, (uint32_t)std::min<uint64_t>((n + 2047) / 2048, (uint64_t)sms * 8), 256, 0, stream, req4, n32, n_ctx,
                S, ctx_dmin, ctx_dmax, hdr);
     launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
-    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr, 0u);
+    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr, 0u, sbits);
     launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
-               hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
+               hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt, sbits);
     const uint32_t cw = 64 - ibits;                         /* key bits per super-pass */
     const uint32_t supers = (sbits + 60 + cw - 1) / cw;     /* for the widest legal span; chunks beyond the key are empty */
     const uint32_t chunk_passes = std::min<uint32_t>(kMaxPasses, (cw + 7) / 8);
@@ -3017,8 +3160,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
       launch_pdl(k_wide_pack, grid_n, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, state->d_priority, sbits, ibits,
                  sp, (const PlanHeader*)hdr, (const uint32_t*)order, buf_a, hist);
       for (uint32_t p = 0; p < chunk_passes; ++p)
-        launch_pdl(k_sort_pass<false>, L.sort_tiles, kSortThreads, sizeof(SortSmem), stream, p, hdr, buf_a, buf_b, hist,
-                   lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words, n32, ibits, 0u, 0u);
+        launch_pdl(k_sort_pass<false, false>, L.sort_tiles, kSortThreads, sizeof(SortSmem), stream, p, hdr, buf_a, buf_b, hist,
+                   lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words, n32, ibits, 0u, 0u, CtxTiles{});
       launch_pdl(k_wide_chase, grid_n, 256, 0, stream, (const PlanHeader*)hdr, (const unsigned long long*)buf_a, buf_b, n32,
                  ibits, sp, (const uint32_t*)order);
       launch_pdl(k_wide_keep, grid_n, 256, 0, stream, (const PlanHeader*)hdr, (const unsigned long long*)buf_a,
@@ -3056,7 +3199,8 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   const bool fused_single = n_ctx == 1 && n > 0 && n <= (uint64_t)kSortTile && !rule_walk;
   /* worth it while the blocks fit a few waves: beyond that the streaming decision kernel of the
    * general path (which finds the grouping by itself) does the positions cheaper than the blocks' scans */
-  const bool fused_grouped = (mode & PARD_MODE_GROUPED) && n_ctx > 1 && n > 0 && !rule_walk && n_ctx <= 4u * (uint32_t)sms;
+  const bool fused_grouped = (mode & PARD_MODE_GROUPED) && n_ctx > 1 && n > 0 && !rule_walk && n_ctx <= 4u * (uint32_t)sms &&
+                             !L.ctx_passes;
   if (fused_single || fused_grouped) {
     LocalArgs la = {};
     la.req = req4; la.ctx_start = fused_single ? nullptr : ctx_start;
@@ -3071,7 +3215,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
       launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr, 0u, 0u);
       /* the queues' constants; what depends on a ctx's deadline range is added by the ctx's block */
       launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax,
-                 ktab, hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
+                 ktab, hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt, sbits);
     }
     launch_pdl((mode & PARD_MODE_RAW) ? k_plan_local<true, 512> : k_plan_local<false, 512>, n_ctx, 512,
                sizeof(LocalSmem<512>), stream, hdr, la);
@@ -3096,7 +3240,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
    * otherwise in case the device finds the requests not grouped) are needed; the element format
    * is fixed here (all bits the queue id and the index leave), tables and decision as in the
    * general path ---- */
-  if ((mode & PARD_MODE_GROUPED) && n_ctx > 1 && n > 0 && !rule_walk) {
+  if ((mode & PARD_MODE_GROUPED) && n_ctx > 1 && n > 0 && !rule_walk && !L.ctx_passes) {
     const uint32_t fmt_dbits = std::min(60u, 64u - ibits - sbits);
     LocalArgs la = {};
     la.req = req4; la.ctx_start = ctx_start;
@@ -3107,7 +3251,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr, fmt_dbits, sbits);
     launch_pdl(k_plan_local<false, 512>, n_ctx, 512, sizeof(LocalSmem<512>), stream, hdr, la);
     launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
-               hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt);
+               hdr, sbits, ibits, 0u, 0u, 0u, 0u, win_off, win_cnt, sbits);
     if (L.n_seg >= kManyQueues)
       launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
                  seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
@@ -3156,24 +3300,37 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     launch_pdl(k_prepass, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax, hdr);
   }
   mark();
+  /* Requests grouped by ctx (the caller's word) with contexts of more than a tile on average: the
+   * radix passes stay inside every ctx's range -- tiles cut at ctx boundaries, digit counts per
+   * ctx, look-back up to the ctx's first tile -- and sort the stage and deadline bits only; the
+   * ctx bits of the key need no pass (C5: four passes instead of five).  Needs the stage in the low
+   * bits of the queue id: stage_stride a power of two. */
+  const bool ctx_sort = (mode & PARD_MODE_GROUPED) && L.ctx_passes && (S & (S - 1)) == 0 && !rule_walk && n > 0;
+  const uint32_t key_sbits = ctx_sort ? ceil_log2(S) : sbits;
+  const CtxTiles ctx_tiles = {ctx_start, (const uint32_t*)(ws + L.tile_first), (const uint32_t*)(ws + L.hist_ctx), n_ctx};
   const bool fold_width = L.n_seg <= kFoldSegs;          /* few queues: k_seg_const's last block finds the key width */
   if (!fold_width) {
     if (n > 0) launch_pdl(k_ctx_span, (n_ctx + 255) / 256, 256, 0, stream, ctx_dmin, ctx_dmax, n_ctx, hdr);
-    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr, arrival_order ? 1u : 0u);
+    launch_pdl(k_key_width, 1, 1, 0, stream, sbits, ibits, hdr, arrival_order ? 1u : 0u, key_sbits);
   }
   /* few queues, decided by the planner's own rule in budget order from the start of every queue:
    * the window tables are counted while the requests are packed */
-  const bool win_hist = n > 0 && L.n_seg <= kHistSegs && !rule_walk && !state->d_priority && !local_cand;
+  const bool win_hist = n > 0 && L.n_seg <= kHistSegs && !rule_walk && !state->d_priority && !local_cand && !ctx_sort;
   launch_pdl(k_seg_const, (L.n_seg + 3) / 4, 128, 0, stream, pipe_table, n_pipelines, *state, n_ctx, ctx_dmin, ctx_dmax, ktab,
              hdr, sbits, ibits, fold_width ? 1u : 0u, arrival_order ? 1u : 0u, win_hist ? 1u : 0u,
-             (mode & PARD_MODE_SCAN) ? 1u : 0u, win_off, win_cnt);
-  if (local_cand && !local_sure) launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr, 0u, 0u);
+             (mode & PARD_MODE_SCAN) ? 1u : 0u, win_off, win_cnt, key_sbits);
+  if ((local_cand && !local_sure) || ctx_sort)
+    launch_pdl(k_ctx_ranges, (n_ctx + 1 + 7) / 8, 256, 0, stream, req4, n32, n_ctx, ctx_start, hdr, 0u, 0u);
+  if (ctx_sort) launch_pdl(k_tile_table, 1, 1024, 0, stream, (const uint32_t*)ctx_start, n_ctx, (uint32_t*)(ws + L.tile_first));
   mark();
   if (local_cand)                                /* every ctx inside one tile: sorted block by block, straight from the requests */
     launch_pdl(k_sort_local, n_ctx, kSortThreads, sizeof(SortSmem), stream, hdr, local_cand, req4, ctx_dmin, ctx_dmax,
                state->d_priority, buf_a, buf_b, local_sure ? (const uint32_t*)nullptr : (const uint32_t*)ctx_start, n32, S,
                ceil_log2(S), ibits);
-  if (n > 0 && !local_sure) {                    /* returns at once when the blocks above did the work */
+  if (ctx_sort) {
+    launch_pdl(k_pack_ctx, L.lb_tiles, 256, 0, stream, req4, S, ctx_dmin, ctx_dmax, state->d_priority, ibits, hdr, buf_a,
+               (uint32_t*)(ws + L.hist_ctx), ctx_tiles);
+  } else if (n > 0 && !local_sure) {             /* returns at once when the blocks above did the work */
     uint32_t grid = (uint32_t)std::min<uint64_t>((n + 255) / 256, (uint64_t)sms * 8);
     launch_pdl(win_hist ? k_pack<true> : k_pack<false>, grid, 256, 0, stream, req4, n32, n_ctx, S, ctx_dmin, ctx_dmax,
                state->d_priority, ibits, hdr, buf_a, hist, local_cand, (const PardSegConst*)ktab, (const uint32_t*)win_off,
@@ -3186,11 +3343,15 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   }
   for (uint32_t p = 0; p < (uint32_t)kMaxPasses; ++p) {
     mark();
-    if (n > 0 && p < L.max_passes && !local_sure)
-      launch_pdl(local_cand ? k_sort_pass<true> : k_sort_pass<false>,
+    if (ctx_sort) {
+      if (p < std::min<uint32_t>(kMaxPasses, (key_sbits + 60 + 7) / 8))
+        launch_pdl(k_sort_pass<false, true>, L.lb_tiles, kSortThreads, sizeof(SortSmem), stream, p, hdr, buf_a, buf_b, hist,
+                   lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words, n32, ibits, 0u, 0u, ctx_tiles);
+    } else if (n > 0 && p < L.max_passes && !local_sure)
+      launch_pdl(local_cand ? k_sort_pass<true, false> : k_sort_pass<false, false>,
                  local_cand ? std::min<uint32_t>(L.sort_tiles, 2u * (uint32_t)sms) : L.sort_tiles, kSortThreads, sizeof(SortSmem), stream,
           p, hdr, buf_a, buf_b, hist, lookback + (p & 1) * lb_words, lookback + ((p + 1) & 1) * lb_words,
-          n32, ibits, (p == 0 && (mode & PARD_MODE_TEST_STALL)) ? 1u : 0u, local_cand);
+          n32, ibits, (p == 0 && (mode & PARD_MODE_TEST_STALL)) ? 1u : 0u, local_cand, CtxTiles{});
   }
   mark();
   if (win_hist) {
@@ -3202,7 +3363,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   else
     launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
                out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits, local_cand, rule_walk ? 0u : 1u);
+               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, ctx_sort ? 64u : sbits, local_cand, rule_walk ? 0u : 1u);
   if (n > 0 && rule_walk) {
     /* a rule without rising thresholds: every queue is walked in order (pard_policy.cu) */
     PolicyArgs pa = {};

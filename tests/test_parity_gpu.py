@@ -390,6 +390,44 @@ def test_block_per_ctx_on_the_grouped_configs(name, kw, mode):
     grouped(inputs.make(name, **kw), mode)
 
 
+def test_grouped_contexts_larger_than_a_tile_sort_inside_their_ranges():
+    """PARD_MODE_GROUPED with contexts of more than a sort tile on average: the radix passes stay
+    inside every ctx's range and leave the ctx bits alone."""
+    for mode in (0, 1):
+        grouped(inputs.make("C5b", n_inst=16, per_inst=65536), mode)
+    grouped(inputs.make("C5", n_inst=9, per_inst=20_001))
+    # ragged: contexts far below a tile, one empty, several of many tiles; priorities
+    rng = np.random.default_rng(15)
+    wl = inputs.make("C5b", n_inst=12, per_inst=30_000)
+    share = rng.uniform(0.05, 1.0, size=wl.n_ctx)
+    share[3] = 0.0
+    share[7] = 1.0
+    keep = rng.random(wl.n) < share[wl.requests["ctx"]]
+    wl.requests = np.ascontiguousarray(wl.requests[keep])
+    assert wl.n > wl.n_ctx * 8192
+    grouped(wl)
+    wl.state.priority = rng.integers(0, 2, size=(wl.n_ctx, wl.state.stage_stride)).astype(np.uint8)
+    grouped(wl)
+    grouped(wl, 1)
+    # a broken promise is reported
+    r = wl.requests.copy()
+    r[[5, wl.n - 7]] = r[[wl.n - 7, 5]]
+    wl.requests = r
+    rc, _ = run_library(wl, pb.PARD_MODE_GROUPED, check=False)
+    assert rc == pb.PARD_EDATA
+    # a stage stride that is not a power of two: the promise is not used, the result is the same
+    p = util.pipeline(inputs.chain_edges(3), 3, [30, 40, 50])
+    n = 60_000
+    ctx = np.sort(rng.integers(0, 3, size=n))
+    st = util.state(3, 3, inputs.n_slots(p), 100, 2)
+    wl3 = inputs.Workload("odd", [p], util.requests(rng.integers(100, 5000, size=n), stage=rng.integers(0, 3, size=n), ctx=ctx), st, 3)
+    grouped(wl3)
+
+
+def test_grouped_contexts_larger_than_a_tile_full_size():
+    grouped(inputs.make("C5"))
+
+
 def test_block_per_ctx_full_size():
     grouped(inputs.make("C4"))
 
@@ -433,10 +471,6 @@ def test_broken_grouping_promise_is_reported():
         rc, _ = run_library(wl, pb.PARD_MODE_GROUPED, check=False)
         assert rc == pb.PARD_EDATA, breach
     grouped(inputs.make("C4b", n_epochs=700, per_epoch=600))
-    # more requests than the contexts could hold: refused before anything is launched
-    big = inputs.make("C5b", n_inst=2, per_inst=9000)
-    rc, _ = run_library(big, pb.PARD_MODE_GROUPED, check=False)
-    assert rc == pb.PARD_EINVAL
     # input errors inside a block-planned ctx
     wl = inputs.make("C1b")
     wl.requests["stage"][100] = 7

@@ -1703,7 +1703,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
           uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
           uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
           uint32_t force_scan, const uint32_t* __restrict__ hist, uint32_t sbits, uint32_t local_candidate,
-          uint32_t tables) {
+          uint32_t tables, uint32_t* __restrict__ seg_kept) {
   pdl_wait();
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1769,7 +1769,7 @@ k_seg_win(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
       if (k > 0) a = p_below + 1;
       if (k < 32) b = p_at;
     }
-    if (lane == 0) { win_off[s] = a - lo[0]; win_cnt[s] = 0; }
+    if (lane == 0) { win_off[s] = a - lo[0]; win_cnt[s] = 0; seg_kept[s] = a - lo[0]; }   /* the kept prefix is the queue's kept count */
     return;
   }
   /* batch windows of the queue: 0..b_last of its requests, plus the end marker */
@@ -1815,7 +1815,7 @@ k_seg_win_many(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
                const PardSegConst* __restrict__ ktab, uint32_t* __restrict__ seg_off,
                uint32_t* __restrict__ out_seg_off, uint32_t* __restrict__ win_off, uint32_t* __restrict__ win_cnt,
                uint32_t* __restrict__ win_own, uint32_t* __restrict__ win_big, uint32_t capacity,
-               uint32_t force_scan, uint32_t tables) {
+               uint32_t force_scan, uint32_t tables, uint32_t* __restrict__ seg_kept) {
   pdl_wait();
   const uint32_t warp_g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t lane = threadIdx.x & 31;
@@ -1857,6 +1857,7 @@ k_seg_win_many(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
         if (mid - lo < threshold_u(slack_of((__ldg(src + mid) >> ibits) & dmask, K), K)) a = mid + 1; else b = mid;
       }
       win_off[s] = a - lo;
+      seg_kept[s] = a - lo;                      /* the kept prefix is the queue's kept count */
       win_cnt[s] = 0;
     } else {
       const long long X = (long long)((src[end - 1] >> ibits) & dmask) - K.A_rel;   /* latest deadline of the queue */
@@ -1886,12 +1887,12 @@ k_seg_win_many(PlanHeader* hdr, const unsigned long long* __restrict__ buf_a,
 
 /* E and Kp of the table entries of one queue: the warp runs over the queue's windows, 32 at a
  * time. */
-__device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* __restrict__ ktab,
+__device__ __forceinline__ uint32_t win_prefix_warp(uint32_t s, const PardSegConst* __restrict__ ktab,
                                                 const uint32_t* __restrict__ win_off,
                                                 const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab,
-                                                uint32_t lane) {
+                                                uint32_t lane, uint32_t raw) {
   const uint32_t w0 = win_off[s], cnt = win_cnt[s];
-  if (cnt == 0) return;
+  if (cnt == 0) return 0xffffffffu;              /* no table (served high budget first, or no such stage) */
   const uint32_t cap = ktab[s].cap;
   WinEntry* tab = wtab + w0;
   const uint32_t P0 = __ldcg(&tab[0].P);          /* other blocks may have written the P (long queues) */
@@ -1922,6 +1923,12 @@ __device__ __forceinline__ void win_prefix_warp(uint32_t s, const PardSegConst* 
     e_carry = __shfl_sync(0xffffffffu, e_inc, 31);
     k_carry = __shfl_sync(0xffffffffu, k_inc, 31);
   }
+  /* With the table complete the queue's number of kept requests is known before any request has
+   * been decided: the last entry closes the queue (P = its length n), the running Kp counts the
+   * kept requests under raw positions, and the running E is the minimum of u_t - t over the whole
+   * queue, so that the admitted count behind the last request is n - 1 + min(E, 1). */
+  const uint32_t n_q = __ldcg(&tab[cnt - 1].P);
+  return n_q == 0 ? 0u : (raw ? k_carry : (uint32_t)((int32_t)n_q - 1 + min(e_carry, 1)));
 }
 
 /* The window tables.  P of every entry: a search in the queue's sorted elements, by one lane
@@ -1935,7 +1942,7 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
              const PardSegConst* __restrict__ ktab, const uint32_t* __restrict__ seg_off,
              const uint32_t* __restrict__ win_off, const uint32_t* __restrict__ win_cnt,
              const uint32_t* __restrict__ win_own, const uint32_t* __restrict__ win_big,
-             uint32_t* __restrict__ win_done, WinEntry* __restrict__ wtab) {
+             uint32_t* __restrict__ win_done, WinEntry* __restrict__ wtab, uint32_t raw, uint32_t* __restrict__ seg_kept) {
   pdl_wait();
   if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t lane = threadIdx.x & 31;
@@ -1988,7 +1995,8 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
     }
     if (__shfl_sync(0xffffffffu, last, 0)) {
       __threadfence();
-      win_prefix_warp(s, ktab, win_off, win_cnt, wtab, lane);
+      const uint32_t kept = win_prefix_warp(s, ktab, win_off, win_cnt, wtab, lane, raw);
+      if (lane == 0 && kept != 0xffffffffu) seg_kept[s] = kept;
     }
   }
 }
@@ -1998,13 +2006,15 @@ k_win_bounds(const PlanHeader* __restrict__ hdr, const unsigned long long* __res
 __global__ void __launch_bounds__(256)
 k_win_prefix(const PlanHeader* __restrict__ hdr, uint32_t n_seg, const PardSegConst* __restrict__ ktab,
              const uint32_t* __restrict__ seg_off, const uint32_t* __restrict__ win_off,
-             const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab) {
+             const uint32_t* __restrict__ win_cnt, WinEntry* __restrict__ wtab, uint32_t raw,
+             uint32_t* __restrict__ seg_kept) {
   pdl_wait();
   if (hdr->use_scan || hdr->wide || hdr->aborted) return;
   const uint32_t s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (s >= n_seg) return;                          /* whole warps leave together */
   if (seg_off[s + 1] - seg_off[s] > kWinLongQueue) return;   /* done by k_win_bounds */
-  win_prefix_warp(s, ktab, win_off, win_cnt, wtab, threadIdx.x & 31);
+  const uint32_t kept = win_prefix_warp(s, ktab, win_off, win_cnt, wtab, threadIdx.x & 31, raw);
+  if ((threadIdx.x & 31) == 0 && kept != 0xffffffffu) seg_kept[s] = kept;     /* the queue's kept count, known before the decision */
 }
 
 /* The window tables of a call with few queues, from the counts k_pack took: P is the running sum
@@ -2058,16 +2068,8 @@ k_win_from_counts(PlanHeader* hdr, uint32_t n_seg, const PardSegConst* __restric
     __threadfence_block();
     __syncwarp();
     /* P as the decision reads it: entry b = requests in windows below b, i.e. the sum up to entry b */
-    win_prefix_warp(q, ktab, win_off, win_cnt, wtab, lane);
-    /* With the tables complete the queue's number of kept requests is known before any request
-     * has been decided: the last entry closes the queue (P = its length), its Kp counts the kept
-     * requests under raw positions, and its E is the minimum of u_t - t over the whole queue, so
-     * that the admitted count after the last request is n - 1 + min(E, 1). */
-    if (lane == 0) {
-      __threadfence_block();
-      const WinEntry last = wtab[off + cnt - 1];
-      s_kept[q] = run == 0 ? 0u : (raw ? last.Kp : (uint32_t)((int32_t)run - 1 + min(last.E, 1)));
-    }
+    const uint32_t kept = win_prefix_warp(q, ktab, win_off, win_cnt, wtab, lane, raw);
+    if (lane == 0) s_kept[q] = kept == 0xffffffffu ? 0u : kept;      /* the queue's kept count, known before the sort */
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -3171,10 +3173,10 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     launch_pdl(k_wide_done, 1, 1, 0, stream, hdr, sbits);
     if (L.n_seg >= kManyQueues)
       launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
-                 seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity, 0u, 0u);
+                 seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity, 0u, 0u, seg_kept);
     else
       launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
-                 out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity, 0u, (const uint32_t*)hist, sbits, 0u, 0u);
+                 out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity, 0u, (const uint32_t*)hist, sbits, 0u, 0u, seg_kept);
     PolicyArgs pa = {};
     pa.hdr = hdr; pa.buf_a = buf_a; pa.buf_b = buf_b;
     pa.n = n32; pa.ibits = ibits; pa.n_seg = L.n_seg; pa.mode = mode;
@@ -3255,31 +3257,28 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     if (L.n_seg >= kManyQueues)
       launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
                  seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-                 (mode & PARD_MODE_SCAN) ? 1u : 0u, 1u);
+                 (mode & PARD_MODE_SCAN) ? 1u : 0u, 1u, seg_kept);
     else
       launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
                  out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-                 (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits, 1u, 1u);
+                 (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, sbits, 1u, 1u, seg_kept);
     uint32_t* tmp = out->d_kept_idx ? kept_tmp : nullptr;
     long long* est = (long long*)out->d_est_us;
     const bool raw = mode & PARD_MODE_RAW;
     launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream,
-        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
-    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab);
+        hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab, raw ? 1u : 0u, seg_kept);
+    launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab, raw ? 1u : 0u, seg_kept);
+    launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+               (unsigned long long*)out->d_n_kept);
     auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
                           : (state->d_priority ? k_decide_win<false, true> : k_decide_win<false, false>);
     launch_pdl(decide_win, (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile), kDecThreads, 0, stream, hdr, buf_a, buf_b, n32,
-               ibits, ktab, seg_off, win_off, win_cnt, wtab, out->d_keep, est, out->d_perm, tmp, (const uint32_t*)seg_off, seg_kept);
+               ibits, ktab, seg_off, win_off, win_cnt, wtab, out->d_keep, est, out->d_perm, out->d_kept_idx,
+               (const uint32_t*)kept_base, (uint32_t*)nullptr);
     launch_pdl(raw ? k_scan_path<true> : k_scan_path<false>, std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 2), kDecThreads, 0,
                stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off, win_off, tile_agg, tile_carry, out->d_keep, est,
                out->d_perm, tmp, seg_kept, kept_base, chunk_base, out->d_seg_kept, (unsigned long long*)out->d_n_kept,
                out->d_kept_idx, 0u);
-    launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
-               (unsigned long long*)out->d_n_kept);
-    if (out->d_kept_idx)
-      launch_pdl(k_kept_move, std::min<uint32_t>(((uint32_t)((n + kCompactChunk - 1) / kCompactChunk) + L.n_seg + 7) / 8,
-                                                 (uint32_t)sms * 8), 256, 0, stream,
-                 kept_tmp, seg_off, seg_kept, kept_base, chunk_base, L.n_seg, out->d_kept_idx);
     while (phase <= PARD_N_PHASES) mark();
     PARD_CUDA_OK(cudaGetLastError());
     if (mode & PARD_MODE_NOWAIT) return PARD_OK;
@@ -3359,11 +3358,11 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   } else if (L.n_seg >= kManyQueues)
     launch_pdl(k_seg_win_many, ((L.n_seg + 31) / 31 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab,
                seg_off, out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-               (mode & PARD_MODE_SCAN) ? 1u : 0u, rule_walk ? 0u : 1u);
+               (mode & PARD_MODE_SCAN) ? 1u : 0u, rule_walk ? 0u : 1u, seg_kept);
   else
     launch_pdl(k_seg_win, (L.n_seg + 1 + 7) / 8, 256, 0, stream, hdr, buf_a, buf_b, n32, ibits, L.n_seg, ktab, seg_off,
                out->d_seg_offsets, win_off, win_cnt, win_own, win_big, L.win_capacity,
-               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, ctx_sort ? 64u : sbits, local_cand, rule_walk ? 0u : 1u);
+               (mode & PARD_MODE_SCAN) ? 1u : 0u, (const uint32_t*)hist, ctx_sort ? 64u : sbits, local_cand, rule_walk ? 0u : 1u, seg_kept);
   if (n > 0 && rule_walk) {
     /* a rule without rising thresholds: every queue is walked in order (pard_policy.cu) */
     PolicyArgs pa = {};
@@ -3383,17 +3382,19 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
     /* window tables, and the decision from them */
     if (!win_hist) {
       launch_pdl(k_win_bounds, std::min<uint32_t>((L.win_capacity + 7) / 8, (uint32_t)sms * 8), 256, 0, stream,
-          hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab);
-      launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab);
+          hdr, buf_a, buf_b, ibits, L.n_seg, ktab, seg_off, win_off, win_cnt, win_own, win_big, win_done, wtab, raw ? 1u : 0u, seg_kept);
+      launch_pdl(k_win_prefix, (L.n_seg + 7) / 8, 256, 0, stream, hdr, L.n_seg, ktab, seg_off, win_off, win_cnt, wtab, raw ? 1u : 0u, seg_kept);
+      /* the tables give every queue's kept count: the output offsets are known before the decision */
+      launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
+                 (unsigned long long*)out->d_n_kept);
     }
     mark();
     const uint32_t win_grid = (uint32_t)((n + (uint64_t)kDecTile - 1) / kDecTile);
     auto decide_win = raw ? (state->d_priority ? k_decide_win<true, true> : k_decide_win<true, false>)
                           : (state->d_priority ? k_decide_win<false, true> : k_decide_win<false, false>);
-    /* counted tables: the queues' kept counts are known, the survivors go straight to the output */
+    /* the survivors go straight to their place in the output */
     launch_pdl(decide_win, win_grid, kDecThreads, 0, stream, hdr, buf_a, buf_b, n32, ibits, ktab, seg_off, win_off, win_cnt, wtab,
-               out->d_keep, est, out->d_perm, win_hist ? out->d_kept_idx : tmp,
-               win_hist ? (const uint32_t*)kept_base : (const uint32_t*)seg_off, win_hist ? (uint32_t*)nullptr : seg_kept);
+               out->d_keep, est, out->d_perm, out->d_kept_idx, (const uint32_t*)kept_base, (uint32_t*)nullptr);
     /* fallback when a queue has too many batch windows: the same decision by scanning, one kernel
      * that returns at once otherwise */
     const uint32_t scan_grid = std::min<uint32_t>(L.dec_tiles, (uint32_t)sms * 2);
@@ -3404,7 +3405,7 @@ extern "C" int pard_plan_policy(const pard_pipeline_t* const* pipelines, uint32_
   }
   if (n == 0) mark();
   mark();
-  if (!win_hist) {                                 /* with counted tables this was known before the sort */
+  if (rule_walk || n == 0) {                       /* the queue walk leaves per-queue lists; an empty call still owes its zeros */
     launch_pdl(k_kept_scan, 1, 1024, 0, stream, seg_kept, L.n_seg, kept_base, chunk_base, out->d_seg_kept,
                (unsigned long long*)out->d_n_kept);
     if (n > 0 && out->d_kept_idx)
@@ -3439,8 +3440,8 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
    * most a sort tile: one kernel.  Else always clear and seg_const; with many queues also
    * key_width (and, when n > 0, ctx_span); when n > 0: prepass, pack, the radix passes, decide_win
    * and the scan path (one kernel that returns at once); with at most 64 queues the counted window
-   * tables (win_from_counts), else the queue boundaries and searched tables (seg_win, win_bounds,
-   * win_prefix) and the packing of the survivors (kept_scan, kept_move). */
+   * tables (win_from_counts), else the queue boundaries, the searched tables and the output
+   * offsets that follow from them (seg_win, win_bounds, win_prefix, kept_scan). */
   const uint64_t n_seg = (uint64_t)n_ctx * (uint64_t)stage_stride;
   const uint32_t width_kernels = n_seg <= kFoldSegs ? 0 : 1;   /* key_width (+ ctx_span when n > 0) */
   const bool local_cand = local_sort_candidate(n, n_ctx);
@@ -3449,7 +3450,7 @@ extern "C" int pard_plan_kernel_launches(uint64_t n, uint32_t n_ctx, int32_t sta
   const bool counted = n > 0 && n_seg <= kHistSegs && !local_cand;
   if (n_ctx == 1 && n > 0 && n <= (uint64_t)kSortTile) *launches = 1;
   else if (n == 0) *launches = 4 + width_kernels;               /* clear, (key_width,) seg_const, seg_win, kept_scan */
-  else *launches = 2 + 2 * width_kernels + 2 + local_kernels + passes + 2 + (counted ? 1 : 5);
+  else *launches = 2 + 2 * width_kernels + 2 + local_kernels + passes + 2 + (counted ? 1 : 4);
   return PARD_OK;
 }
 

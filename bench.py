@@ -722,7 +722,13 @@ def run_ours(args):
                 others[name] = {"requests": wlo.n, "contexts": wlo.n_ctx, "us_per_step": 1e6 * so / 50,
                                 "requests_per_s": wlo.n * 50 / so, "keep_fraction": kfo,
                                 "mode": "PARD_MODE_GROUPED" if name in ("C4", "C5") else "default"}
-                del plo, wlo
+                del plo
+                if name in ("C4", "C5"):                  # and without the caller's word, for comparison
+                    plo = DevicePlan(wlo, dev, 0)
+                    so, _ = timed_steps(plo, 50, 5, None)
+                    others[name]["us_per_step_without_the_promise"] = 1e6 * so / 50
+                    del plo
+                del wlo
             # the many-context workloads also against the oracle on all host cores (bounded samples)
             others["C4"]["cpu_baseline_all_cores"] = oracle_all_cores("C4", {"n_epochs": 512, "per_epoch": 8192})
             others["C5"]["cpu_baseline_all_cores"] = oracle_all_cores("C5", {"n_inst": 64, "per_inst": 65536})

@@ -193,7 +193,7 @@ typedef struct pard_plan_out {
                                      promise then includes that NO ctx holds more than
                                      8,192.  Up to a few hundred contexts one thread block
                                      plans each ctx from start to end in shared memory --
-                                     constants, sort, positions, decisions -- in five
+                                     constants, sort, positions, decisions -- in six
                                      kernel launches instead of about twenty, two to three
                                      times faster on small and medium calls; beyond that a
                                      block per ctx reads, checks and sorts its ctx and the

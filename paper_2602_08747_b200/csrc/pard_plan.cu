@@ -1289,7 +1289,9 @@ __device__ __forceinline__ TileCtx make_tile_ctx(const PlanHeader* hdr, const un
   T.imask = (1u << ibits) - 1;                                 /* ibits <= 30 */
   T.kshift = ibits + dbits;                                    /* < 64 */
   T.dmask = dbits >= 64 ? ~0ull : ((1ull << dbits) - 1);
-  T.narrow = dbits <= 29;
+  /* the offsets that occur, not the field they sit in (a call whose element format is fixed by
+   * the host may have a wider field than its deadline spans need) */
+  T.narrow = dbits <= 29 || (hdr->span_max >> 29) == 0;
   T.hdr = const_cast<PlanHeader*>(hdr);
   return T;
 }

